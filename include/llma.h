@@ -1,0 +1,198 @@
+/*
+ * llma.h -- C ABI of the LLMA reference-copy decoding engine for one NVIDIA B200 (sm_100a).
+ *
+ * LLMA ("inference with reference", arXiv 2304.04487) speeds up greedy decoding when the
+ * output shares token spans with reference documents.  At every decoding step the last n
+ * generated tokens are matched against the references (Section 2.2); on a match the k
+ * tokens that follow it are copied into the decoder input and all k+1 positions are
+ * evaluated in ONE causal forward pass (Eq. 3); the longest prefix of copied tokens that
+ * agrees with the model's own argmax outputs is kept, plus one more output token
+ * (Algorithm 1).  The result is token-for-token what greedy decoding (Eq. 2)
+ * produces.
+ *
+ * Every step of that path -- trigger search, copy + embedding gather, the decoder layers
+ * (RMSNorm, QKV projection + rotary embedding + K/V append, causal attention over the K/V
+ * cache, output projection, SiLU-gated feed-forward), LM head + per-row argmax, acceptance
+ * and K/V commit -- runs in CUDA kernels of this library.  There is no CPU fallback: every
+ * entry point fails with LLMA_ERR_CUDA if no usable device is present.
+ *
+ * Conventions
+ *   - All functions return 0 (LLMA_OK) or a negative llma_status; nothing throws or aborts.
+ *     After an argument error the engine is unchanged and usable.
+ *   - "device" pointers are CUDA device pointers valid on the engine's device; "host"
+ *     pointers are ordinary process memory.  The library never frees caller memory.
+ *   - Weight matrices are row-major [out_features, in_features] with no padding, fp32
+ *     (dtype LLMA_DTYPE_F32) or bf16 (LLMA_DTYPE_BF16); norm gains are always fp32.  The
+ *     engine BORROWS them: keep them alive and unmodified until llma_destroy.
+ *   - Token ids are int32 in [0, vocab).
+ *   - Calls on one engine must not overlap in time; different engines are independent.
+ */
+#ifndef LLMA_H_
+#define LLMA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct llma_engine llma_engine; /* opaque */
+
+typedef enum {
+    LLMA_OK = 0,
+    LLMA_ERR_NULL = -1,           /* a required pointer was NULL */
+    LLMA_ERR_CONFIG = -2,         /* unsupported or inconsistent llma_config */
+    LLMA_ERR_TOKEN_RANGE = -3,    /* a token id outside [0, vocab) */
+    LLMA_ERR_CAPACITY = -4,       /* sequence would exceed max_seq, or batch index out of range */
+    LLMA_ERR_REF_TOO_LONG = -5,   /* reference longer than max_ref or malformed doc_offsets */
+    LLMA_ERR_STATE = -6,          /* call not valid in the sequence's current state */
+    LLMA_ERR_CUDA = -7,           /* a CUDA call failed (llma_last_cuda_error has the code) */
+    LLMA_ERR_DEVICE_TIMEOUT = -8, /* a bounded on-device wait ran out; the step's results are void */
+    LLMA_ERR_ARG = -9             /* n < 1, k outside [0, max_k], max_new < 0 ... */
+} llma_status;
+
+enum { LLMA_DTYPE_F32 = 0, LLMA_DTYPE_BF16 = 1 };
+enum { LLMA_GEMM_AUTO = 0, LLMA_GEMM_SIMT = 1, LLMA_GEMM_TCGEN05 = 2 };
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t dtype;        /* storage type of weights and K/V cache: LLMA_DTYPE_* */
+    int32_t max_batch;    /* sequences held at once; max_batch * (max_k + 1) must be <= 32 */
+    int32_t max_seq;      /* K/V rows per sequence */
+    int32_t max_ref;      /* reference tokens per sequence */
+    int32_t max_k;        /* largest copy length k that will be requested (0..31) */
+    float rms_eps;        /* RMSNorm epsilon */
+    float rope_theta;     /* rotary base; pairing is (i, i + head_dim/2) */
+    int32_t eos_id;       /* -1: none.  Otherwise a sequence stops after emitting this id */
+    int32_t gemm_impl;    /* LLMA_GEMM_*; AUTO = tensor-core kernels for bf16, SIMT for fp32 */
+    int32_t keep_logits;  /* 1: keep the last step's logits for llma_debug_logits */
+} llma_config;
+
+/* Device pointers.  Per-layer arrays are HOST arrays of n_layers device pointers. */
+typedef struct {
+    const void *tok_emb;           /* [vocab, d_model] */
+    const void *lm_head;           /* [vocab, d_model] */
+    const float *final_norm;       /* [d_model] */
+    const float *const *attn_norm; /* [d_model] each */
+    const void *const *wq;         /* [n_heads*head_dim, d_model] each */
+    const void *const *wk;
+    const void *const *wv;
+    const void *const *wo;         /* [d_model, n_heads*head_dim] */
+    const float *const *ffn_norm;  /* [d_model] */
+    const void *const *w_gate;     /* [d_ffn, d_model] */
+    const void *const *w_up;       /* [d_ffn, d_model] */
+    const void *const *w_down;     /* [d_model, d_ffn] */
+} llma_weights;
+
+/* Decode statistics of Section 4.2 (triggers, accepted copied tokens, decoding steps),
+ * summed over the sequences of the last llma_generate call, plus device time. */
+typedef struct {
+    int64_t steps;            /* decoding steps taken (forward passes), per-sequence sum */
+    int64_t trigger_steps;    /* steps in which a copy was applied */
+    int64_t copied_accepted;  /* copied tokens that survived verification */
+    int64_t tokens;           /* tokens emitted = steps + copied_accepted */
+    int64_t launches;         /* kernels launched by this library during the call */
+    float device_ms;          /* CUDA-event time from first to last kernel of the call */
+} llma_stats;
+
+/* Per-sequence record of the most recent step (for tests and tracing). */
+typedef struct {
+    int32_t pos;       /* first copied reference index, -1 when nothing was copied */
+    int32_t k_eff;     /* copied tokens fed to the model */
+    int32_t accepted;  /* copied tokens kept */
+    int32_t emitted;   /* tokens appended this step (0 if the sequence was idle) */
+} llma_step_info;
+
+/*
+ * Create an engine on the current CUDA device.  `cuda_stream` is a cudaStream_t (may be
+ * NULL for the default stream); all work of the engine is issued on it.  Allocates the K/V
+ * cache ([layer][seq][head][max_seq][head_dim], zero-filled), reference storage and
+ * workspaces.  Supported: head_dim 64 or 128; d_model, n_heads*head_dim and d_ffn multiples
+ * of 64; max_batch*(max_k+1) <= 32.  Errors: NULL, CONFIG, CUDA.
+ */
+int llma_create(const llma_config *cfg, const llma_weights *w, void *cuda_stream, llma_engine **out);
+
+/* Free everything the engine owns (synchronises the stream first).  NULL is allowed. */
+int llma_destroy(llma_engine *e);
+
+/*
+ * Load a prompt x (host, n_prompt >= 1 tokens) into sequence slot `seq`: positions
+ * 0..n_prompt-2 are pushed through the decoder and cached; the last prompt token becomes
+ * the pending input of the first decoding step (Algorithm 1 starts with y empty and calls
+ * the model inside its loop, so prefill emits nothing).  Clears the sequence's output and
+ * statistics; keeps its reference.  Synchronous.  Errors: NULL, CAPACITY, TOKEN_RANGE, CUDA.
+ */
+int llma_prefill(llma_engine *e, int32_t seq, const int32_t *prompt, int32_t n_prompt);
+
+/*
+ * Set the reference documents D of a sequence (Section 2.2): `tokens` (host, n_tokens ids)
+ * is the concatenation of n_docs documents; doc_offsets (host, n_docs+1 non-decreasing
+ * values from 0 to n_tokens) delimits them, or NULL for a single document.  Neither the
+ * matched n-gram nor the copied span crosses a document boundary.  n_tokens = 0 clears the
+ * reference (plain greedy).  Copied to the device during the call.
+ * Errors: NULL, REF_TOO_LONG, TOKEN_RANGE, CAPACITY, CUDA.
+ */
+int llma_set_reference(llma_engine *e, int32_t seq, const int32_t *tokens, int32_t n_tokens,
+                       const int32_t *doc_offsets, int32_t n_docs);
+
+/*
+ * One iteration of Algorithm 1's loop body for every prefilled, unfinished sequence:
+ * trigger search with match length n >= 1, copy of up to k (0 <= k <= max_k) tokens, one
+ * (k+1)-row forward pass, acceptance, K/V commit.  Synchronous.  out_tokens (host,
+ * [max_batch][max_k+1]) receives each sequence's new tokens, n_out (host, [max_batch]) how
+ * many (0 for idle slots).  The copy is additionally capped so the sequence never exceeds
+ * max_seq.  k = 0 or an empty reference is a plain greedy step (Eq. 2).
+ * Errors: NULL, ARG, STATE (no sequence prefilled), CAPACITY, CUDA, DEVICE_TIMEOUT.
+ */
+int llma_step(llma_engine *e, int32_t n, int32_t k, int32_t *out_tokens, int32_t *n_out);
+
+/*
+ * Algorithm 1's whole loop: decode exactly max_new further tokens for every prefilled
+ * sequence (fewer only if eos_id is hit), with no host involvement inside a step and no
+ * per-step host synchronisation.  out_tokens (host, [max_batch][max_new]) and n_out (host,
+ * [max_batch]) receive the tokens; stats may be NULL.  The copy length of a step is
+ * k_eff = min(k, tokens left in the matched document, tokens still to emit - 1), so exactly
+ * max_new tokens come out.  Requires kv_len + max_new <= max_seq for every active sequence.
+ * Errors: NULL, ARG, STATE, CAPACITY, CUDA, DEVICE_TIMEOUT.
+ */
+int llma_generate(llma_engine *e, int32_t max_new, int32_t n, int32_t k, int32_t *out_tokens,
+                  int32_t *n_out, llma_stats *stats);
+
+/*
+ * Roll a sequence back to the state right after llma_prefill (output emptied, K/V length
+ * reset to n_prompt-1; the cached prompt rows are reused, later rows are overwritten by the
+ * next steps).  Lets several decodes share one prefill.  Errors: CAPACITY, STATE, CUDA.
+ */
+int llma_rewind(llma_engine *e, int32_t seq);
+
+/* Forget a sequence entirely (slot becomes idle; its reference is cleared). */
+int llma_reset(llma_engine *e, int32_t seq);
+
+/* Record of the last step for each sequence: info is a host array [max_batch]. */
+int llma_last_step_info(llma_engine *e, llma_step_info *info);
+
+/*
+ * Parity harness only (requires keep_logits = 1): copy the logits of the last step to
+ * `out` (host, [rows][vocab] fp32) where row j of sequence s is at index s*(max_k+1)+j and
+ * rows is max_batch*(max_k+1).  Rows that were not part of the step hold stale values.
+ * Errors: NULL, STATE, CUDA.
+ */
+int llma_debug_logits(llma_engine *e, float *out);
+
+/* Parity harness only: copy K (which=0) or V (which=1) cache row `pos` of a layer and
+ * sequence to `out` (host, [n_heads*head_dim] fp32, widened exactly).  Errors: ARG, CUDA. */
+int llma_debug_kv_row(llma_engine *e, int32_t layer, int32_t seq, int32_t pos, int32_t which, float *out);
+
+/* Committed K/V length of a sequence (prompt rows + emitted tokens - 1), or a negative status. */
+int llma_kv_len(llma_engine *e, int32_t seq);
+
+/* The CUDA error code behind the most recent LLMA_ERR_CUDA on this thread (0 if none). */
+int llma_last_cuda_error(void);
+
+/* Static description of a status code. */
+const char *llma_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLMA_H_ */

@@ -1,0 +1,63 @@
+// Shared declarations of the LLMA engine's CUDA translation units (library-private).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace llma {
+
+constexpr int kMaxRows = 32;  // query rows of one forward pass (all sequences together)
+
+// Per-sequence decoding state, resident in device memory.  Field order is mirrored by the
+// host when it reads the array back.
+struct SeqState {
+    int32_t active;      // 1 after prefill
+    int32_t done;        // 1 once target_len (or EOS) is reached
+    int32_t kv_len;      // committed K/V rows
+    int32_t pending;     // newest token, not yet in the cache: input row 0 of the next step
+    int32_t y_len;       // tokens emitted so far
+    int32_t target_len;  // stop once y_len reaches this
+    int32_t ref_len;     // reference tokens stored for this sequence
+    int32_t prompt_len;
+    int32_t pos, k_eff, nrows;  // plan of the step in flight
+    int32_t last_pos, last_k_eff, last_accepted, last_emitted;
+    int32_t steps, trigger_steps, copied_accepted;
+};
+
+// One forward pass works on up to kMaxRows rows; these arrays say what each row is.
+struct RowDesc {
+    int32_t tok[kMaxRows];  // input token id
+    int32_t pos[kMaxRows];  // absolute position in its sequence, -1 = row unused
+    int32_t seq[kMaxRows];  // sequence slot
+    int32_t rows_used;      // 1 + highest used row index (0 = nothing to do)
+    int32_t max_pos;        // highest position among used rows (-1 if none)
+};
+
+enum : int32_t {
+    kDevErrNone = 0,
+    kDevErrTimeout = 1,   // a bounded wait ran out
+    kDevErrCapacity = 2,  // a step would have written past max_seq
+    kDevErrToken = 3,     // a token id out of range reached the device
+};
+
+struct ModelDims {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t hd_total;  // n_heads * head_dim
+    int32_t max_batch, max_seq, max_ref, kp1;  // kp1 = max_k + 1 rows reserved per sequence
+    float rms_eps;
+    int32_t eos_id;
+};
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// K/V cache addressing: [layer][seq][head][max_seq][head_dim]; returns the row index
+__host__ __device__ __forceinline__ int64_t kv_row_index(const ModelDims& d, int layer, int seq, int head, int pos) {
+    return ((((int64_t)layer * d.max_batch + seq) * d.n_heads + head) * d.max_seq + pos);
+}
+
+}  // namespace llma
