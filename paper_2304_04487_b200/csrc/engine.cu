@@ -1,0 +1,167 @@
+// C ABI of the LLMA engine: object lifetime, prompt prefill, reference upload, the decoding
+// step (Algorithm 1's loop body) and the whole decoding loop.  See include/llma.h.
+#include "engine.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+
+using namespace llma;
+
+static thread_local int g_last_cuda_error = 0;
+void llma::note_cuda_error(cudaError_t err) {
+    g_last_cuda_error = (int)err;
+    (void)cudaGetLastError();
+}
+
+static size_t esize(const llma_engine* e) { return e->bf16 ? 2 : 4; }
+
+template <typename T>
+static cudaError_t dalloc(T** p, size_t count, bool zero = true) {
+    cudaError_t r = cudaMalloc((void**)p, count * sizeof(T));
+    if (r != cudaSuccess) return r;
+    if (zero) r = cudaMemset(*p, 0, count * sizeof(T));
+    return r;
+}
+
+extern "C" int llma_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" const char* llma_strerror(int s) {
+    switch (s) {
+        case LLMA_OK: return "ok";
+        case LLMA_ERR_NULL: return "required pointer is NULL";
+        case LLMA_ERR_CONFIG: return "unsupported or inconsistent configuration";
+        case LLMA_ERR_TOKEN_RANGE: return "token id outside [0, vocab)";
+        case LLMA_ERR_CAPACITY: return "sequence capacity (max_seq / max_batch) exceeded";
+        case LLMA_ERR_REF_TOO_LONG: return "reference too long or malformed document offsets";
+        case LLMA_ERR_STATE: return "call not valid in the current state";
+        case LLMA_ERR_CUDA: return "CUDA call failed";
+        case LLMA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+        case LLMA_ERR_ARG: return "argument out of range";
+        default: return "unknown status";
+    }
+}
+
+static void free_engine(llma_engine* e) {
+    if (!e) return;
+    for (auto& kv : e->step_graphs) cudaGraphExecDestroy(kv.second);
+    cudaFree(e->seq_state); cudaFree(e->rows); cudaFree(e->ref); cudaFree(e->doc_start); cudaFree(e->doc_end);
+    cudaFree(e->y); cudaFree(e->out_tok); cudaFree(e->dev_err); cudaFree(e->x); cudaFree(e->qkv);
+    cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
+    cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
+    if (e->h_state) cudaFreeHost(e->h_state);
+    if (e->h_rows) cudaFreeHost(e->h_rows);
+    if (e->h_err) cudaFreeHost(e->h_err);
+    if (e->ev0) cudaEventDestroy(e->ev0);
+    if (e->ev1) cudaEventDestroy(e->ev1);
+    delete e;
+}
+
+extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* cuda_stream, llma_engine** out) {
+    if (!cfg || !w || !out) return LLMA_ERR_NULL;
+    *out = nullptr;
+    const int L = cfg->n_layers;
+    if (L < 1 || cfg->d_model < 64 || cfg->n_heads < 1 || cfg->d_ffn < 64 || cfg->vocab < 2) return LLMA_ERR_CONFIG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return LLMA_ERR_CONFIG;
+    const int HD = cfg->n_heads * cfg->head_dim;
+    if (cfg->d_model % 64 || HD % 64 || cfg->d_ffn % 64) return LLMA_ERR_CONFIG;
+    if (cfg->dtype != LLMA_DTYPE_F32 && cfg->dtype != LLMA_DTYPE_BF16) return LLMA_ERR_CONFIG;
+    if (cfg->max_batch < 1 || cfg->max_k < 0 || cfg->max_batch * (cfg->max_k + 1) > kMaxRows) return LLMA_ERR_CONFIG;
+    if (cfg->max_seq < 2 || cfg->max_ref < 0 || !(cfg->rms_eps >= 0.f) || !(cfg->rope_theta > 0.f)) return LLMA_ERR_CONFIG;
+    if (cfg->gemm_impl < LLMA_GEMM_AUTO || cfg->gemm_impl > LLMA_GEMM_TCGEN05) return LLMA_ERR_CONFIG;
+    if (cfg->gemm_impl == LLMA_GEMM_TCGEN05 && cfg->dtype != LLMA_DTYPE_BF16) return LLMA_ERR_CONFIG;
+    if (!w->tok_emb || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
+        !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
+        return LLMA_ERR_NULL;
+    for (int l = 0; l < L; ++l)
+        if (!w->attn_norm[l] || !w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->ffn_norm[l] ||
+            !w->w_gate[l] || !w->w_up[l] || !w->w_down[l])
+            return LLMA_ERR_NULL;
+
+    int dev = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    llma_engine* e = new (std::nothrow) llma_engine();
+    if (!e) return LLMA_ERR_CUDA;
+    e->cfg = *cfg;
+    e->device = dev;
+    e->stream = (cudaStream_t)cuda_stream;
+    e->bf16 = cfg->dtype == LLMA_DTYPE_BF16;
+    e->gemm_impl = cfg->gemm_impl == LLMA_GEMM_AUTO ? LLMA_GEMM_SIMT : cfg->gemm_impl;
+    ModelDims& d = e->dims;
+    d.n_layers = L; d.d_model = cfg->d_model; d.n_heads = cfg->n_heads; d.head_dim = cfg->head_dim;
+    d.d_ffn = cfg->d_ffn; d.vocab = cfg->vocab; d.hd_total = HD; d.max_batch = cfg->max_batch;
+    d.max_seq = cfg->max_seq; d.max_ref = cfg->max_ref > 0 ? cfg->max_ref : 1; d.kp1 = cfg->max_k + 1;
+    d.rms_eps = cfg->rms_eps; d.eos_id = cfg->eos_id;
+    e->tok_emb = w->tok_emb; e->lm_head = w->lm_head; e->final_norm = w->final_norm;
+    for (int l = 0; l < L; ++l) {
+        e->attn_norm.push_back(w->attn_norm[l]); e->ffn_norm.push_back(w->ffn_norm[l]);
+        e->wq.push_back(w->wq[l]); e->wk.push_back(w->wk[l]); e->wv.push_back(w->wv[l]); e->wo.push_back(w->wo[l]);
+        e->w_gate.push_back(w->w_gate[l]); e->w_up.push_back(w->w_up[l]); e->w_down.push_back(w->w_down[l]);
+    }
+    e->y_cap = d.max_seq;
+    e->prompt_last.assign((size_t)d.max_batch, 0);
+
+#define CREATE_TRY(expr)                              \
+    do {                                              \
+        cudaError_t _e = (expr);                      \
+        if (_e != cudaSuccess) {                      \
+            llma::note_cuda_error(_e);                \
+            free_engine(e);                           \
+            return LLMA_ERR_CUDA;                     \
+        }                                             \
+    } while (0)
+
+    const size_t B = d.max_batch, es = esize(e);
+    CREATE_TRY(dalloc(&e->seq_state, B));
+    CREATE_TRY(dalloc(&e->rows, 1));
+    CREATE_TRY(dalloc(&e->ref, B * d.max_ref));
+    CREATE_TRY(dalloc(&e->doc_start, B * d.max_ref));
+    CREATE_TRY(dalloc(&e->doc_end, B * d.max_ref));
+    CREATE_TRY(dalloc(&e->y, B * e->y_cap));
+    CREATE_TRY(dalloc(&e->out_tok, (size_t)kMaxRows));
+    CREATE_TRY(dalloc(&e->dev_err, 1));
+    CREATE_TRY(dalloc(&e->x, (size_t)kMaxRows * d.d_model));
+    CREATE_TRY(dalloc(&e->qkv, (size_t)kMaxRows * 3 * HD));
+    CREATE_TRY(dalloc(&e->gate_up, (size_t)kMaxRows * 2 * d.d_ffn));
+    CREATE_TRY(dalloc(&e->logits, (size_t)kMaxRows * d.vocab));
+    CREATE_TRY(dalloc((char**)&e->x_hat, (size_t)kMaxRows * d.d_model * es));
+    CREATE_TRY(dalloc((char**)&e->attn, (size_t)kMaxRows * HD * es));
+    CREATE_TRY(dalloc((char**)&e->h, (size_t)kMaxRows * d.d_ffn * es));
+    const size_t kv_elems = (size_t)L * B * d.n_heads * d.max_seq * d.head_dim;
+    CREATE_TRY(dalloc((char**)&e->kcache, kv_elems * es));
+    CREATE_TRY(dalloc((char**)&e->vcache, kv_elems * es));
+
+    // rotary table: angle(pos, i) = pos * theta^(-2i/hd), evaluated in double on the host
+    {
+        const int half = d.head_dim / 2;
+        std::vector<float> c((size_t)d.max_seq * half), s((size_t)d.max_seq * half);
+        for (int i = 0; i < half; ++i) {
+            const double inv = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)d.head_dim);
+            for (int p = 0; p < d.max_seq; ++p) {
+                const double a = (double)p * inv;
+                c[(size_t)p * half + i] = (float)std::cos(a);
+                s[(size_t)p * half + i] = (float)std::sin(a);
+            }
+        }
+        CREATE_TRY(dalloc(&e->rope_cos, c.size(), false));
+        CREATE_TRY(dalloc(&e->rope_sin, s.size(), false));
+        CREATE_TRY(cudaMemcpy(e->rope_cos, c.data(), c.size() * 4, cudaMemcpyHostToDevice));
+        CREATE_TRY(cudaMemcpy(e->rope_sin, s.data(), s.size() * 4, cudaMemcpyHostToDevice));
+    }
+    CREATE_TRY(cudaMallocHost((void**)&e->h_state, B * sizeof(SeqState)));
+    CREATE_TRY(cudaMallocHost((void**)&e->h_rows, sizeof(RowDesc)));
+    CREATE_TRY(cudaMallocHost((void**)&e->h_err, sizeof(int32_t)));
+    CREATE_TRY(cudaEventCreate(&e->ev0));
+    CREATE_TRY(cudaEventCreate(&e->ev1));
+    CREATE_TRY(cudaDeviceSynchronize());
+#undef CREATE_TRY
+    *out = e;
+    return LLMA_OK;
+}
+
+extern "C" int llma_destroy(llma_engine* e) {
+    if (!e) return LLMA_OK;
+    cudaStreamSynchronize(e->stream);
+    free_engine(e);
+    return LLMA_OK;
+}

@@ -1,0 +1,59 @@
+// Engine object behind the C ABI (library-private).
+#pragma once
+#include <map>
+#include <utility>
+#include <vector>
+
+#include "../../include/llma.h"
+#include "kernels.h"
+
+struct llma_engine {
+    llma_config cfg;
+    llma::ModelDims dims;
+    bool bf16 = false;
+    int gemm_impl = LLMA_GEMM_SIMT;
+    cudaStream_t stream = nullptr;
+    int device = 0;
+
+    // borrowed weights (host copies of the per-layer pointer arrays)
+    const void *tok_emb = nullptr, *lm_head = nullptr;
+    const float* final_norm = nullptr;
+    std::vector<const float*> attn_norm, ffn_norm;
+    std::vector<const void*> wq, wk, wv, wo, w_gate, w_up, w_down;
+
+    // device state
+    llma::SeqState* seq_state = nullptr;
+    llma::RowDesc* rows = nullptr;
+    int32_t *ref = nullptr, *doc_start = nullptr, *doc_end = nullptr, *y = nullptr, *out_tok = nullptr;
+    int32_t* dev_err = nullptr;
+    int32_t y_cap = 0;
+    float *x = nullptr, *qkv = nullptr, *gate_up = nullptr, *logits = nullptr;
+    void *x_hat = nullptr, *attn = nullptr, *h = nullptr;
+    float *rope_cos = nullptr, *rope_sin = nullptr;
+    void *kcache = nullptr, *vcache = nullptr;
+
+    // pinned host staging
+    llma::SeqState* h_state = nullptr;
+    llma::RowDesc* h_rows = nullptr;
+    int32_t* h_err = nullptr;
+
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    std::map<std::pair<int, int>, cudaGraphExec_t> step_graphs;  // keyed by (n, k)
+    int64_t launches_per_step = 0;
+    int64_t launch_counter = 0;  // kernels enqueued since it was last cleared
+    bool last_step_valid = false;
+    std::vector<int32_t> prompt_last;  // last prompt token of every sequence (the first pending input)
+};
+
+namespace llma {
+void note_cuda_error(cudaError_t err);  // remembers the code for llma_last_cuda_error, clears the sticky flag
+}
+
+#define CU_TRY(expr)                          \
+    do {                                      \
+        cudaError_t _e = (expr);              \
+        if (_e != cudaSuccess) {              \
+            llma::note_cuda_error(_e);        \
+            return LLMA_ERR_CUDA;             \
+        }                                     \
+    } while (0)

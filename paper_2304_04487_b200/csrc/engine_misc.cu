@@ -1,0 +1,104 @@
+// Small state-management and inspection entry points of the C ABI.
+#include <cstring>
+#include <vector>
+
+#include "engine.h"
+
+using namespace llma;
+
+static int fetch_state(llma_engine* e) {
+    CU_TRY(cudaMemcpyAsync(e->h_state, e->seq_state, e->dims.max_batch * sizeof(SeqState), cudaMemcpyDeviceToHost,
+                           e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    return LLMA_OK;
+}
+
+static int store_state(llma_engine* e, int seq) {
+    CU_TRY(cudaMemcpyAsync(e->seq_state + seq, e->h_state + seq, sizeof(SeqState), cudaMemcpyHostToDevice, e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    return LLMA_OK;
+}
+
+extern "C" int llma_rewind(llma_engine* e, int32_t seq) {
+    if (!e) return LLMA_ERR_NULL;
+    if (seq < 0 || seq >= e->dims.max_batch) return LLMA_ERR_CAPACITY;
+    int rc = fetch_state(e);
+    if (rc) return rc;
+    SeqState& S = e->h_state[seq];
+    if (!S.active) return LLMA_ERR_STATE;
+    const int32_t ref_len = S.ref_len, plen = S.prompt_len;
+    const int32_t last_tok = e->prompt_last[seq];  // kept on the host by llma_prefill
+    std::memset(&S, 0, sizeof(S));
+    S.active = 1; S.kv_len = plen - 1; S.pending = last_tok; S.ref_len = ref_len; S.prompt_len = plen;
+    S.pos = -1; S.last_pos = -1; S.done = 1;
+    e->last_step_valid = false;
+    return store_state(e, seq);
+}
+
+extern "C" int llma_reset(llma_engine* e, int32_t seq) {
+    if (!e) return LLMA_ERR_NULL;
+    if (seq < 0 || seq >= e->dims.max_batch) return LLMA_ERR_CAPACITY;
+    int rc = fetch_state(e);
+    if (rc) return rc;
+    std::memset(&e->h_state[seq], 0, sizeof(SeqState));
+    e->h_state[seq].pos = -1; e->h_state[seq].last_pos = -1;
+    e->last_step_valid = false;
+    return store_state(e, seq);
+}
+
+extern "C" int llma_last_step_info(llma_engine* e, llma_step_info* info) {
+    if (!e || !info) return LLMA_ERR_NULL;
+    int rc = fetch_state(e);
+    if (rc) return rc;
+    for (int s = 0; s < e->dims.max_batch; ++s) {
+        const SeqState& S = e->h_state[s];
+        info[s].pos = S.last_pos; info[s].k_eff = S.last_k_eff;
+        info[s].accepted = S.last_accepted; info[s].emitted = S.last_emitted;
+    }
+    return LLMA_OK;
+}
+
+extern "C" int llma_debug_logits(llma_engine* e, float* out) {
+    if (!e || !out) return LLMA_ERR_NULL;
+    if (!e->cfg.keep_logits || !e->last_step_valid) return LLMA_ERR_STATE;
+    const size_t rows = (size_t)e->dims.max_batch * e->dims.kp1;
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    CU_TRY(cudaMemcpy(out, e->logits, rows * e->dims.vocab * sizeof(float), cudaMemcpyDeviceToHost));
+    return LLMA_OK;
+}
+
+extern "C" int llma_debug_kv_row(llma_engine* e, int32_t layer, int32_t seq, int32_t pos, int32_t which, float* out) {
+    if (!e || !out) return LLMA_ERR_NULL;
+    const ModelDims& d = e->dims;
+    if (layer < 0 || layer >= d.n_layers || seq < 0 || seq >= d.max_batch || pos < 0 || pos >= d.max_seq ||
+        (which != 0 && which != 1))
+        return LLMA_ERR_ARG;
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    const char* base = (const char*)(which ? e->vcache : e->kcache);
+    const size_t es = e->bf16 ? 2 : 4;
+    std::vector<unsigned char> tmp((size_t)d.head_dim * es);
+    for (int h = 0; h < d.n_heads; ++h) {
+        const size_t off = (size_t)kv_row_index(d, layer, seq, h, pos) * d.head_dim * es;
+        CU_TRY(cudaMemcpy(tmp.data(), base + off, tmp.size(), cudaMemcpyDeviceToHost));
+        for (int i = 0; i < d.head_dim; ++i) {
+            float v;
+            if (e->bf16) {
+                uint32_t u = (uint32_t)(((const uint16_t*)tmp.data())[i]) << 16;
+                std::memcpy(&v, &u, 4);
+            } else {
+                v = ((const float*)tmp.data())[i];
+            }
+            out[(size_t)h * d.head_dim + i] = v;
+        }
+    }
+    return LLMA_OK;
+}
+
+extern "C" int llma_kv_len(llma_engine* e, int32_t seq) {
+    if (!e) return LLMA_ERR_NULL;
+    if (seq < 0 || seq >= e->dims.max_batch) return LLMA_ERR_CAPACITY;
+    int rc = fetch_state(e);
+    if (rc) return rc;
+    if (!e->h_state[seq].active) return LLMA_ERR_STATE;
+    return e->h_state[seq].kv_len;
+}

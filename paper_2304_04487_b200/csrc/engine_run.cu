@@ -1,0 +1,291 @@
+// Decoding entry points of the C ABI: prefill, reference upload, step, generate.
+#include <algorithm>
+#include <climits>
+#include <cstring>
+#include <vector>
+
+#include "engine.h"
+
+using namespace llma;
+
+// ---- one decoder forward over the rows described by e->rows ---------------------------------
+// Every kernel reads the row descriptors from device memory, so the same launch sequence
+// serves any mix of rows (greedy, copy steps, prompt chunks) and can be replayed as a graph.
+static void enqueue_forward(llma_engine* e, bool lm_head) {
+    const ModelDims& d = e->dims;
+    cudaStream_t st = e->stream;
+    const bool b = e->bf16;
+    const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
+    for (int l = 0; l < d.n_layers; ++l) {
+        launch_rmsnorm(st, b, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_gemm_simt(st, b, e->rows, e->wq[l], e->x_hat, e->qkv, HD, D, 3 * HD, false);
+        launch_gemm_simt(st, b, e->rows, e->wk[l], e->x_hat, e->qkv + HD, HD, D, 3 * HD, false);
+        launch_gemm_simt(st, b, e->rows, e->wv[l], e->x_hat, e->qkv + 2 * HD, HD, D, 3 * HD, false);
+        launch_qkv_post(st, b, d, l, e->rows, e->qkv, e->rope_cos, e->rope_sin, e->kcache, e->vcache);
+        launch_attention_simt(st, b, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        launch_gemm_simt(st, b, e->rows, e->wo[l], e->attn, e->x, D, HD, D, true);
+        launch_rmsnorm(st, b, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_gemm_simt(st, b, e->rows, e->w_gate[l], e->x_hat, e->gate_up, F, D, 2 * F, false);
+        launch_gemm_simt(st, b, e->rows, e->w_up[l], e->x_hat, e->gate_up + F, F, D, 2 * F, false);
+        launch_silu_mul(st, b, e->rows, e->gate_up, e->h, F);
+        launch_gemm_simt(st, b, e->rows, e->w_down[l], e->h, e->x, D, F, D, true);
+        e->launch_counter += 12;
+    }
+    if (lm_head) {
+        launch_rmsnorm(st, b, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        launch_gemm_simt(st, b, e->rows, e->lm_head, e->x_hat, e->logits, d.vocab, D, d.vocab, false);
+        launch_argmax(st, e->rows, e->logits, d.vocab, e->out_tok);
+        e->launch_counter += 3;
+    }
+}
+
+// plan (trigger search + copy) -> embedding gather -> forward -> accept + K/V commit
+static void enqueue_step(llma_engine* e, int n, int k) {
+    const ModelDims& d = e->dims;
+    launch_plan(e->stream, d, e->seq_state, e->rows, e->ref, e->doc_start, e->doc_end, e->y, e->y_cap, n, k,
+                e->dev_err);
+    launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+    e->launch_counter += 3;
+    enqueue_forward(e, true);
+    launch_accept(e->stream, d, e->seq_state, e->ref, e->out_tok, e->y, e->y_cap);
+    e->launch_counter += 1;
+}
+
+static int check_device_error(llma_engine* e) {
+    CU_TRY(cudaMemcpyAsync(e->h_err, e->dev_err, sizeof(int32_t), cudaMemcpyDeviceToHost, e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    const int32_t code = *e->h_err;
+    if (code == kDevErrNone) return LLMA_OK;
+    CU_TRY(cudaMemsetAsync(e->dev_err, 0, sizeof(int32_t), e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    if (code == kDevErrTimeout) return LLMA_ERR_DEVICE_TIMEOUT;
+    if (code == kDevErrCapacity) return LLMA_ERR_CAPACITY;
+    return LLMA_ERR_TOKEN_RANGE;
+}
+
+static int read_state(llma_engine* e) {
+    CU_TRY(cudaMemcpyAsync(e->h_state, e->seq_state, e->dims.max_batch * sizeof(SeqState), cudaMemcpyDeviceToHost,
+                           e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    return LLMA_OK;
+}
+
+static int write_state(llma_engine* e, int seq) {
+    CU_TRY(cudaMemcpyAsync(e->seq_state + seq, e->h_state + seq, sizeof(SeqState), cudaMemcpyHostToDevice, e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    return LLMA_OK;
+}
+
+extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, int32_t n_prompt) {
+    if (!e || !prompt) return LLMA_ERR_NULL;
+    const ModelDims& d = e->dims;
+    if (seq < 0 || seq >= d.max_batch) return LLMA_ERR_CAPACITY;
+    if (n_prompt < 1) return LLMA_ERR_ARG;
+    if (n_prompt > d.max_seq) return LLMA_ERR_CAPACITY;
+    for (int i = 0; i < n_prompt; ++i)
+        if (prompt[i] < 0 || prompt[i] >= d.vocab) return LLMA_ERR_TOKEN_RANGE;
+    int rc = read_state(e);
+    if (rc) return rc;
+    // push prompt[0 .. P-2] through the decoder, kMaxRows consecutive positions per pass
+    const int n_cache = n_prompt - 1;
+    for (int p0 = 0; p0 < n_cache; p0 += kMaxRows) {
+        const int cnt = std::min(kMaxRows, n_cache - p0);
+        RowDesc* R = e->h_rows;
+        for (int r = 0; r < kMaxRows; ++r) {
+            R->tok[r] = r < cnt ? prompt[p0 + r] : 0;
+            R->pos[r] = r < cnt ? p0 + r : -1;
+            R->seq[r] = seq;
+        }
+        R->rows_used = cnt;
+        R->max_pos = p0 + cnt - 1;
+        CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));
+        launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+        enqueue_forward(e, false);
+        CU_TRY(cudaGetLastError());
+        CU_TRY(cudaStreamSynchronize(e->stream));  // h_rows is reused by the next chunk
+    }
+    SeqState& S = e->h_state[seq];
+    const int32_t keep_ref = S.ref_len;
+    std::memset(&S, 0, sizeof(S));
+    S.active = 1; S.kv_len = n_cache; S.pending = prompt[n_prompt - 1]; S.ref_len = keep_ref;
+    S.prompt_len = n_prompt; S.pos = -1; S.last_pos = -1; S.target_len = 0; S.done = 1;
+    rc = write_state(e, seq);
+    if (rc) return rc;
+    e->prompt_last[seq] = prompt[n_prompt - 1];
+    e->last_step_valid = false;
+    return check_device_error(e);
+}
+
+extern "C" int llma_set_reference(llma_engine* e, int32_t seq, const int32_t* tokens, int32_t n_tokens,
+                                  const int32_t* doc_offsets, int32_t n_docs) {
+    if (!e) return LLMA_ERR_NULL;
+    const ModelDims& d = e->dims;
+    if (seq < 0 || seq >= d.max_batch) return LLMA_ERR_CAPACITY;
+    if (n_tokens < 0) return LLMA_ERR_ARG;
+    if (n_tokens > 0 && !tokens) return LLMA_ERR_NULL;
+    if (n_tokens > e->cfg.max_ref) return LLMA_ERR_REF_TOO_LONG;
+    std::vector<int32_t> ds((size_t)std::max(n_tokens, 1)), de((size_t)std::max(n_tokens, 1));
+    if (doc_offsets) {
+        if (n_docs < 1 || doc_offsets[0] != 0 || doc_offsets[n_docs] != n_tokens) return LLMA_ERR_REF_TOO_LONG;
+        for (int j = 0; j < n_docs; ++j) {
+            if (doc_offsets[j + 1] < doc_offsets[j]) return LLMA_ERR_REF_TOO_LONG;
+            for (int i = doc_offsets[j]; i < doc_offsets[j + 1]; ++i) { ds[i] = doc_offsets[j]; de[i] = doc_offsets[j + 1]; }
+        }
+    } else {
+        for (int i = 0; i < n_tokens; ++i) { ds[i] = 0; de[i] = n_tokens; }
+    }
+    for (int i = 0; i < n_tokens; ++i)
+        if (tokens[i] < 0 || tokens[i] >= d.vocab) return LLMA_ERR_TOKEN_RANGE;
+    if (n_tokens > 0) {
+        const size_t off = (size_t)seq * d.max_ref, nb = (size_t)n_tokens * sizeof(int32_t);
+        CU_TRY(cudaMemcpyAsync(e->ref + off, tokens, nb, cudaMemcpyHostToDevice, e->stream));
+        CU_TRY(cudaMemcpyAsync(e->doc_start + off, ds.data(), nb, cudaMemcpyHostToDevice, e->stream));
+        CU_TRY(cudaMemcpyAsync(e->doc_end + off, de.data(), nb, cudaMemcpyHostToDevice, e->stream));
+    }
+    CU_TRY(cudaMemcpyAsync(&e->seq_state[seq].ref_len, &n_tokens, sizeof(int32_t), cudaMemcpyHostToDevice, e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));  // the host vectors die at return
+    return LLMA_OK;
+}
+
+static int check_nk(const llma_engine* e, int n, int k) {
+    if (n < 1 || k < 0 || k > e->cfg.max_k) return LLMA_ERR_ARG;
+    return LLMA_OK;
+}
+
+extern "C" int llma_step(llma_engine* e, int32_t n, int32_t k, int32_t* out_tokens, int32_t* n_out) {
+    if (!e || !out_tokens || !n_out) return LLMA_ERR_NULL;
+    int rc = check_nk(e, n, k);
+    if (rc) return rc;
+    const ModelDims& d = e->dims;
+    rc = read_state(e);
+    if (rc) return rc;
+    bool any = false;
+    std::vector<int32_t> y0((size_t)d.max_batch, 0);
+    for (int s = 0; s < d.max_batch; ++s) {
+        SeqState& S = e->h_state[s];
+        y0[s] = S.y_len;
+        if (!S.active) continue;
+        if (S.kv_len + 1 > d.max_seq || S.y_len + 1 > e->y_cap) return LLMA_ERR_CAPACITY;
+        any = true;
+    }
+    if (!any) return LLMA_ERR_STATE;
+    for (int s = 0; s < d.max_batch; ++s) {
+        SeqState& S = e->h_state[s];
+        if (!S.active) continue;
+        // a lone step has no output budget of its own: only the capacities bound the copy
+        S.target_len = std::min(e->y_cap, S.y_len + (d.max_seq - S.kv_len));
+        S.done = 0;
+        rc = write_state(e, s);
+        if (rc) return rc;
+    }
+    enqueue_step(e, n, k);
+    CU_TRY(cudaGetLastError());
+    rc = check_device_error(e);
+    if (rc) return rc;
+    rc = read_state(e);
+    if (rc) return rc;
+    for (int s = 0; s < d.max_batch; ++s) {
+        const SeqState& S = e->h_state[s];
+        const int m = S.active ? S.y_len - y0[s] : 0;
+        n_out[s] = m;
+        if (m > 0)
+            CU_TRY(cudaMemcpy(out_tokens + (size_t)s * d.kp1, e->y + (size_t)s * e->y_cap + y0[s],
+                              (size_t)m * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    }
+    e->last_step_valid = true;
+    return LLMA_OK;
+}
+
+static int get_step_graph(llma_engine* e, int n, int k, cudaGraphExec_t* out) {
+    auto it = e->step_graphs.find({n, k});
+    if (it != e->step_graphs.end()) { *out = it->second; return LLMA_OK; }
+    cudaGraph_t g = nullptr;
+    const int64_t before = e->launch_counter;
+    CU_TRY(cudaStreamBeginCapture(e->stream, cudaStreamCaptureModeThreadLocal));
+    enqueue_step(e, n, k);
+    cudaError_t ce = cudaStreamEndCapture(e->stream, &g);
+    e->launches_per_step = e->launch_counter - before;
+    e->launch_counter = before;
+    CU_TRY(ce);
+    cudaGraphExec_t ge = nullptr;
+    ce = cudaGraphInstantiate(&ge, g, 0);
+    cudaGraphDestroy(g);
+    CU_TRY(ce);
+    e->step_graphs[{n, k}] = ge;
+    *out = ge;
+    return LLMA_OK;
+}
+
+extern "C" int llma_generate(llma_engine* e, int32_t max_new, int32_t n, int32_t k, int32_t* out_tokens,
+                             int32_t* n_out, llma_stats* stats) {
+    if (!e || !out_tokens || !n_out) return LLMA_ERR_NULL;
+    int rc = check_nk(e, n, k);
+    if (rc) return rc;
+    if (max_new < 0) return LLMA_ERR_ARG;
+    const ModelDims& d = e->dims;
+    rc = read_state(e);
+    if (rc) return rc;
+    bool any = false;
+    std::vector<SeqState> s0(e->h_state, e->h_state + d.max_batch);
+    for (int s = 0; s < d.max_batch; ++s) {
+        const SeqState& S = s0[s];
+        if (!S.active) continue;
+        if (S.kv_len + max_new > d.max_seq || S.y_len + max_new > e->y_cap) return LLMA_ERR_CAPACITY;
+        any = true;
+    }
+    if (!any) return LLMA_ERR_STATE;
+    for (int s = 0; s < d.max_batch; ++s) {
+        SeqState& S = e->h_state[s];
+        if (!S.active) continue;
+        S.target_len = S.y_len + max_new;
+        S.done = max_new == 0;
+        rc = write_state(e, s);
+        if (rc) return rc;
+    }
+    cudaGraphExec_t graph = nullptr;
+    rc = get_step_graph(e, n, k, &graph);
+    if (rc) return rc;
+
+    // Each step emits between 1 and k+1 tokens per sequence, so ceil(left / (k+1)) more steps
+    // can never be too many.  Launch that many back to back, look at the counters once, repeat.
+    int64_t launches = 0;
+    CU_TRY(cudaEventRecord(e->ev0, e->stream));
+    for (;;) {
+        int left = 0;
+        for (int s = 0; s < d.max_batch; ++s) {
+            const SeqState& S = e->h_state[s];
+            if (S.active && !S.done) left = std::max(left, S.target_len - S.y_len);
+        }
+        if (left <= 0) break;
+        const int batch = (left + k) / (k + 1);
+        for (int i = 0; i < batch; ++i) CU_TRY(cudaGraphLaunch(graph, e->stream));
+        launches += (int64_t)batch * e->launches_per_step;
+        rc = read_state(e);
+        if (rc) return rc;
+    }
+    CU_TRY(cudaEventRecord(e->ev1, e->stream));
+    rc = check_device_error(e);
+    if (rc) return rc;
+
+    llma_stats st;
+    std::memset(&st, 0, sizeof(st));
+    for (int s = 0; s < d.max_batch; ++s) {
+        const SeqState& S = e->h_state[s];
+        const int m = S.active ? S.y_len - s0[s].y_len : 0;
+        n_out[s] = m;
+        if (m > 0)
+            CU_TRY(cudaMemcpy(out_tokens + (size_t)s * max_new, e->y + (size_t)s * e->y_cap + s0[s].y_len,
+                              (size_t)m * sizeof(int32_t), cudaMemcpyDeviceToHost));
+        if (S.active) {
+            st.steps += S.steps - s0[s].steps;
+            st.trigger_steps += S.trigger_steps - s0[s].trigger_steps;
+            st.copied_accepted += S.copied_accepted - s0[s].copied_accepted;
+            st.tokens += m;
+        }
+    }
+    st.launches = launches;
+    CU_TRY(cudaEventElapsedTime(&st.device_ms, e->ev0, e->ev1));
+    if (stats) *stats = st;
+    e->last_step_valid = launches > 0;
+    return LLMA_OK;
+}

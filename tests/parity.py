@@ -1,0 +1,101 @@
+"""Step-by-step parity harness: CUDA engine vs CPU oracle on the same seeded inputs.
+
+Integer results (match position, copy length, accepted count, tokens) must be equal;
+logits must agree within the stated tolerance on every row of every step.  Where the
+two argmaxes differ, the oracle's top-1/top-2 margin at that row must be below
+``tie_margin`` (the decision is then legitimately ambiguous across precisions): the event
+is counted and both sides continue from the GPU's tokens, which the oracle's
+position-indexed cache allows without any special handling.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from oracle import decoding as D
+
+
+@dataclass
+class ParityReport:
+    steps: int = 0
+    tokens: List[int] = field(default_factory=list)
+    near_ties: int = 0
+    max_logit_err: float = 0.0
+    max_logit_scale: float = 0.0
+    trigger_steps: int = 0
+    copied_accepted: int = 0
+    rows_compared: int = 0
+
+
+def logits_close(got: np.ndarray, want: np.ndarray, mode: str) -> float:
+    """Returns the error measure and asserts the tolerance.
+    fp32: |d| <= 1e-4 * max(1, max|want|) per row.  bf16: |d| <= 2e-2 absolute."""
+    err = float(np.abs(got - want).max())
+    if mode == "fp32":
+        tol = 1e-4 * max(1.0, float(np.abs(want).max()))
+    else:
+        tol = 2e-2
+    assert err <= tol, f"logit error {err:.3e} above tolerance {tol:.3e} ({mode})"
+    return err
+
+
+def step_parity(eng, oracle_model, prompt: Sequence[int], ref: Sequence[int], offs: Optional[Sequence[int]],
+                n: int, k: int, n_new: int, mode: str, seq: int = 0, tie_margin: float = 1e-3) -> ParityReport:
+    """Drive ``eng.llma_step`` and the oracle side by side for ``n_new`` tokens."""
+    rep = ParityReport()
+    ref = [int(t) for t in ref]
+    kp1 = eng.max_k + 1
+    eng.llma_prefill(seq, prompt)
+    eng.llma_set_reference(seq, ref, offs)
+    L, pending = D.prefill(oracle_model, prompt)
+    assert eng.llma_kv_len(seq) == L
+    y: List[int] = []
+    while len(y) < n_new:
+        matched, pos, _ = D.match_ngrams(y, ref, offs, n)
+        k_eff = D.copy_length(pos, len(ref), offs, k, eng.max_seq - L) if matched else 0
+        inputs = [pending] + (ref[pos:pos + k_eff] if k_eff > 0 else [])
+        want_rows = np.stack([oracle_model.forward(tok, L + j) for j, tok in enumerate(inputs)])
+        outs = want_rows.argmax(1).tolist()
+        a = 0
+        while a < k_eff and outs[a] == ref[pos + a]:
+            a += 1
+        want_tokens = outs[:a + 1]
+
+        got_tokens = eng.llma_step(n, k)[seq]
+        info = eng.llma_last_step_info()[seq]
+        assert info.k_eff == k_eff, (rep.steps, info.k_eff, k_eff)
+        assert info.pos == (pos if k_eff > 0 else -1), (rep.steps, info.pos, pos)
+        got_rows = eng.llma_debug_logits()[seq * kp1: seq * kp1 + k_eff + 1]
+        for j in range(k_eff + 1):
+            rep.max_logit_err = max(rep.max_logit_err, logits_close(got_rows[j], want_rows[j], mode))
+            rep.max_logit_scale = max(rep.max_logit_scale, float(np.abs(want_rows[j]).max()))
+        rep.rows_compared += k_eff + 1
+        # the engine's acceptance must be Algorithm 1 applied to its own argmaxes
+        gouts = got_rows.argmax(1).tolist()
+        ga = 0
+        while ga < k_eff and gouts[ga] == ref[pos + ga]:
+            ga += 1
+        assert got_tokens == gouts[:ga + 1], (rep.steps, got_tokens, gouts, ga)
+        assert info.accepted == ga and info.emitted == ga + 1
+        if got_tokens != want_tokens:
+            j = next(i for i in range(min(len(got_tokens), len(want_tokens))) if got_tokens[i] != want_tokens[i])
+            srt = np.sort(want_rows[j])
+            margin = float(srt[-1] - srt[-2])
+            assert margin < tie_margin, f"tokens differ at step {rep.steps} row {j} with oracle margin {margin:.3e}"
+            rep.near_ties += 1
+        y.extend(got_tokens)
+        L += len(got_tokens)
+        pending = got_tokens[-1]
+        assert eng.llma_kv_len(seq) == L
+        rep.steps += 1
+        rep.trigger_steps += int(k_eff > 0)
+        rep.copied_accepted += len(got_tokens) - 1
+    rep.tokens = y
+    return rep
+
+
+def make_overlap_reference(y_star: Sequence[int], doc_lengths: Sequence[int], overlap: float, vocab: int, seed: int = 0):
+    from workloads import build_reference
+    return build_reference(y_star, doc_lengths, overlap, vocab, seed=seed)

@@ -1,0 +1,189 @@
+"""GPU parity tests: the CUDA engine (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from oracle import decoding as D
+from oracle import model as OM
+from workloads import SHAPES, ModelShape, build_reference, make_prompt, make_weights
+
+from parity import step_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _engine(shape, w, **kw):
+    from paper_2304_04487_b200 import Engine
+    return Engine(shape, w, **kw)
+
+
+_cache = {}
+
+
+def _weights(shape, seed=0, std=0.02):
+    key = (shape.name, seed, std)
+    if key not in _cache:
+        _cache[key] = make_weights(shape, seed=seed, std=std)
+    return _cache[key]
+
+
+def _greedy_star(shape, w, prompt, n_new, max_seq):
+    key = ("y*", shape.name, id(w), len(prompt), n_new)
+    if key not in _cache:
+        _cache[key] = D.greedy_decode(OM.OracleModel(shape, w, max_seq=max_seq), prompt, n_new).tokens
+    return _cache[key]
+
+
+# ---- configuration 1 of the benchmark set: tiny fp32 decoder, n=2, k=4, 64 new tokens ---------------
+def test_tiny_fp32_stepwise_parity():
+    shape = SHAPES["tiny-fp32"]
+    w = _weights(shape)
+    prompt = make_prompt(128, shape.vocab, seed=1)
+    N, max_seq = 64, 256
+    y_star = _greedy_star(shape, w, prompt, N, max_seq)
+    ref, offs, info = build_reference(y_star, [256], 0.6, shape.vocab, seed=0)
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=256, max_k=4, keep_logits=True)
+    rep = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, offs, 2, 4, N, "fp32")
+    assert rep.near_ties == 0
+    assert rep.tokens[:N] == y_star                      # lossless: equals the oracle's greedy output
+    assert rep.trigger_steps > 5 and rep.copied_accepted > 10, (rep, info)
+    assert rep.max_logit_err <= 1e-4 * max(1.0, rep.max_logit_scale)
+
+
+@pytest.mark.parametrize("name,n,k,P,N", [("tiny-bf16", 1, 8, 70, 48), ("small-bf16", 1, 5, 45, 40),
+                                           ("small-bf16", 2, 16, 33, 40)])
+def test_bf16_stepwise_parity(name, n, k, P, N):
+    shape = SHAPES[name]
+    w = _weights(shape)
+    prompt = make_prompt(P, shape.vocab, seed=2)
+    max_seq = P + N + 40
+    y_star = _greedy_star(shape, w, prompt, N, max_seq)
+    ref, offs, _ = build_reference(y_star, [60, 60, 40], 0.7, shape.vocab, seed=1)
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=200, max_k=k, keep_logits=True)
+    rep = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, offs, n, k, N, "bf16")
+    assert rep.max_logit_err <= 2e-2
+    assert rep.near_ties <= 3, rep.near_ties
+    assert rep.trigger_steps > 0
+
+
+# ---- the whole loop: llma_generate vs Algorithm 1 on the oracle, LLMA == greedy on the GPU -----------
+@pytest.mark.parametrize("name", ["tiny-fp32", "tiny-bf16"])
+def test_generate_lossless_and_trace(name):
+    shape = SHAPES[name]
+    w = _weights(shape)
+    prompt = make_prompt(40, shape.vocab, seed=3)
+    N, max_seq = 64, 128
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=300, max_k=18)
+    eng.llma_prefill(0, prompt)
+    (g_tokens,), g_stats = eng.llma_generate(N, 1, 0)
+    assert len(g_tokens) == N and g_stats.steps == N and g_stats.trigger_steps == 0 and g_stats.tokens == N
+    if name == "tiny-fp32":
+        assert g_tokens == _greedy_star(shape, w, prompt, N, max_seq)
+    # references built from the engine's own greedy output: integer behaviour is then fully
+    # determined by (y, D, n, k) and must equal Algorithm 2's model-free prediction
+    refs = {
+        "spliced": build_reference(g_tokens, [100, 100, 60], 0.8, shape.vocab, seed=4)[:2],
+        "self": (np.asarray(g_tokens, np.int32), None),
+        "repeats": (np.asarray(g_tokens[5:15] * 3 + g_tokens[30:50] + g_tokens[5:12], np.int32),
+                    np.asarray([0, 30, 30, 50, 57], np.int32)),
+        "empty": (np.zeros(0, np.int32), None),
+    }
+    for rname, (ref, offs) in refs.items():
+        eng.llma_set_reference(0, ref, offs)
+        for n, k in ((1, 4), (1, 8), (2, 3), (3, 18), (1, 1)):
+            eng.llma_rewind(0)
+            (toks,), st = eng.llma_generate(N, n, k)
+            assert toks == g_tokens, (rname, n, k)                       # identical to greedy on the same engine
+            sim = D.simulate_decoding_sequence(g_tokens, ref.tolist(), None if offs is None else offs.tolist(), n, k)
+            assert st.steps == len(sim), (rname, n, k, st.steps, len(sim))
+            assert st.tokens == N == st.steps + st.copied_accepted
+            assert st.trigger_steps == sum(1 for i, _ in sim if i > 1)
+            assert st.launches > 0 and st.device_ms > 0
+    # stepping by hand gives the same per-step (inputs, outputs) sequence as Algorithm 2
+    ref, offs = refs["spliced"]
+    eng.llma_set_reference(0, ref, offs)
+    eng.llma_rewind(0)
+    sim = D.simulate_decoding_sequence(g_tokens, ref.tolist(), offs.tolist(), 1, 6)
+    # (llma_step has no output budget of its own; far from the end of y that makes no difference)
+    got, out = [], []
+    while len(out) < 20:
+        t = eng.llma_step(1, 6)[0]
+        i = eng.llma_last_step_info()[0]
+        got.append((1 + i.k_eff, i.emitted)); out += t
+    assert out == g_tokens[:len(out)]
+    assert got == sim[:len(got)]
+
+
+def test_logits_bitwise_independent_of_k():
+    """Rows of a (k+1)-row verification step must be bit-identical to the rows that one-token
+    greedy steps compute at the same positions."""
+    for name in ("tiny-fp32", "small-bf16"):
+        shape = SHAPES[name]
+        w = _weights(shape)
+        prompt = make_prompt(37, shape.vocab, seed=5)
+        N, max_seq = 24, 96
+        eng = _engine(shape, w, max_seq=max_seq, max_ref=64, max_k=16, keep_logits=True)
+        eng.llma_prefill(0, prompt)
+        rows_greedy, toks = [], []
+        for _ in range(N):
+            toks += eng.llma_step(1, 0)[0]
+            rows_greedy.append(eng.llma_debug_logits()[0].copy())
+        eng.llma_set_reference(0, toks, None)
+        for k in (1, 4, 7, 16):
+            eng.llma_rewind(0)
+            i = 0
+            while i < N - 17:
+                t = eng.llma_step(1, k)[0]
+                lg = eng.llma_debug_logits()
+                for j in range(len(t)):
+                    assert np.array_equal(lg[j].view(np.uint32), rows_greedy[i + j].view(np.uint32)), (name, k, i, j)
+                assert t == toks[i:i + len(t)]
+                i += len(t)
+        # run twice: same bits (no race in any reduction)
+        eng.llma_rewind(0)
+        eng.llma_step(1, 0); a = eng.llma_debug_logits()[0].copy()
+        eng.llma_rewind(0)
+        eng.llma_step(1, 0); b = eng.llma_debug_logits()[0].copy()
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_kv_rows_match_oracle():
+    shape = SHAPES["small-bf16"]
+    w = _weights(shape)
+    prompt = make_prompt(40, shape.vocab, seed=6)
+    eng = _engine(shape, w, max_seq=64, max_ref=8, max_k=0)
+    om = OM.OracleModel(shape, w, max_seq=64)
+    eng.llma_prefill(0, prompt)
+    D.prefill(om, prompt)
+    bad = 0
+    for layer in (0, shape.n_layers - 1):
+        for pos in (0, 17, 31, 32, 38):
+            for which in (0, 1):
+                got = eng.llma_debug_kv_row(layer, 0, pos, which)
+                want = om.read_cache(layer, pos, which)
+                # bf16 rows: equal up to one rounding step of the stored type
+                assert np.abs(got - want).max() <= 2.0 ** -7 * max(1e-3, np.abs(want).max())
+                bad += int((got != want).sum())
+    assert bad < 0.2 * 2 * 5 * 2 * shape.n_heads * shape.head_dim
+
+
+def test_two_sequences_ragged():
+    shape = SHAPES["tiny-bf16"]
+    w = _weights(shape)
+    N, max_seq = 40, 128
+    prompts = [make_prompt(30, shape.vocab, seed=7), make_prompt(51, shape.vocab, seed=8)]
+    singles = []
+    for p in prompts:
+        e1 = _engine(shape, w, max_seq=max_seq, max_ref=128, max_k=7)
+        e1.llma_prefill(0, p)
+        (t,), _ = e1.llma_generate(N, 1, 0)
+        singles.append(t)
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=128, max_k=7, max_batch=2)
+    for s, p in enumerate(prompts):
+        eng.llma_prefill(s, p)
+    eng.llma_set_reference(0, singles[0][4:30], None)
+    eng.llma_set_reference(1, build_reference(singles[1], [64, 64], 0.6, shape.vocab, seed=9)[0], [0, 64, 128])
+    toks, st = eng.llma_generate(N, 1, 7)
+    assert toks[0] == singles[0] and toks[1] == singles[1]        # each sequence unaffected by its neighbour
+    assert st.tokens == 2 * N and st.copied_accepted > 0
+    infos = eng.llma_last_step_info()
+    assert len(infos) == 2
