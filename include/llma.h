@@ -186,6 +186,10 @@ int llma_debug_kv_row(llma_engine *e, int32_t layer, int32_t seq, int32_t pos, i
 /* Committed K/V length of a sequence (prompt rows + emitted tokens - 1), or a negative status. */
 int llma_kv_len(llma_engine *e, int32_t seq);
 
+/* Which GEMM implementation the engine resolved to (LLMA_GEMM_SIMT or LLMA_GEMM_TCGEN05), or a
+ * negative status. */
+int llma_gemm_impl(llma_engine *e);
+
 /* The CUDA error code behind the most recent LLMA_ERR_CUDA on this thread (0 if none). */
 int llma_last_cuda_error(void);
 

@@ -47,7 +47,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_gemm_impl", "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
         L.llma_debug_logits.argtypes = [vp, C.POINTER(C.c_float)]
         L.llma_debug_kv_row.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_float)]
         L.llma_kv_len.argtypes = [vp, i32]
+        L.llma_gemm_impl.argtypes = [vp]
         L.llma_last_cuda_error.argtypes = []
         L.llma_strerror.argtypes = [C.c_int]
         L.llma_strerror.restype = C.c_char_p
@@ -198,6 +199,9 @@ class Engine:
 
     def llma_kv_len(self, seq: int) -> int:
         return self._check(lib().llma_kv_len(self._h, seq), "llma_kv_len")
+
+    def llma_gemm_impl(self) -> int:
+        return self._check(lib().llma_gemm_impl(self._h), "llma_gemm_impl")
 
     def llma_destroy(self) -> None:
         if getattr(self, "_h", None):

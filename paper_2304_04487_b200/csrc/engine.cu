@@ -2,6 +2,7 @@
 // step (Algorithm 1's loop body) and the whole decoding loop.  See include/llma.h.
 #include "engine.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -49,6 +50,7 @@ static void free_engine(llma_engine* e) {
     cudaFree(e->y); cudaFree(e->out_tok); cudaFree(e->dev_err); cudaFree(e->x); cudaFree(e->qkv);
     cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
     cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
+    cudaFree(e->gemm_ws); cudaFree(e->gemm_cnt); cudaFree(e->part_max); cudaFree(e->part_idx);
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
     if (e->h_err) cudaFreeHost(e->h_err);
@@ -69,7 +71,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     if (cfg->max_batch < 1 || cfg->max_k < 0 || cfg->max_batch * (cfg->max_k + 1) > kMaxRows) return LLMA_ERR_CONFIG;
     if (cfg->max_seq < 2 || cfg->max_ref < 0 || !(cfg->rms_eps >= 0.f) || !(cfg->rope_theta > 0.f)) return LLMA_ERR_CONFIG;
     if (cfg->gemm_impl < LLMA_GEMM_AUTO || cfg->gemm_impl > LLMA_GEMM_TCGEN05) return LLMA_ERR_CONFIG;
-    if (cfg->gemm_impl == LLMA_GEMM_TCGEN05 && cfg->dtype != LLMA_DTYPE_BF16) return LLMA_ERR_CONFIG;
     if (!w->tok_emb || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
         !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
         return LLMA_ERR_NULL;
@@ -86,7 +87,9 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     e->device = dev;
     e->stream = (cudaStream_t)cuda_stream;
     e->bf16 = cfg->dtype == LLMA_DTYPE_BF16;
-    e->gemm_impl = cfg->gemm_impl == LLMA_GEMM_AUTO ? LLMA_GEMM_SIMT : cfg->gemm_impl;
+    const bool tc_ok = cfg->dtype == LLMA_DTYPE_BF16 && HD % 128 == 0 && cfg->d_model % 128 == 0;
+    if (cfg->gemm_impl == LLMA_GEMM_TCGEN05 && !tc_ok) return LLMA_ERR_CONFIG;
+    e->gemm_impl = cfg->gemm_impl == LLMA_GEMM_AUTO ? (tc_ok ? LLMA_GEMM_TCGEN05 : LLMA_GEMM_SIMT) : cfg->gemm_impl;
     ModelDims& d = e->dims;
     d.n_layers = L; d.d_model = cfg->d_model; d.n_heads = cfg->n_heads; d.head_dim = cfg->head_dim;
     d.d_ffn = cfg->d_ffn; d.vocab = cfg->vocab; d.hd_total = HD; d.max_batch = cfg->max_batch;
@@ -147,6 +150,36 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         CREATE_TRY(dalloc(&e->rope_sin, s.size(), false));
         CREATE_TRY(cudaMemcpy(e->rope_cos, c.data(), c.size() * 4, cudaMemcpyHostToDevice));
         CREATE_TRY(cudaMemcpy(e->rope_sin, s.data(), s.size() * 4, cudaMemcpyHostToDevice));
+    }
+    if (e->gemm_impl == LLMA_GEMM_TCGEN05) {
+        cudaDeviceProp prop;
+        CREATE_TRY(cudaGetDeviceProperties(&prop, dev));
+        if (prop.major != 10) { free_engine(e); return LLMA_ERR_CONFIG; }  // tcgen05 needs sm_100
+        e->num_sms = prop.multiProcessorCount;
+        const int vt = (d.vocab + 127) / 128;
+        const int max_tiles = std::max(std::max(vt, 3 * HD / 128), std::max((d.d_ffn + 63) / 64, (d.d_model + 127) / 128));
+        CREATE_TRY(dalloc(&e->gemm_ws, (size_t)e->num_sms * 2 * 128 * 32));
+        CREATE_TRY(dalloc(&e->gemm_cnt, (size_t)max_tiles));
+        CREATE_TRY(dalloc(&e->part_max, (size_t)vt * 32));
+        CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * 32));
+        e->maps.resize(L);
+        int bad = 0;
+        for (int l = 0; l < L; ++l) {
+            llma_engine::LayerMaps& m = e->maps[l];
+            bad |= make_tensor_map_bf16(&m.wq, e->wq[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wk, e->wk[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wv, e->wv[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wo, e->wo[l], d.d_model, HD, 128);
+            bad |= make_tensor_map_bf16(&m.w_gate, e->w_gate[l], d.d_ffn, d.d_model, 64);
+            bad |= make_tensor_map_bf16(&m.w_up, e->w_up[l], d.d_ffn, d.d_model, 64);
+            bad |= make_tensor_map_bf16(&m.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
+        }
+        bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
+        bad |= make_tensor_map_bf16(&e->map_x_hat, e->x_hat, kMaxRows, d.d_model, kMaxRows);
+        bad |= make_tensor_map_bf16(&e->map_attn, e->attn, kMaxRows, HD, kMaxRows);
+        bad |= make_tensor_map_bf16(&e->map_h, e->h, kMaxRows, d.d_ffn, kMaxRows);
+        if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
+        CREATE_TRY(init_gemm_tcgen05());
     }
     CREATE_TRY(cudaMallocHost((void**)&e->h_state, B * sizeof(SeqState)));
     CREATE_TRY(cudaMallocHost((void**)&e->h_rows, sizeof(RowDesc)));

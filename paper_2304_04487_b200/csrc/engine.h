@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "../../include/llma.h"
+#include "gemm_tcgen05.cuh"
 #include "kernels.h"
 
 struct llma_engine {
@@ -31,6 +32,16 @@ struct llma_engine {
     void *x_hat = nullptr, *attn = nullptr, *h = nullptr;
     float *rope_cos = nullptr, *rope_sin = nullptr;
     void *kcache = nullptr, *vcache = nullptr;
+
+    // tensor-core GEMM path (bf16): TMA descriptors of weights and activation buffers, work buffers
+    struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };
+    std::vector<LayerMaps> maps;
+    CUtensorMap map_lm_head, map_x_hat, map_attn, map_h;
+    int num_sms = 0;
+    float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
+    int32_t* gemm_cnt = nullptr;    // per-tile arrival counters
+    float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
+    int32_t* part_idx = nullptr;
 
     // pinned host staging
     llma::SeqState* h_state = nullptr;

@@ -102,3 +102,8 @@ extern "C" int llma_kv_len(llma_engine* e, int32_t seq) {
     if (!e->h_state[seq].active) return LLMA_ERR_STATE;
     return e->h_state[seq].kv_len;
 }
+
+extern "C" int llma_gemm_impl(llma_engine* e) {
+    if (!e) return LLMA_ERR_NULL;
+    return e->gemm_impl;
+}

@@ -11,7 +11,61 @@ using namespace llma;
 // ---- one decoder forward over the rows described by e->rows ---------------------------------
 // Every kernel reads the row descriptors from device memory, so the same launch sequence
 // serves any mix of rows (greedy, copy steps, prompt chunks) and can be replayed as a graph.
+static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int k_in, int tiles_per_map) {
+    GemmArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.mode = mode; a.n_out = n_out; a.n_tiles = n_tiles; a.chunks = k_in / 64; a.tiles_per_map = tiles_per_map;
+    a.rows = e->rows; a.ws = e->gemm_ws; a.cnt = e->gemm_cnt; a.dev_err = e->dev_err;
+    a.dims = e->dims;
+    return a;
+}
+
+static void run_gemm(llma_engine* e, const GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1,
+                     const CUtensorMap& a2, const CUtensorMap& b) {
+    const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
+    launch_gemm_tcgen05(e->stream, grid, a, a0, a1, a2, b);
+}
+
+// Tensor-core path (bf16): 7 kernels per layer, every projection fused with what follows it.
+static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
+    const ModelDims& d = e->dims;
+    cudaStream_t st = e->stream;
+    const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
+    for (int l = 0; l < d.n_layers; ++l) {
+        const llma_engine::LayerMaps& m = e->maps[l];
+        launch_rmsnorm(st, true, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
+        q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
+        q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
+        run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
+        launch_attention_simt(st, true, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
+        o.out_f32 = e->x; o.ld = D;
+        run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
+        launch_rmsnorm(st, true, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
+        gu.out_bf16 = (__nv_bfloat16*)e->h;
+        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
+        GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
+        dn.out_f32 = e->x; dn.ld = D;
+        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->map_h);
+        e->launch_counter += 7;
+    }
+    if (lm_head) {
+        const int vt = (d.vocab + 127) / 128;
+        launch_rmsnorm(st, true, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        GemmArgs lm = gemm_args(e, kGemmLmHead, d.vocab, vt, D, vt);
+        lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
+        lm.part_max = e->part_max; lm.part_idx = e->part_idx;
+        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
+        launch_argmax_final(st, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
+        e->launch_counter += 3;
+    }
+}
+
 static void enqueue_forward(llma_engine* e, bool lm_head) {
+    if (e->gemm_impl == LLMA_GEMM_TCGEN05) { enqueue_forward_tc(e, lm_head); return; }
+
     const ModelDims& d = e->dims;
     cudaStream_t st = e->stream;
     const bool b = e->bf16;

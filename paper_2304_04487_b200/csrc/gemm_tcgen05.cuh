@@ -1,0 +1,70 @@
+// Weight-streaming GEMM for the decoder's projections (library-private interface).
+//
+//   out[r, n] = sum_k W[n, k] * a[r, k],  r < 32 activation rows, W bf16 [n_out, k_in].
+//
+// The weight matrix is the MMA's M operand (128 output features per tile) and the 32
+// activation rows are its N operand, so every weight byte crosses HBM exactly once per
+// step however many rows are verified.  Work is the flat list of (tile, 64-wide k-chunk)
+// pairs, cut into equal contiguous ranges, one per CTA; partial tiles are summed in a fixed
+// order that depends on the matrix shape and grid only -- never on the rows in use.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace llma {
+
+enum GemmMode : int32_t {
+    kGemmQKV = 0,     // A maps = {wq, wk, wv}; rotary embedding; q -> qkv buffer, k/v -> cache
+    kGemmResid = 1,   // x[r, n] += acc
+    kGemmSwiGLU = 2,  // A maps = {w_gate, w_up}, 64 + 64 rows per tile; h = silu(g) * u (bf16)
+    kGemmLmHead = 3,  // per-tile (max, argmax) per row; optional logits store
+};
+
+struct GemmArgs {
+    int32_t mode;
+    int32_t n_out;          // output features (per matrix for QKV; d_ffn for SwiGLU)
+    int32_t n_tiles;        // tiles over all matrices
+    int32_t chunks;         // k_in / 64
+    int32_t tiles_per_map;  // tiles per A map
+    const RowDesc* rows;
+    float* ws;              // partial tiles [grid][2][128][32] fp32
+    int32_t* cnt;           // arrival counters [n_tiles], zero between launches
+    int32_t* dev_err;
+    float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
+    int32_t ld;             // leading dimension of out_f32
+    __nv_bfloat16* out_bf16;  // SwiGLU: h [32][d_ffn]
+    // QKV
+    ModelDims dims;
+    int32_t layer;
+    const float *rope_cos, *rope_sin;
+    __nv_bfloat16 *kcache, *vcache;
+    // LmHead
+    float* part_max;        // [n_tiles][32]
+    int32_t* part_idx;
+};
+
+constexpr int kGemmStages = 8;
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kGemmABytes = 128 * 64 * 2;
+constexpr uint32_t kGemmBBytes = kMaxRows * 64 * 2;
+constexpr size_t kGemmSmemBytes = 1024 + (size_t)kGemmStages * (kGemmABytes + kGemmBBytes) + 128 * 33 * 4 + 256;
+
+// grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)
+int gemm_grid_for(int64_t work, int num_sms);
+
+// Encode a 2-D bf16 row-major [rows, cols] tensor for TMA with a {64, box_rows} box and
+// 128-byte swizzle.  Returns a CUresult (0 = success).
+int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+// Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
+cudaError_t init_gemm_tcgen05();
+
+void launch_gemm_tcgen05(cudaStream_t st, int grid, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
+                         const CUtensorMap& a2, const CUtensorMap& b);
+
+// out_tok[r] = index of the largest logit over all tiles (lowest index on ties)
+void launch_argmax_final(cudaStream_t st, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
+                         int32_t n_tiles, int32_t* out_tok);
+
+}  // namespace llma

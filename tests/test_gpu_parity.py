@@ -50,7 +50,7 @@ def test_tiny_fp32_stepwise_parity():
 
 
 @pytest.mark.parametrize("name,n,k,P,N", [("tiny-bf16", 1, 8, 70, 48), ("small-bf16", 1, 5, 45, 40),
-                                           ("small-bf16", 2, 16, 33, 40)])
+                                           ("small-bf16", 2, 16, 33, 40), ("mid-bf16", 1, 8, 50, 32)])
 def test_bf16_stepwise_parity(name, n, k, P, N):
     shape = SHAPES[name]
     w = _weights(shape)
@@ -59,6 +59,7 @@ def test_bf16_stepwise_parity(name, n, k, P, N):
     y_star = _greedy_star(shape, w, prompt, N, max_seq)
     ref, offs, _ = build_reference(y_star, [60, 60, 40], 0.7, shape.vocab, seed=1)
     eng = _engine(shape, w, max_seq=max_seq, max_ref=200, max_k=k, keep_logits=True)
+    assert eng.llma_gemm_impl() == 2                     # bf16 shapes run the tensor-core GEMMs
     rep = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, offs, n, k, N, "bf16")
     assert rep.max_logit_err <= 2e-2
     assert rep.near_ties <= 3, rep.near_ties

@@ -61,6 +61,8 @@ SHAPES: Dict[str, ModelShape] = {
     "tiny-bf16": ModelShape("tiny-bf16", 2, 256, 4, 64, 1024, 4096, "bf16"),
     # head_dim 128 at small width, several row tiles and a ragged vocab tail
     "small-bf16": ModelShape("small-bf16", 3, 512, 4, 128, 1408, 5000, "bf16"),
+    # wide enough that every projection is split over several CTAs along k
+    "mid-bf16": ModelShape("mid-bf16", 2, 1024, 8, 128, 2816, 8000, "bf16"),
     "llama7b-shape": ModelShape("llama7b-shape", 32, 4096, 32, 128, 11008, 32000, "bf16"),
     "llama13b-shape": ModelShape("llama13b-shape", 40, 5120, 40, 128, 13824, 32000, "bf16"),
 }
