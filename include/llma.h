@@ -186,6 +186,39 @@ int llma_debug_kv_row(llma_engine *e, int32_t layer, int32_t seq, int32_t pos, i
 /* Committed K/V length of a sequence (prompt rows + emitted tokens - 1), or a negative status. */
 int llma_kv_len(llma_engine *e, int32_t seq);
 
+/* Kernel classes reported by llma_profile_steps. */
+enum {
+    LLMA_K_PLAN = 0,      /* trigger search + copy planning */
+    LLMA_K_EMBED,         /* embedding gather */
+    LLMA_K_NORM,          /* RMSNorm */
+    LLMA_K_GEMM_QKV,      /* QKV projection (tensor-core path: + rotary + K/V append) */
+    LLMA_K_ATTN,          /* causal attention over the K/V cache */
+    LLMA_K_GEMM_O,        /* output projection + residual */
+    LLMA_K_GEMM_GATEUP,   /* gate/up projections (tensor-core path: + SiLU gating) */
+    LLMA_K_GEMM_DOWN,     /* down projection + residual */
+    LLMA_K_GEMM_LMHEAD,   /* LM head (tensor-core path: + per-tile argmax) */
+    LLMA_K_ARGMAX,        /* final per-row argmax */
+    LLMA_K_ACCEPT,        /* acceptance + K/V commit */
+    LLMA_K_EPILOGUE,      /* separate rotary / gating kernels of the SIMT path */
+    LLMA_K_COUNT
+};
+
+typedef struct {
+    double ms[LLMA_K_COUNT];        /* stream time attributed to each class, summed over the steps */
+    int64_t launches[LLMA_K_COUNT]; /* kernel launches of each class */
+    int64_t steps;
+    double total_ms;
+} llma_profile;
+
+/*
+ * Measurement aid: run `steps` decoding steps exactly like llma_step (state advances, tokens
+ * are appended) but with a CUDA event recorded on the engine's stream after every kernel
+ * launch; the time between consecutive events is attributed to the kernel just launched.
+ * Launches are direct (no graph), so the figures include the gap to the previous kernel.
+ * Errors: as llma_step.
+ */
+int llma_profile_steps(llma_engine *e, int32_t n, int32_t k, int32_t steps, llma_profile *out);
+
 /* Which GEMM implementation the engine resolved to (LLMA_GEMM_SIMT or LLMA_GEMM_TCGEN05), or a
  * negative status. */
 int llma_gemm_impl(llma_engine *e);

@@ -35,6 +35,15 @@ class LlmaStepInfo(C.Structure):
     _fields_ = [("pos", C.c_int32), ("k_eff", C.c_int32), ("accepted", C.c_int32), ("emitted", C.c_int32)]
 
 
+K_NAMES = ("plan", "embed", "norm", "gemm_qkv", "attn", "gemm_o", "gemm_gateup", "gemm_down", "gemm_lmhead",
+           "argmax", "accept", "epilogue")
+
+
+class LlmaProfile(C.Structure):
+    _fields_ = [("ms", C.c_double * len(K_NAMES)), ("launches", C.c_int64 * len(K_NAMES)),
+                ("steps", C.c_int64), ("total_ms", C.c_double)]
+
+
 class LlmaError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -47,7 +56,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_gemm_impl", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -72,6 +81,7 @@ def lib() -> C.CDLL:
         L.llma_debug_kv_row.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_float)]
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
+        L.llma_profile_steps.argtypes = [vp, i32, i32, i32, C.POINTER(LlmaProfile)]
         L.llma_last_cuda_error.argtypes = []
         L.llma_strerror.argtypes = [C.c_int]
         L.llma_strerror.restype = C.c_char_p
@@ -199,6 +209,14 @@ class Engine:
 
     def llma_kv_len(self, seq: int) -> int:
         return self._check(lib().llma_kv_len(self._h, seq), "llma_kv_len")
+
+    def llma_profile_steps(self, n: int, k: int, steps: int) -> Dict[str, Dict[str, float]]:
+        pr = LlmaProfile()
+        self._check(lib().llma_profile_steps(self._h, n, k, steps, C.byref(pr)), "llma_profile_steps")
+        out = {name: {"ms_per_step": pr.ms[i] / pr.steps, "launches_per_step": pr.launches[i] / pr.steps}
+               for i, name in enumerate(K_NAMES) if pr.launches[i]}
+        out["_total"] = {"ms_per_step": pr.total_ms / pr.steps, "launches_per_step": float(sum(pr.launches)) / pr.steps}
+        return out
 
     def llma_gemm_impl(self) -> int:
         return self._check(lib().llma_gemm_impl(self._h), "llma_gemm_impl")

@@ -54,6 +54,7 @@ static void free_engine(llma_engine* e) {
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
     if (e->h_err) cudaFreeHost(e->h_err);
+    for (cudaEvent_t ev : e->prof_ev) cudaEventDestroy(ev);
     if (e->ev0) cudaEventDestroy(e->ev0);
     if (e->ev1) cudaEventDestroy(e->ev1);
     delete e;

@@ -53,6 +53,10 @@ struct llma_engine {
     int64_t launches_per_step = 0;
     int64_t launch_counter = 0;  // kernels enqueued since it was last cleared
     bool last_step_valid = false;
+    bool prof_on = false;               // llma_profile_steps: record an event after every launch
+    std::vector<cudaEvent_t> prof_ev;
+    std::vector<int> prof_cls;
+    size_t prof_n = 0;
     std::vector<int32_t> prompt_last;  // last prompt token of every sequence (the first pending input)
 };
 

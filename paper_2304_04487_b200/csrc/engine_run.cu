@@ -11,6 +11,20 @@ using namespace llma;
 // ---- one decoder forward over the rows described by e->rows ---------------------------------
 // Every kernel reads the row descriptors from device memory, so the same launch sequence
 // serves any mix of rows (greedy, copy steps, prompt chunks) and can be replayed as a graph.
+// When profiling is on, an event after every launch lets llma_profile_steps attribute the
+// stream time between consecutive events to the kernel class just launched.
+static inline void mark(llma_engine* e, int cls) {
+    if (!e->prof_on) return;
+    if (e->prof_n >= e->prof_ev.size()) {
+        cudaEvent_t ev = nullptr;
+        if (cudaEventCreate(&ev) != cudaSuccess) { e->prof_on = false; return; }
+        e->prof_ev.push_back(ev);
+        e->prof_cls.push_back(cls);
+    }
+    e->prof_cls[e->prof_n] = cls;
+    cudaEventRecord(e->prof_ev[e->prof_n++], e->stream);
+}
+
 static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int k_in, int tiles_per_map) {
     GemmArgs a;
     std::memset(&a, 0, sizeof(a));
@@ -34,31 +48,41 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     for (int l = 0; l < d.n_layers; ++l) {
         const llma_engine::LayerMaps& m = e->maps[l];
         launch_rmsnorm(st, true, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
         run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
+        mark(e, LLMA_K_GEMM_QKV);
         launch_attention_simt(st, true, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D;
         run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
+        mark(e, LLMA_K_GEMM_O);
         launch_rmsnorm(st, true, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         gu.out_bf16 = (__nv_bfloat16*)e->h;
         run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
+        mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D;
         run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->map_h);
+        mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 7;
     }
     if (lm_head) {
         const int vt = (d.vocab + 127) / 128;
         launch_rmsnorm(st, true, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         GemmArgs lm = gemm_args(e, kGemmLmHead, d.vocab, vt, D, vt);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
         run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
+        mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax_final(st, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
+        mark(e, LLMA_K_ARGMAX);
         e->launch_counter += 3;
     }
 }
@@ -72,23 +96,38 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
     for (int l = 0; l < d.n_layers; ++l) {
         launch_rmsnorm(st, b, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->wq[l], e->x_hat, e->qkv, HD, D, 3 * HD, false);
+        mark(e, LLMA_K_GEMM_QKV);
         launch_gemm_simt(st, b, e->rows, e->wk[l], e->x_hat, e->qkv + HD, HD, D, 3 * HD, false);
+        mark(e, LLMA_K_GEMM_QKV);
         launch_gemm_simt(st, b, e->rows, e->wv[l], e->x_hat, e->qkv + 2 * HD, HD, D, 3 * HD, false);
+        mark(e, LLMA_K_GEMM_QKV);
         launch_qkv_post(st, b, d, l, e->rows, e->qkv, e->rope_cos, e->rope_sin, e->kcache, e->vcache);
+        mark(e, LLMA_K_EPILOGUE);
         launch_attention_simt(st, b, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        mark(e, LLMA_K_ATTN);
         launch_gemm_simt(st, b, e->rows, e->wo[l], e->attn, e->x, D, HD, D, true);
+        mark(e, LLMA_K_GEMM_O);
         launch_rmsnorm(st, b, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->w_gate[l], e->x_hat, e->gate_up, F, D, 2 * F, false);
+        mark(e, LLMA_K_GEMM_GATEUP);
         launch_gemm_simt(st, b, e->rows, e->w_up[l], e->x_hat, e->gate_up + F, F, D, 2 * F, false);
+        mark(e, LLMA_K_GEMM_GATEUP);
         launch_silu_mul(st, b, e->rows, e->gate_up, e->h, F);
+        mark(e, LLMA_K_EPILOGUE);
         launch_gemm_simt(st, b, e->rows, e->w_down[l], e->h, e->x, D, F, D, true);
+        mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 12;
     }
     if (lm_head) {
         launch_rmsnorm(st, b, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->lm_head, e->x_hat, e->logits, d.vocab, D, d.vocab, false);
+        mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax(st, e->rows, e->logits, d.vocab, e->out_tok);
+        mark(e, LLMA_K_ARGMAX);
         e->launch_counter += 3;
     }
 }
@@ -98,10 +137,13 @@ static void enqueue_step(llma_engine* e, int n, int k) {
     const ModelDims& d = e->dims;
     launch_plan(e->stream, d, e->seq_state, e->rows, e->ref, e->doc_start, e->doc_end, e->y, e->y_cap, n, k,
                 e->dev_err);
+    mark(e, LLMA_K_PLAN);
     launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+    mark(e, LLMA_K_EMBED);
     e->launch_counter += 3;
     enqueue_forward(e, true);
     launch_accept(e->stream, d, e->seq_state, e->ref, e->out_tok, e->y, e->y_cap);
+    mark(e, LLMA_K_ACCEPT);
     e->launch_counter += 1;
 }
 
@@ -154,6 +196,7 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
         R->max_pos = p0 + cnt - 1;
         CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));
         launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+        mark(e, LLMA_K_EMBED);
         enqueue_forward(e, false);
         CU_TRY(cudaGetLastError());
         CU_TRY(cudaStreamSynchronize(e->stream));  // h_rows is reused by the next chunk
@@ -341,5 +384,49 @@ extern "C" int llma_generate(llma_engine* e, int32_t max_new, int32_t n, int32_t
     CU_TRY(cudaEventElapsedTime(&st.device_ms, e->ev0, e->ev1));
     if (stats) *stats = st;
     e->last_step_valid = launches > 0;
+    return LLMA_OK;
+}
+
+extern "C" int llma_profile_steps(llma_engine* e, int32_t n, int32_t k, int32_t steps, llma_profile* out) {
+    if (!e || !out) return LLMA_ERR_NULL;
+    int rc = check_nk(e, n, k);
+    if (rc) return rc;
+    if (steps < 1) return LLMA_ERR_ARG;
+    std::memset(out, 0, sizeof(*out));
+    std::vector<int32_t> toks((size_t)e->dims.max_batch * e->dims.kp1), cnt((size_t)e->dims.max_batch);
+    for (int i = 0; i < steps; ++i) {
+        // same state handling as llma_step, but the launches are bracketed by events
+        rc = read_state(e);
+        if (rc) return rc;
+        bool any = false;
+        for (int s = 0; s < e->dims.max_batch; ++s) {
+            SeqState& S = e->h_state[s];
+            if (!S.active) continue;
+            if (S.kv_len + 1 > e->dims.max_seq) return LLMA_ERR_CAPACITY;
+            S.target_len = std::min(e->y_cap, S.y_len + (e->dims.max_seq - S.kv_len));
+            S.done = 0;
+            rc = write_state(e, s);
+            if (rc) return rc;
+            any = true;
+        }
+        if (!any) return LLMA_ERR_STATE;
+        e->prof_on = true;
+        e->prof_n = 0;
+        mark(e, -1);
+        enqueue_step(e, n, k);
+        e->prof_on = false;
+        CU_TRY(cudaGetLastError());
+        rc = check_device_error(e);
+        if (rc) return rc;
+        for (size_t j = 1; j < e->prof_n; ++j) {
+            float ms = 0.f;
+            CU_TRY(cudaEventElapsedTime(&ms, e->prof_ev[j - 1], e->prof_ev[j]));
+            const int c = e->prof_cls[j];
+            if (c >= 0 && c < LLMA_K_COUNT) { out->ms[c] += ms; out->launches[c] += 1; }
+            out->total_ms += ms;
+        }
+        out->steps += 1;
+    }
+    e->last_step_valid = true;
     return LLMA_OK;
 }

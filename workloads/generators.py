@@ -4,7 +4,8 @@ Everything here is input data: normal/uniform draws, bf16 storage conversion of
 the drawn weights, and the splicing of token spans into reference documents.
 No decoding arithmetic lives in this file.
 
-Streams (all numpy Philox, keyed by (seed, stream id)) so that every tensor can
+Streams (numpy SFC64 seeded by (seed, tensor index) for weights, Philox keyed by
+(seed, stream id) for tokens) so that every tensor can
 be regenerated on its own and in parallel:
     weights  seed 0   one stream per tensor (index in ``weight_names``)
     prompt   seed 1
@@ -89,10 +90,14 @@ def _weight_dims(shape: ModelShape, name: str) -> Tuple[int, ...]:
 
 def bf16_bits_from_f32(x: np.ndarray) -> np.ndarray:
     """Storage conversion fp32 -> bf16 bit patterns (round to nearest, ties to even)."""
-    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
-    lsb = (u >> np.uint32(16)) & np.uint32(1)
-    r = u + np.uint32(0x7FFF) + lsb
-    return (r >> np.uint32(16)).astype(np.uint16)
+    u = np.array(x, dtype=np.float32, copy=True, order="C").view(np.uint32)
+    shape = u.shape
+    u = u.reshape(-1)
+    lsb = u >> np.uint32(16)
+    lsb &= np.uint32(1)
+    u += np.uint32(0x7FFF)
+    u += lsb
+    return np.ascontiguousarray(u.view(np.uint16)[1::2]).reshape(shape)   # high halves (little endian)
 
 
 def f32_from_bf16_bits(b: np.ndarray) -> np.ndarray:
@@ -105,7 +110,7 @@ def _gen_one(shape: ModelShape, name: str, index: int, seed: int, std: float) ->
     if len(dims) == 1:  # norm gains
         g = np.ones(dims, dtype=np.float32)
         return g
-    rng = np.random.Generator(np.random.Philox(key=[seed, index]))
+    rng = np.random.Generator(np.random.SFC64(np.random.SeedSequence([seed, index])))
     rows, cols = dims
     out_dtype = np.float32 if shape.dtype == "fp32" else np.uint16
     out = np.empty(dims, dtype=out_dtype)
