@@ -219,6 +219,17 @@ typedef struct {
  */
 int llma_profile_steps(llma_engine *e, int32_t n, int32_t k, int32_t steps, llma_profile *out);
 
+/*
+ * The engine's projection kernel on its own: out[r, n] = sum_k W[n, k] * a[r, k] for the 32
+ * activation rows a step can hold (Eq. 3 evaluates k+1 <= 32 positions against every weight
+ * matrix in one pass).  W: device, bf16, row-major [n_out, k_in]; a: device, bf16, row-major
+ * [32, k_in]; out: device, fp32, row-major [32, n_out].  k_in must be a multiple of 64; W and a
+ * 16-byte aligned.  Allocates its split-k scratch with cudaMalloc and frees it before returning;
+ * synchronous.  Errors: NULL, ARG, CONFIG (not an sm_100 device), CUDA, DEVICE_TIMEOUT.
+ */
+int llma_gemm_rows32_bf16(const void *W, const void *a, float *out, int32_t n_out, int32_t k_in,
+                          void *cuda_stream);
+
 /* Which GEMM implementation the engine resolved to (LLMA_GEMM_SIMT or LLMA_GEMM_TCGEN05), or a
  * negative status. */
 int llma_gemm_impl(llma_engine *e);

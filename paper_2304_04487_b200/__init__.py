@@ -11,5 +11,6 @@ from .binding import (  # noqa: F401
     LlmaStats,
     LlmaStepInfo,
     lib,
+    llma_gemm_rows32_bf16,
     LIB_PATH,
 )

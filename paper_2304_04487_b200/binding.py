@@ -56,7 +56,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -81,6 +81,7 @@ def lib() -> C.CDLL:
         L.llma_debug_kv_row.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_float)]
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
+        L.llma_gemm_rows32_bf16.argtypes = [vp, vp, vp, i32, i32, vp]
         L.llma_profile_steps.argtypes = [vp, i32, i32, i32, C.POINTER(LlmaProfile)]
         L.llma_last_cuda_error.argtypes = []
         L.llma_strerror.argtypes = [C.c_int]
@@ -98,6 +99,19 @@ def _i32(a) -> np.ndarray:
 
 def _pi32(a: np.ndarray):
     return a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def llma_gemm_rows32_bf16(W, a, out, stream=None) -> None:
+    """W [n_out, k_in] bf16, a [32, k_in] bf16, out [32, n_out] fp32: CUDA torch tensors (device memory only)."""
+    import torch
+    assert W.dtype == torch.bfloat16 and a.dtype == torch.bfloat16 and out.dtype == torch.float32
+    assert W.is_contiguous() and a.is_contiguous() and out.is_contiguous() and a.shape[0] == 32
+    n_out, k_in = W.shape
+    assert a.shape[1] == k_in and tuple(out.shape) == (32, n_out)
+    st = stream if stream is not None else torch.cuda.current_stream(W.device)
+    rc = lib().llma_gemm_rows32_bf16(W.data_ptr(), a.data_ptr(), out.data_ptr(), n_out, k_in, st.cuda_stream)
+    if rc != 0:
+        raise LlmaError(rc, "llma_gemm_rows32_bf16")
 
 
 class Engine:

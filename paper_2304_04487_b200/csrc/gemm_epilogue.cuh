@@ -21,6 +21,16 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
         if (j < rows_used) g.out_f32[(int64_t)j * g.ld + col] += acc[j];
 }
 
+// out[r, n] = acc
+__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int row, const float (&acc)[32],
+                                               int rows_used) {
+    const int col = tile * 128 + row;
+    if (col >= g.n_out) return;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        if (j < rows_used) g.out_f32[(int64_t)j * g.ld + col] = acc[j];
+}
+
 // QKV: rotary embedding on q and k (pair (i, i + hd/2)), q to the fp32 qkv buffer, k and v
 // rows into the bf16 cache at (sequence, position) of every used row.
 __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, const float (&acc)[32],

@@ -18,17 +18,13 @@ namespace llma {
 
 using namespace ptx;
 
-struct Segment {
-    int tile, c0, c1;
-};
-
 // Range of flat (tile, chunk) work items owned by CTA b of G.
 __device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b) {
-    const int rows_used = g.rows->rows_used;
+    const int rows_used = g.rows ? g.rows->rows_used : kMaxRows;
     if (rows_used <= 0) return;  // uniform over the grid: nothing to verify this step
 
     extern __shared__ uint8_t smem_raw[];
@@ -199,6 +195,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 case kGemmQKV: epilogue_qkv(g, tile, row, acc, rows_used, stage); break;
                 case kGemmResid: epilogue_resid(g, tile, row, acc, rows_used); break;
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, acc, rows_used, stage); break;
+                case kGemmStore: epilogue_store(g, tile, row, acc, rows_used); break;
                 default: epilogue_lmhead(g, tile, row, acc, rows_used, stage); break;
             }
         }

@@ -19,6 +19,7 @@ enum GemmMode : int32_t {
     kGemmResid = 1,   // x[r, n] += acc
     kGemmSwiGLU = 2,  // A maps = {w_gate, w_up}, 64 + 64 rows per tile; h = silu(g) * u (bf16)
     kGemmLmHead = 3,  // per-tile (max, argmax) per row; optional logits store
+    kGemmStore = 4,   // out[r, n] = acc for all 32 rows (stand-alone product)
 };
 
 struct GemmArgs {
@@ -27,7 +28,7 @@ struct GemmArgs {
     int32_t n_tiles;        // tiles over all matrices
     int32_t chunks;         // k_in / 64
     int32_t tiles_per_map;  // tiles per A map
-    const RowDesc* rows;
+    const RowDesc* rows;    // nullptr: all 32 rows are in use
     float* ws;              // partial tiles [grid][2][128][32] fp32
     int32_t* cnt;           // arrival counters [n_tiles], zero between launches
     int32_t* dev_err;
