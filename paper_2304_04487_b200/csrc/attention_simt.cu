@@ -39,7 +39,8 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(ModelDims dims, int
                                                              const RowDesc* __restrict__ rows,
                                                              const float* __restrict__ qkv,
                                                              const T* __restrict__ kcache,
-                                                             const T* __restrict__ vcache, T* __restrict__ attn_out) {
+                                                             const T* __restrict__ vcache, void* __restrict__ attn_out,
+                                                             int act_layout) {
     const int head = blockIdx.x, r = blockIdx.y;
     const int pos = rows->pos[r];
     if (pos < 0) return;
@@ -88,9 +89,8 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(ModelDims dims, int
 #pragma unroll
             for (int e = 0; e < EPL; ++e) num[e] += f * sacc[w][lane * EPL + e];
         }
-        T* o = attn_out + (int64_t)r * HD + head * hd + lane * EPL;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) o[e] = from_f32<T>(num[e] / den);
+        for (int e = 0; e < EPL; ++e) store_act(attn_out, act_layout, r, head * hd + lane * EPL + e, HD, num[e] / den);
     }
 }
 
@@ -106,17 +106,17 @@ void launch_qkv_post(cudaStream_t st, bool bf16, const ModelDims& dims, int laye
 }
 
 void launch_attention_simt(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, const RowDesc* rows,
-                           const float* qkv, const void* kcache, const void* vcache, void* attn_out) {
+                           const float* qkv, const void* kcache, const void* vcache, void* attn_out, int act_layout) {
     dim3 grid(dims.n_heads, kMaxRows);
     const bool hd128 = dims.head_dim == 128;
     if (bf16) {
-        auto K = (const __nv_bfloat16*)kcache; auto V = (const __nv_bfloat16*)vcache; auto O = (__nv_bfloat16*)attn_out;
-        if (hd128) attention_simt_kernel<__nv_bfloat16, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, O);
-        else attention_simt_kernel<__nv_bfloat16, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, O);
+        auto K = (const __nv_bfloat16*)kcache; auto V = (const __nv_bfloat16*)vcache;
+        if (hd128) attention_simt_kernel<__nv_bfloat16, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        else attention_simt_kernel<__nv_bfloat16, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
     } else {
-        auto K = (const float*)kcache; auto V = (const float*)vcache; auto O = (float*)attn_out;
-        if (hd128) attention_simt_kernel<float, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, O);
-        else attention_simt_kernel<float, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, O);
+        auto K = (const float*)kcache; auto V = (const float*)vcache;
+        if (hd128) attention_simt_kernel<float, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        else attention_simt_kernel<float, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
     }
 }
 

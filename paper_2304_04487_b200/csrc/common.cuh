@@ -55,6 +55,24 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// Activations that feed a projection are kept in one of two layouts:
+//   kActF32   fp32 [kMaxRows][K]                       (CUDA-core GEMM)
+//   kActSplit bf16 [2*kMaxRows][K]: row r holds hi = bf16(v), row kMaxRows + r holds
+//             lo = bf16(v - hi), so hi + lo carries 16 mantissa bits through a bf16 tensor-core
+//             product (the two halves are summed in the GEMM's fp32 accumulator epilogue)
+enum ActLayout : int32_t { kActF32 = 0, kActSplit = 1 };
+
+__device__ __forceinline__ void store_act(void* buf, int layout, int r, int64_t i, int64_t K, float v) {
+    if (layout == kActF32) {
+        reinterpret_cast<float*>(buf)[(int64_t)r * K + i] = v;
+    } else {
+        __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(buf);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        b[(int64_t)r * K + i] = hi;
+        b[(int64_t)(kMaxRows + r) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+}
+
 // K/V cache addressing: [layer][seq][head][max_seq][head_dim]; returns the row index
 __host__ __device__ __forceinline__ int64_t kv_row_index(const ModelDims& d, int layer, int seq, int head, int pos) {
     return ((((int64_t)layer * d.max_batch + seq) * d.n_heads + head) * d.max_seq + pos);

@@ -128,9 +128,10 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     CREATE_TRY(dalloc(&e->qkv, (size_t)kMaxRows * 3 * HD));
     CREATE_TRY(dalloc(&e->gate_up, (size_t)kMaxRows * 2 * d.d_ffn));
     CREATE_TRY(dalloc(&e->logits, (size_t)kMaxRows * d.vocab));
-    CREATE_TRY(dalloc((char**)&e->x_hat, (size_t)kMaxRows * d.d_model * es));
-    CREATE_TRY(dalloc((char**)&e->attn, (size_t)kMaxRows * HD * es));
-    CREATE_TRY(dalloc((char**)&e->h, (size_t)kMaxRows * d.d_ffn * es));
+    // activation operands: fp32 [32][K] (CUDA-core GEMM) or split bf16 [64][K] (tensor cores): 4 bytes each
+    CREATE_TRY(dalloc((char**)&e->x_hat, (size_t)kMaxRows * d.d_model * 4));
+    CREATE_TRY(dalloc((char**)&e->attn, (size_t)kMaxRows * HD * 4));
+    CREATE_TRY(dalloc((char**)&e->h, (size_t)kMaxRows * d.d_ffn * 4));
     const size_t kv_elems = (size_t)L * B * d.n_heads * d.max_seq * d.head_dim;
     CREATE_TRY(dalloc((char**)&e->kcache, kv_elems * es));
     CREATE_TRY(dalloc((char**)&e->vcache, kv_elems * es));
@@ -176,9 +177,9 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
             bad |= make_tensor_map_bf16(&m.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
         }
         bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
-        bad |= make_tensor_map_bf16(&e->map_x_hat, e->x_hat, kMaxRows, d.d_model, kMaxRows);
-        bad |= make_tensor_map_bf16(&e->map_attn, e->attn, kMaxRows, HD, kMaxRows);
-        bad |= make_tensor_map_bf16(&e->map_h, e->h, kMaxRows, d.d_ffn, kMaxRows);
+        bad |= make_tensor_map_bf16(&e->map_x_hat, e->x_hat, kGemmN, d.d_model, kGemmN);
+        bad |= make_tensor_map_bf16(&e->map_attn, e->attn, kGemmN, HD, kGemmN);
+        bad |= make_tensor_map_bf16(&e->map_h, e->h, kGemmN, d.d_ffn, kGemmN);
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
         CREATE_TRY(init_gemm_tcgen05());
     }

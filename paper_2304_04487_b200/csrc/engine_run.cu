@@ -47,23 +47,23 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
     for (int l = 0; l < d.n_layers; ++l) {
         const llma_engine::LayerMaps& m = e->maps[l];
-        launch_rmsnorm(st, true, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
         run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
         mark(e, LLMA_K_GEMM_QKV);
-        launch_attention_simt(st, true, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        launch_attention_simt(st, true, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn, kActSplit);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D;
         run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
         mark(e, LLMA_K_GEMM_O);
-        launch_rmsnorm(st, true, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
-        gu.out_bf16 = (__nv_bfloat16*)e->h;
+        gu.out_act = e->h;
         run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
         mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
@@ -74,7 +74,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     }
     if (lm_head) {
         const int vt = (d.vocab + 127) / 128;
-        launch_rmsnorm(st, true, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         GemmArgs lm = gemm_args(e, kGemmLmHead, d.vocab, vt, D, vt);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
@@ -95,36 +95,36 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
     const bool b = e->bf16;
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
     for (int l = 0; l < d.n_layers; ++l) {
-        launch_rmsnorm(st, b, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
-        launch_gemm_simt(st, b, e->rows, e->wq[l], e->x_hat, e->qkv, HD, D, 3 * HD, false);
+        launch_gemm_simt(st, b, e->rows, e->wq[l], (const float*)e->x_hat, e->qkv, HD, D, 3 * HD, false);
         mark(e, LLMA_K_GEMM_QKV);
-        launch_gemm_simt(st, b, e->rows, e->wk[l], e->x_hat, e->qkv + HD, HD, D, 3 * HD, false);
+        launch_gemm_simt(st, b, e->rows, e->wk[l], (const float*)e->x_hat, e->qkv + HD, HD, D, 3 * HD, false);
         mark(e, LLMA_K_GEMM_QKV);
-        launch_gemm_simt(st, b, e->rows, e->wv[l], e->x_hat, e->qkv + 2 * HD, HD, D, 3 * HD, false);
+        launch_gemm_simt(st, b, e->rows, e->wv[l], (const float*)e->x_hat, e->qkv + 2 * HD, HD, D, 3 * HD, false);
         mark(e, LLMA_K_GEMM_QKV);
         launch_qkv_post(st, b, d, l, e->rows, e->qkv, e->rope_cos, e->rope_sin, e->kcache, e->vcache);
         mark(e, LLMA_K_EPILOGUE);
-        launch_attention_simt(st, b, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn);
+        launch_attention_simt(st, b, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn, kActF32);
         mark(e, LLMA_K_ATTN);
-        launch_gemm_simt(st, b, e->rows, e->wo[l], e->attn, e->x, D, HD, D, true);
+        launch_gemm_simt(st, b, e->rows, e->wo[l], (const float*)e->attn, e->x, D, HD, D, true);
         mark(e, LLMA_K_GEMM_O);
-        launch_rmsnorm(st, b, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
-        launch_gemm_simt(st, b, e->rows, e->w_gate[l], e->x_hat, e->gate_up, F, D, 2 * F, false);
+        launch_gemm_simt(st, b, e->rows, e->w_gate[l], (const float*)e->x_hat, e->gate_up, F, D, 2 * F, false);
         mark(e, LLMA_K_GEMM_GATEUP);
-        launch_gemm_simt(st, b, e->rows, e->w_up[l], e->x_hat, e->gate_up + F, F, D, 2 * F, false);
+        launch_gemm_simt(st, b, e->rows, e->w_up[l], (const float*)e->x_hat, e->gate_up + F, F, D, 2 * F, false);
         mark(e, LLMA_K_GEMM_GATEUP);
-        launch_silu_mul(st, b, e->rows, e->gate_up, e->h, F);
+        launch_silu_mul(st, e->rows, e->gate_up, (float*)e->h, F);
         mark(e, LLMA_K_EPILOGUE);
-        launch_gemm_simt(st, b, e->rows, e->w_down[l], e->h, e->x, D, F, D, true);
+        launch_gemm_simt(st, b, e->rows, e->w_down[l], (const float*)e->h, e->x, D, F, D, true);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 12;
     }
     if (lm_head) {
-        launch_rmsnorm(st, b, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
-        launch_gemm_simt(st, b, e->rows, e->lm_head, e->x_hat, e->logits, d.vocab, D, d.vocab, false);
+        launch_gemm_simt(st, b, e->rows, e->lm_head, (const float*)e->x_hat, e->logits, d.vocab, D, d.vocab, false);
         mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax(st, e->rows, e->logits, d.vocab, e->out_tok);
         mark(e, LLMA_K_ARGMAX);

@@ -6,12 +6,13 @@
 using namespace llma;
 
 namespace llma {
-// Shared by the stand-alone entry points: checks, TMA descriptors, one launch.
+// Shared by the stand-alone entry points: TMA descriptors and one launch.  `a` is the split
+// activation buffer [64][k_in] (hi rows, then lo rows).
 int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, int32_t k_in, float* ws,
                        int32_t* cnt, int32_t* dev_err, int grid, cudaStream_t st) {
     CUtensorMap ma, mb;
     if (make_tensor_map_bf16(&ma, W, (uint64_t)n_out, (uint64_t)k_in, 128) != 0) return LLMA_ERR_ARG;
-    if (make_tensor_map_bf16(&mb, a, kMaxRows, (uint64_t)k_in, kMaxRows) != 0) return LLMA_ERR_ARG;
+    if (make_tensor_map_bf16(&mb, a, kGemmN, (uint64_t)k_in, kGemmN) != 0) return LLMA_ERR_ARG;
     GemmArgs g;
     std::memset(&g, 0, sizeof(g));
     g.mode = kGemmStore; g.n_out = n_out; g.n_tiles = (n_out + 127) / 128; g.chunks = k_in / 64;
@@ -37,19 +38,25 @@ extern "C" int llma_gemm_rows32_bf16(const void* W, const void* a, float* out, i
     const int n_tiles = (n_out + 127) / 128;
     const int grid = gemm_grid_for((int64_t)n_tiles * (k_in / 64), prop.multiProcessorCount);
     float* ws = nullptr;
-    int32_t* cnt = nullptr;  // counters, then one error word
+    int32_t* cnt = nullptr;   // counters, then one error word
+    __nv_bfloat16* a2 = nullptr;  // the kernel's operand: rows 0..31 = a, rows 32..63 = 0 (no low half)
+    const size_t a_bytes = (size_t)kMaxRows * k_in * sizeof(__nv_bfloat16);
     CU_TRY(cudaMalloc((void**)&ws, (size_t)grid * 2 * 128 * 32 * sizeof(float)));
     cudaError_t ce = cudaMalloc((void**)&cnt, ((size_t)n_tiles + 1) * sizeof(int32_t));
-    if (ce != cudaSuccess) { cudaFree(ws); llma::note_cuda_error(ce); return LLMA_ERR_CUDA; }
+    if (ce == cudaSuccess) ce = cudaMalloc((void**)&a2, 2 * a_bytes);
+    if (ce != cudaSuccess) { cudaFree(ws); cudaFree(cnt); llma::note_cuda_error(ce); return LLMA_ERR_CUDA; }
     int rc = LLMA_OK;
     int32_t err = 0;
     ce = cudaMemsetAsync(cnt, 0, ((size_t)n_tiles + 1) * sizeof(int32_t), st);
-    if (ce == cudaSuccess) rc = gemm_rows32_launch(W, a, out, n_out, k_in, ws, cnt, cnt + n_tiles, grid, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(a2, a, a_bytes, cudaMemcpyDeviceToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync((char*)a2 + a_bytes, 0, a_bytes, st);
+    if (ce == cudaSuccess) rc = gemm_rows32_launch(W, a2, out, n_out, k_in, ws, cnt, cnt + n_tiles, grid, st);
     if (ce == cudaSuccess && rc == LLMA_OK)
         ce = cudaMemcpyAsync(&err, cnt + n_tiles, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
     cudaFree(ws);
     cudaFree(cnt);
+    cudaFree(a2);
     if (ce != cudaSuccess) { llma::note_cuda_error(ce); return LLMA_ERR_CUDA; }
     if (rc) return rc;
     return err == kDevErrNone ? LLMA_OK : LLMA_ERR_DEVICE_TIMEOUT;

@@ -77,7 +77,7 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
     if (f < g.n_out) {
         for (int j = row >> 6; j < rows_used; j += 2) {
             const float gate = stage[fi][j], up = stage[64 + fi][j];
-            g.out_bf16[(int64_t)j * g.n_out + f] = __float2bfloat16_rn(gate / (1.f + expf(-gate)) * up);
+            store_act(g.out_act, kActSplit, j, f, g.n_out, gate / (1.f + expf(-gate)) * up);
         }
     }
     epi_sync();

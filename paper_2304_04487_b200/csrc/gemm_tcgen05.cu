@@ -5,7 +5,7 @@
 //   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue
 //   warp  4    producer: one thread issues the TMA loads of weight and activation tiles
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
-// Two accumulators (2 x 32 TMEM columns) let the epilogue of one tile overlap the MMAs of
+// Two accumulators (2 x 64 TMEM columns: 32 for the hi half of the activations, 32 for lo) let the epilogue of one tile overlap the MMAs of
 // the next.  Every wait is bounded: when one runs out the kernel raises the device error
 // word, stops issuing work, lets its outstanding copies land, frees TMEM and returns.
 #include <cuda.h>
@@ -55,7 +55,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         fence_mbar_init();
     }
     if (warp == 5) {
-        tmem_alloc(smem_u32((const void*)&sh[0]), 64);
+        tmem_alloc(smem_u32((const void*)&sh[0]), 2 * kGemmN);
         tmem_relinquish();
     }
     if (warp == 4 && lane == 0) {
@@ -99,7 +99,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else if (warp == 5) {
         // ------------------------------- MMA issuer ---------------------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_m128(kMaxRows);
+            constexpr uint32_t idesc = idesc_bf16_m128(kGemmN);
             int64_t it = 0;
             int seg = 0;
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
@@ -109,7 +109,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const uint32_t use = (uint32_t)(seg >> 1);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxRows;
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kGemmN;
                 for (int c = c0; c < c1; ++c, ++it) {
                     const int s = (int)(it % kGemmStages);
                     const uint32_t ph = (uint32_t)((it / kGemmStages) & 1);
@@ -148,7 +148,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             if (!ok) break;
             tc_fence_after();
             float acc[32];
-            tmem_ld_32cols(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * kMaxRows, acc);
+            {
+                float lo[32];
+                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * kGemmN;
+                tmem_ld_32cols(t0, acc);
+                tmem_ld_32cols(t0 + kMaxRows, lo);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
@@ -204,7 +211,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 64);
+        tmem_dealloc(tmem_base, 2 * kGemmN);
     }
 }
 

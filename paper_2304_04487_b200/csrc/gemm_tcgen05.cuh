@@ -2,7 +2,11 @@
 //
 //   out[r, n] = sum_k W[n, k] * a[r, k],  r < 32 activation rows, W bf16 [n_out, k_in].
 //
-// The weight matrix is the MMA's M operand (128 output features per tile) and the 32
+// The activations arrive split into two bf16 halves (ActLayout kActSplit: 64 rows, hi then lo);
+// the MMA's N dimension is those 64 rows and the epilogue adds the hi and lo columns, so the
+// product keeps 16 mantissa bits of the activations at no cost in weight traffic.
+//
+// The weight matrix is the MMA's M operand (128 output features per tile) and the
 // activation rows are its N operand, so every weight byte crosses HBM exactly once per
 // step however many rows are verified.  Work is the flat list of (tile, 64-wide k-chunk)
 // pairs, cut into equal contiguous ranges, one per CTA; partial tiles are summed in a fixed
@@ -34,7 +38,7 @@ struct GemmArgs {
     int32_t* dev_err;
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
     int32_t ld;             // leading dimension of out_f32
-    __nv_bfloat16* out_bf16;  // SwiGLU: h [32][d_ffn]
+    void* out_act;          // SwiGLU: h in ActLayout kActSplit [64][d_ffn]
     // QKV
     ModelDims dims;
     int32_t layer;
@@ -45,10 +49,11 @@ struct GemmArgs {
     int32_t* part_idx;
 };
 
-constexpr int kGemmStages = 8;
+constexpr int kGemmStages = 7;
+constexpr int kGemmN = 2 * kMaxRows;  // MMA N: hi rows then lo rows
 constexpr int kGemmThreads = 192;
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
-constexpr uint32_t kGemmBBytes = kMaxRows * 64 * 2;
+constexpr uint32_t kGemmBBytes = kGemmN * 64 * 2;
 constexpr size_t kGemmSmemBytes = 1024 + (size_t)kGemmStages * (kGemmABytes + kGemmBBytes) + 128 * 33 * 4 + 256;
 
 // grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)

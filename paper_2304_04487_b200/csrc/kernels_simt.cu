@@ -10,15 +10,13 @@
 namespace llma {
 
 // ---- RMSNorm -----------------------------------------------------------------------------
-template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ x,
-                                                      const float* __restrict__ g, T* __restrict__ out, int d,
-                                                      float eps) {
+                                                      const float* __restrict__ g, void* __restrict__ out, int layout,
+                                                      int d, float eps) {
     const int r = blockIdx.x;
     const float* xr = x + (int64_t)r * d;
-    T* orow = out + (int64_t)r * d;
     if (rows->pos[r] < 0) {
-        for (int i = threadIdx.x; i < d; i += blockDim.x) orow[i] = from_f32<T>(0.f);
+        for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, r, i, d, 0.f);
         return;
     }
     float ss = 0.f;
@@ -30,7 +28,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const RowDesc* __restrict_
     float tot = 0.f;
     for (int w = 0; w < 8; ++w) tot += red[w];  // fixed order
     const float inv = rsqrtf(tot / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) orow[i] = from_f32<T>(xr[i] * inv * g[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, r, i, d, xr[i] * inv * g[i]);
 }
 
 // ---- small-M GEMM: one warp per output feature --------------------------------------------
@@ -59,7 +57,7 @@ template <> struct Vec16<__nv_bfloat16> {
 
 template <typename T, int RB>  // RB rows handled per pass over the weight row
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const RowDesc* __restrict__ rows, const T* __restrict__ W,
-                                                        const T* __restrict__ a, float* __restrict__ out, int n_out,
+                                                        const float* __restrict__ a, float* __restrict__ out, int n_out,
                                                         int k_in, int ld_out, int accumulate) {
     constexpr int V = Vec16<T>::N;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -77,10 +75,14 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const RowDesc* __restric
 #pragma unroll
             for (int r = 0; r < RB; ++r) {
                 if (r0 + r < rows_used) {
-                    float av[V];
-                    Vec16<T>::load(a + (int64_t)(r0 + r) * k_in + kk, av);
+                    const float* ap = a + (int64_t)(r0 + r) * k_in + kk;
 #pragma unroll
-                    for (int v = 0; v < V; ++v) acc[r] = fmaf(wv[v], av[v], acc[r]);
+                    for (int v4 = 0; v4 < V; v4 += 4) {
+                        float av[4];
+                        Vec16<float>::load(ap + v4, av);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) acc[r] = fmaf(wv[v4 + v], av[v], acc[r]);
+                    }
                 }
             }
         }
@@ -97,9 +99,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const RowDesc* __restric
 }
 
 // ---- SiLU gating ----------------------------------------------------------------------------
-template <typename T>
 __global__ void silu_mul_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ gate_up,
-                                T* __restrict__ h, int d_ffn) {
+                                float* __restrict__ h, int d_ffn) {
     const int r = blockIdx.y;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= d_ffn) return;
@@ -109,7 +110,7 @@ __global__ void silu_mul_kernel(const RowDesc* __restrict__ rows, const float* _
         const float u = gate_up[(int64_t)r * 2 * d_ffn + d_ffn + i];
         v = g / (1.f + expf(-g)) * u;
     }
-    h[(int64_t)r * d_ffn + i] = from_f32<T>(v);
+    h[(int64_t)r * d_ffn + i] = v;
 }
 
 // ---- per-row argmax, lowest index on ties --------------------------------------------------
@@ -139,28 +140,25 @@ __global__ void __launch_bounds__(256) argmax_kernel(const RowDesc* __restrict__
 }
 
 // ---- launchers -------------------------------------------------------------------------------
-void launch_rmsnorm(cudaStream_t st, bool bf16, const RowDesc* rows, const float* x, const float* g, void* x_hat,
+void launch_rmsnorm(cudaStream_t st, int act_layout, const RowDesc* rows, const float* x, const float* g, void* x_hat,
                     int32_t d, float eps) {
-    if (bf16) rmsnorm_kernel<__nv_bfloat16><<<kMaxRows, 256, 0, st>>>(rows, x, g, (__nv_bfloat16*)x_hat, d, eps);
-    else rmsnorm_kernel<float><<<kMaxRows, 256, 0, st>>>(rows, x, g, (float*)x_hat, d, eps);
+    rmsnorm_kernel<<<kMaxRows, 256, 0, st>>>(rows, x, g, x_hat, act_layout, d, eps);
 }
 
-void launch_gemm_simt(cudaStream_t st, bool bf16, const RowDesc* rows, const void* W, const void* a, float* out,
+void launch_gemm_simt(cudaStream_t st, bool bf16, const RowDesc* rows, const void* W, const float* a, float* out,
                       int32_t n_out, int32_t k_in, int32_t ld_out, bool accumulate) {
     const int blocks = (n_out + 7) / 8;
     if (bf16)
         gemm_simt_kernel<__nv_bfloat16, 8><<<blocks, 256, 0, st>>>(rows, (const __nv_bfloat16*)W,
-                                                                    (const __nv_bfloat16*)a, out, n_out, k_in, ld_out,
-                                                                    accumulate ? 1 : 0);
+                                                                    a, out, n_out, k_in, ld_out, accumulate ? 1 : 0);
     else
-        gemm_simt_kernel<float, 8><<<blocks, 256, 0, st>>>(rows, (const float*)W, (const float*)a, out, n_out, k_in,
+        gemm_simt_kernel<float, 8><<<blocks, 256, 0, st>>>(rows, (const float*)W, a, out, n_out, k_in,
                                                            ld_out, accumulate ? 1 : 0);
 }
 
-void launch_silu_mul(cudaStream_t st, bool bf16, const RowDesc* rows, const float* gate_up, void* h, int32_t d_ffn) {
+void launch_silu_mul(cudaStream_t st, const RowDesc* rows, const float* gate_up, float* h, int32_t d_ffn) {
     dim3 grid((d_ffn + 255) / 256, kMaxRows);
-    if (bf16) silu_mul_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(rows, gate_up, (__nv_bfloat16*)h, d_ffn);
-    else silu_mul_kernel<float><<<grid, 256, 0, st>>>(rows, gate_up, (float*)h, d_ffn);
+    silu_mul_kernel<<<grid, 256, 0, st>>>(rows, gate_up, h, d_ffn);
 }
 
 void launch_argmax(cudaStream_t st, const RowDesc* rows, const float* logits, int32_t vocab, int32_t* out_tok) {

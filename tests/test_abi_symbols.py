@@ -12,7 +12,7 @@ def test_library_exports_header_symbols():
     from paper_2304_04487_b200 import LIB_PATH, lib
     from paper_2304_04487_b200.binding import EXPORTS
     header = open(os.path.join(ROOT, "include", "llma.h")).read()
-    declared = set(re.findall(r"\b(llma_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(llma_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
     L = ctypes.CDLL(LIB_PATH)
     for name in declared:
