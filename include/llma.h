@@ -230,6 +230,33 @@ int llma_profile_steps(llma_engine *e, int32_t n, int32_t k, int32_t steps, llma
 int llma_gemm_rows32_bf16(const void *W, const void *a, float *out, int32_t n_out, int32_t k_in,
                           void *cuda_stream);
 
+/*
+ * The same product as llma_gemm_rows32_bf16 for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is forbidden or unsafe -- inside a host
+ * process whose memory pool owns the whole GPU and treats any outside allocation as a
+ * budget violation, in a latency-critical serving loop where an allocation would serialise
+ * the device, or in a plug-in that is only handed pre-allocated buffers.  This call performs
+ * no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ * Arguments, layouts and results are exactly those of llma_gemm_rows32_bf16 (W, a, out are
+ * caller-owned device buffers).  The split-k partial tiles, arrival counters and the operand
+ * staging live in a fixed array of about 7 MiB that is part of the library image: every GPU
+ * that loads the library holds it until the process exits.  Limits that follow from its size:
+ * n_out <= 262144 and k_in <= 16384; larger sizes return LLMA_ERR_CAPACITY and do nothing.
+ *
+ * The first call on a device resolves the array's device address (with the caller's current
+ * device) and opts the kernel into its shared-memory size; make that first call before any
+ * stream capture is begun.  All calls on a device share the array and it keeps the previous
+ * call's contents: the call clears what has to start at zero itself, but two calls that
+ * overlap on the GPU (different streams, or different threads) race on it and give wrong
+ * results -- serialise them.  Synchronous.
+ * Errors: NULL, ARG, CAPACITY, CONFIG (not an sm_100 device), CUDA, DEVICE_TIMEOUT.
+ */
+int llma_gemm_rows32_bf16_noalloc(const void *W, const void *a, float *out, int32_t n_out, int32_t k_in,
+                                  void *cuda_stream);
+
 /* Which GEMM implementation the engine resolved to (LLMA_GEMM_SIMT or LLMA_GEMM_TCGEN05), or a
  * negative status. */
 int llma_gemm_impl(llma_engine *e);

@@ -12,5 +12,6 @@ from .binding import (  # noqa: F401
     LlmaStepInfo,
     lib,
     llma_gemm_rows32_bf16,
+    llma_gemm_rows32_bf16_noalloc,
     LIB_PATH,
 )

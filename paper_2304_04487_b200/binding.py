@@ -56,7 +56,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_gemm_rows32_bf16_noalloc", "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
         L.llma_gemm_rows32_bf16.argtypes = [vp, vp, vp, i32, i32, vp]
+        L.llma_gemm_rows32_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, vp]
         L.llma_profile_steps.argtypes = [vp, i32, i32, i32, C.POINTER(LlmaProfile)]
         L.llma_last_cuda_error.argtypes = []
         L.llma_strerror.argtypes = [C.c_int]
@@ -112,6 +113,21 @@ def llma_gemm_rows32_bf16(W, a, out, stream=None) -> None:
     rc = lib().llma_gemm_rows32_bf16(W.data_ptr(), a.data_ptr(), out.data_ptr(), n_out, k_in, st.cuda_stream)
     if rc != 0:
         raise LlmaError(rc, "llma_gemm_rows32_bf16")
+
+
+def llma_gemm_rows32_bf16_noalloc(W, a, out, stream=None) -> None:
+    """Same product as ``llma_gemm_rows32_bf16`` through the entry point that allocates nothing
+    (its scratch is a fixed array inside the library).  For callers that may not call
+    cudaMalloc; calls on one device must not overlap."""
+    import torch
+    assert W.dtype == torch.bfloat16 and a.dtype == torch.bfloat16 and out.dtype == torch.float32
+    assert W.is_contiguous() and a.is_contiguous() and out.is_contiguous() and a.shape[0] == 32
+    n_out, k_in = W.shape
+    assert a.shape[1] == k_in and tuple(out.shape) == (32, n_out)
+    st = stream if stream is not None else torch.cuda.current_stream(W.device)
+    rc = lib().llma_gemm_rows32_bf16_noalloc(W.data_ptr(), a.data_ptr(), out.data_ptr(), n_out, k_in, st.cuda_stream)
+    if rc != 0:
+        raise LlmaError(rc, "llma_gemm_rows32_bf16_noalloc")
 
 
 class Engine:
