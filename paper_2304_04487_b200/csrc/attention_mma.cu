@@ -1,0 +1,298 @@
+// Split-KV causal attention for the k+1 query rows of a step (bf16 K/V cache).
+//
+// Grid (chunk, head, sequence).  A CTA owns 128 consecutive cache positions of one head:
+// its K and V tiles arrive by TMA (128-byte swizzle) and are read ONCE for all the rows of
+// the step, which is what makes verification of k+1 positions cost the K/V traffic of one.
+// Each of the 4 warps takes 32 of the positions: S = Q K^T and O = P V on the tensor cores
+// (mma.sync m16n8k16, bf16 in, fp32 accumulate), softmax statistics by warp shuffles.
+// Q and P enter the MMAs as hi + lo bf16 pairs, so they keep 16 mantissa bits.
+// The warps' partial (max, sum, O) are merged in warp order, the chunk's partial goes to an
+// fp32 workspace, and the last CTA of a (sequence, head) to finish merges the chunks in
+// ascending order.  For a query at absolute position p every one of these decompositions
+// is a function of p alone (chunks and warp spans are fixed position ranges, later positions
+// are masked to exact zeros), so a row's result does not depend on the other rows.
+#include <cuda.h>
+
+#include "attention_mma.cuh"
+#include "ptx_sm100.cuh"
+
+namespace llma {
+
+using namespace ptx;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// (hi, lo) bf16 pairs of two floats, packed for an MMA operand register (x in the low half)
+__device__ __forceinline__ void split_pack(float x, float y, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+    const __nv_bfloat16 xl = __float2bfloat16_rn(x - __bfloat162float(xh));
+    const __nv_bfloat16 yl = __float2bfloat16_rn(y - __bfloat162float(yh));
+    hi = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+    lo = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+}
+
+template <int HD>
+struct AttnSmem {
+    static constexpr int kBoxes = HD / 64;                    // 64-column TMA boxes per K (or V) tile
+    static constexpr uint32_t kBoxBytes = kAttnChunk * 128;   // 128 rows x 128 bytes
+    static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;
+    static constexpr uint32_t kQStride = HD * 2 + 16;         // bytes per Q row (padded: conflict-free ldmatrix)
+    static constexpr uint32_t offK = 0, offV = kTileBytes;
+    static constexpr uint32_t offQhi = 2 * kTileBytes, offQlo = offQhi + kMaxRows * kQStride;
+    static constexpr uint32_t offO = offQlo + kMaxRows * kQStride;      // fp32 [16][HD] merged tile
+    static constexpr uint32_t offStat = offO + 16 * HD * 4;              // m_w[4][16], l_w[4][16], misc
+    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+                                                            const __grid_constant__ CUtensorMap map_v) {
+    using L = AttnSmem<HD>;
+    const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const ModelDims& d = a.dims;
+
+    // rows of this sequence in the step: contiguous, found by a scan of the 32 descriptors
+    int first = -1, cnt = 0, maxpos = -1;
+    for (int r = 0; r < a.rows->rows_used; ++r) {
+        const int p = a.rows->pos[r];
+        if (p >= 0 && a.rows->seq[r] == seq) { if (first < 0) first = r; cnt = r - first + 1; maxpos = max(maxpos, p); }
+    }
+    const int c0 = chunk * kAttnChunk;
+    if (cnt == 0 || c0 > maxpos) return;  // uniform over the CTA
+    const int n_active = maxpos / kAttnChunk + 1;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+    float* sO = reinterpret_cast<float*>(gbase + L::offO);
+    float* s_m = reinterpret_cast<float*>(gbase + L::offStat);   // [4][16]
+    float* s_l = s_m + 64;                                        // [4][16]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(s_l + 64);
+    volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 1);
+    const uint32_t bar_u = smem_u32(bar);
+
+    if (threadIdx.x == 0) { mbar_init(bar_u, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0);
+        mbar_arrive_expect_tx(bar_u, 2 * L::kTileBytes);
+        for (int b = 0; b < L::kBoxes; ++b) {
+            tma_load_2d(base + L::offK + b * L::kBoxBytes, &map_k, bar_u, b * 64, row0);
+            tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_u, b * 64, row0);
+        }
+    }
+    // stage Q (this head, this sequence's rows) as hi / lo bf16; rows past cnt are zero
+    {
+        const int HDT = d.hd_total;
+        for (int idx = threadIdx.x; idx < kMaxRows * HD; idx += blockDim.x) {
+            const int r = idx / HD, i = idx - r * HD;
+            const float v = r < cnt ? a.qkv[(int64_t)(first + r) * 3 * HDT + head * HD + i] : 0.f;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+            *reinterpret_cast<__nv_bfloat16*>(gbase + L::offQhi + r * L::kQStride + i * 2) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(gbase + L::offQlo + r * L::kQStride + i * 2) = lo;
+        }
+    }
+    if (threadIdx.x == 0) {
+        const bool ok = mbar_wait(bar_u, 0);
+        if (!ok) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
+    }
+    __syncthreads();
+    if (flag[0]) return;  // the copy never landed: give up (error word is set)
+
+    const float scale = rsqrtf((float)HD);
+    const int n_mt = (cnt + 15) >> 4;
+    const int wpos0 = warp * 32;  // this warp's positions inside the chunk
+    const int64_t part_base = (((int64_t)seq * d.n_heads + head) * a.n_chunks + chunk) * kMaxRows;
+
+    for (int mt = 0; mt < n_mt; ++mt) {
+        // ---------------- S = Q K^T over this warp's 32 positions ----------------------------
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
+        const int mi = lane >> 3, t8 = lane & 7;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+            uint32_t ah[4], al[4];
+            const uint32_t qoff = (uint32_t)(mt * 16 + (mi & 1) * 8 + t8) * L::kQStride + (uint32_t)(ks * 16 + (mi >> 1) * 8) * 2;
+            ldsm_x4(base + L::offQhi + qoff, ah);
+            ldsm_x4(base + L::offQlo + qoff, al);
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+                const int row = wpos0 + np * 16 + (mi >> 1) * 8 + t8;
+                const int col = ks * 16 + (mi & 1) * 8;
+                const uint32_t kaddr = base + L::offK + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                       ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                uint32_t b[4];
+                ldsm_x4(kaddr, b);
+                mma_bf16(s[2 * np], ah, b[0], b[1]);
+                mma_bf16(s[2 * np], al, b[0], b[1]);
+                mma_bf16(s[2 * np + 1], ah, b[2], b[3]);
+                mma_bf16(s[2 * np + 1], al, b[2], b[3]);
+            }
+        }
+        // ---------------- causal mask, softmax statistics of the warp's span --------------------
+        const int r_lo = mt * 16 + (lane >> 2), r_hi = r_lo + 8;
+        const int lim_lo = r_lo < cnt ? a.rows->pos[first + r_lo] : -1;
+        const int lim_hi = r_hi < cnt ? a.rows->pos[first + r_hi] : -1;
+        float m_lo = -INFINITY, m_hi = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int p = c0 + wpos0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                const int lim = e < 2 ? lim_lo : lim_hi;
+                const float v = p <= lim ? s[nt][e] * scale : -INFINITY;
+                s[nt][e] = v;
+                if (e < 2) m_lo = fmaxf(m_lo, v); else m_hi = fmaxf(m_hi, v);
+            }
+        }
+        m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 1)); m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 2));
+        m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 1)); m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 2));
+        const float ref_lo = m_lo == -INFINITY ? 0.f : m_lo, ref_hi = m_hi == -INFINITY ? 0.f : m_hi;
+        float l_lo = 0.f, l_hi = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float pe = expf(s[nt][e] - (e < 2 ? ref_lo : ref_hi));  // exp(-inf) = 0 for masked positions
+                s[nt][e] = pe;
+                if (e < 2) l_lo += pe; else l_hi += pe;
+            }
+        }
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+        // ---------------- O = P V ----------------------------------------------------------------
+        float o[HD / 8][4];
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+#pragma unroll
+        for (int kp = 0; kp < 2; ++kp) {
+            uint32_t ph[4], pl[4];
+            split_pack(s[2 * kp][0], s[2 * kp][1], ph[0], pl[0]);
+            split_pack(s[2 * kp][2], s[2 * kp][3], ph[1], pl[1]);
+            split_pack(s[2 * kp + 1][0], s[2 * kp + 1][1], ph[2], pl[2]);
+            split_pack(s[2 * kp + 1][2], s[2 * kp + 1][3], ph[3], pl[3]);
+#pragma unroll
+            for (int nn = 0; nn < HD / 16; ++nn) {
+                const int row = wpos0 + kp * 16 + (mi & 1) * 8 + t8;
+                const int col = nn * 16 + (mi >> 1) * 8;
+                const uint32_t vaddr = base + L::offV + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                       ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                uint32_t b[4];
+                ldsm_x4_trans(vaddr, b);
+                mma_bf16(o[2 * nn], ph, b[0], b[1]);
+                mma_bf16(o[2 * nn], pl, b[0], b[1]);
+                mma_bf16(o[2 * nn + 1], ph, b[2], b[3]);
+                mma_bf16(o[2 * nn + 1], pl, b[2], b[3]);
+            }
+        }
+        // ---------------- merge the 4 warps in warp order ------------------------------------------
+        if ((lane & 3) == 0) {
+            s_m[warp * 16 + (lane >> 2)] = m_lo; s_m[warp * 16 + (lane >> 2) + 8] = m_hi;
+            s_l[warp * 16 + (lane >> 2)] = l_lo; s_l[warp * 16 + (lane >> 2) + 8] = l_hi;
+        }
+        __syncthreads();
+        float M_lo = -INFINITY, M_hi = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) { M_lo = fmaxf(M_lo, s_m[w * 16 + (lane >> 2)]); M_hi = fmaxf(M_hi, s_m[w * 16 + (lane >> 2) + 8]); }
+        const float f_lo = m_lo == -INFINITY ? 0.f : expf(m_lo - M_lo);
+        const float f_hi = m_hi == -INFINITY ? 0.f : expf(m_hi - M_hi);
+        for (int w = 0; w < 4; ++w) {
+            if (warp == w) {
+#pragma unroll
+                for (int nt = 0; nt < HD / 8; ++nt) {
+                    float* p_lo = sO + (lane >> 2) * HD + nt * 8 + 2 * (lane & 3);
+                    float* p_hi = p_lo + 8 * HD;
+                    if (w == 0) {
+                        p_lo[0] = f_lo * o[nt][0]; p_lo[1] = f_lo * o[nt][1];
+                        p_hi[0] = f_hi * o[nt][2]; p_hi[1] = f_hi * o[nt][3];
+                    } else {
+                        p_lo[0] += f_lo * o[nt][0]; p_lo[1] += f_lo * o[nt][1];
+                        p_hi[0] += f_hi * o[nt][2]; p_hi[1] += f_hi * o[nt][3];
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        // ---------------- chunk partial -> workspace -----------------------------------------------
+        const int rows_here = min(16, cnt - mt * 16);
+        for (int idx = threadIdx.x; idx < rows_here * HD; idx += blockDim.x) {
+            const int r = idx / HD, i = idx - r * HD;
+            a.ws_o[(part_base + mt * 16 + r) * HD + i] = sO[r * HD + i];
+        }
+        if (threadIdx.x < rows_here) {
+            const int r = threadIdx.x;
+            float M = -INFINITY;
+            for (int w = 0; w < 4; ++w) M = fmaxf(M, s_m[w * 16 + r]);
+            float lsum = 0.f;
+            for (int w = 0; w < 4; ++w) {
+                const float mw = s_m[w * 16 + r];
+                lsum += mw == -INFINITY ? 0.f : expf(mw - M) * s_l[w * 16 + r];
+            }
+            a.ws_ml[(part_base + mt * 16 + r) * 2] = M;
+            a.ws_ml[(part_base + mt * 16 + r) * 2 + 1] = lsum;
+        }
+        __syncthreads();
+    }
+
+    // ---------------- last CTA of this (sequence, head): merge the chunks in ascending order ----------
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int old = atomicAdd(&a.cnt[seq * d.n_heads + head], 1);
+        const bool last = old == n_active - 1;
+        if (last) a.cnt[seq * d.n_heads + head] = 0;
+        flag[1] = last ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!flag[1]) return;
+    __threadfence();
+    const int64_t head_base = ((int64_t)seq * d.n_heads + head) * a.n_chunks * kMaxRows;
+    for (int idx = threadIdx.x; idx < cnt * HD; idx += blockDim.x) {
+        const int r = idx / HD, i = idx - r * HD;
+        const int nc = a.rows->pos[first + r] / kAttnChunk + 1;
+        float M = -INFINITY;
+        for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(&a.ws_ml[(head_base + (int64_t)c * kMaxRows + r) * 2]));
+        float num = 0.f, den = 0.f;
+        for (int c = 0; c < nc; ++c) {
+            const int64_t pr = head_base + (int64_t)c * kMaxRows + r;
+            const float mc = __ldcg(&a.ws_ml[pr * 2]);
+            const float f = mc == -INFINITY ? 0.f : expf(mc - M);
+            den += f * __ldcg(&a.ws_ml[pr * 2 + 1]);
+            num += f * __ldcg(&a.ws_o[pr * HD + i]);
+        }
+        store_act(a.attn_out, kActSplit, first + r, (int64_t)head * HD + i, d.hd_total, num / den);
+    }
+}
+
+cudaError_t init_attention_mma() {
+    cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(AttnSmem<128>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)(AttnSmem<64>::kBytes + 1024));
+}
+
+void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v) {
+    dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
+    if (a.dims.head_dim == 128)
+        attention_mma_kernel<128><<<grid, 128, AttnSmem<128>::kBytes + 1024, st>>>(a, map_k, map_v);
+    else
+        attention_mma_kernel<64><<<grid, 128, AttnSmem<64>::kBytes + 1024, st>>>(a, map_k, map_v);
+}
+
+}  // namespace llma

@@ -1,0 +1,27 @@
+// Tensor-core split-KV attention (library-private interface).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace llma {
+
+constexpr int kAttnChunk = 128;  // cache positions per CTA; chunk c covers [128c, 128c + 128)
+
+struct AttnArgs {
+    ModelDims dims;
+    int32_t layer;
+    int32_t n_chunks;        // grid.x = ceil(max_seq / 128); CTAs past a sequence's last position exit
+    const RowDesc* rows;
+    const float* qkv;        // [32][3*H*hd] fp32, q already rotated
+    void* attn_out;          // ActLayout kActSplit [64][H*hd]
+    float* ws_o;             // chunk partials [seq][head][chunk][32][hd] fp32
+    float* ws_ml;            // [seq][head][chunk][32][2] = (max, sum)
+    int32_t* cnt;            // arrival counters [seq][head], zero between launches
+    int32_t* dev_err;
+};
+
+cudaError_t init_attention_mma();
+void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v);
+
+}  // namespace llma

@@ -50,6 +50,7 @@ static void free_engine(llma_engine* e) {
     cudaFree(e->y); cudaFree(e->out_tok); cudaFree(e->dev_err); cudaFree(e->x); cudaFree(e->qkv);
     cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
     cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
+    cudaFree(e->attn_ws_o); cudaFree(e->attn_ws_ml); cudaFree(e->attn_cnt);
     cudaFree(e->gemm_ws); cudaFree(e->gemm_cnt); cudaFree(e->part_max); cudaFree(e->part_idx);
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
@@ -182,6 +183,18 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         bad |= make_tensor_map_bf16(&e->map_h, e->h, kGemmN, d.d_ffn, kGemmN);
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
         CREATE_TRY(init_gemm_tcgen05());
+        e->attn_chunks = (d.max_seq + kAttnChunk - 1) / kAttnChunk;
+        const size_t parts = (size_t)B * d.n_heads * e->attn_chunks * kMaxRows;
+        CREATE_TRY(dalloc(&e->attn_ws_o, parts * d.head_dim));
+        CREATE_TRY(dalloc(&e->attn_ws_ml, parts * 2));
+        CREATE_TRY(dalloc(&e->attn_cnt, B * d.n_heads));
+        const uint64_t kv_rows = (uint64_t)L * B * d.n_heads * d.max_seq;
+        if (make_tensor_map_bf16(&e->map_kcache, e->kcache, kv_rows, d.head_dim, kAttnChunk) ||
+            make_tensor_map_bf16(&e->map_vcache, e->vcache, kv_rows, d.head_dim, kAttnChunk)) {
+            free_engine(e);
+            return LLMA_ERR_CONFIG;
+        }
+        CREATE_TRY(init_attention_mma());
     }
     CREATE_TRY(cudaMallocHost((void**)&e->h_state, B * sizeof(SeqState)));
     CREATE_TRY(cudaMallocHost((void**)&e->h_rows, sizeof(RowDesc)));

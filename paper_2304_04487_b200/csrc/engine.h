@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "../../include/llma.h"
+#include "attention_mma.cuh"
 #include "gemm_tcgen05.cuh"
 #include "kernels.h"
 
@@ -42,6 +43,12 @@ struct llma_engine {
     int32_t* gemm_cnt = nullptr;    // per-tile arrival counters
     float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
     int32_t* part_idx = nullptr;
+
+    // tensor-core attention: TMA descriptors of the K/V cache, chunk partials, arrival counters
+    CUtensorMap map_kcache, map_vcache;
+    int attn_chunks = 0;
+    float *attn_ws_o = nullptr, *attn_ws_ml = nullptr;
+    int32_t* attn_cnt = nullptr;
 
     // pinned host staging
     llma::SeqState* h_state = nullptr;

@@ -54,7 +54,11 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
         run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
         mark(e, LLMA_K_GEMM_QKV);
-        launch_attention_simt(st, true, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn, kActSplit);
+        AttnArgs at;
+        at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
+        at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml; at.cnt = e->attn_cnt;
+        at.dev_err = e->dev_err;
+        launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D;

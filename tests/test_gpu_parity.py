@@ -50,7 +50,9 @@ def test_tiny_fp32_stepwise_parity():
 
 
 @pytest.mark.parametrize("name,n,k,P,N", [("tiny-bf16", 1, 8, 70, 48), ("small-bf16", 1, 5, 45, 40),
-                                           ("small-bf16", 2, 16, 33, 40), ("mid-bf16", 1, 8, 50, 32)])
+                                           ("small-bf16", 2, 16, 33, 40), ("mid-bf16", 1, 8, 50, 32),
+                                           # contexts spanning several 128-position attention chunks with a ragged tail
+                                           ("tiny-bf16", 1, 8, 300, 24), ("small-bf16", 1, 20, 250, 30)])
 def test_bf16_stepwise_parity(name, n, k, P, N):
     shape = SHAPES[name]
     w = _weights(shape)
