@@ -157,6 +157,8 @@ def main():
     ap.add_argument("--workload", default="llama7b-rag", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-steps", type=int, default=6)
+    ap.add_argument("--profile-only", action="store_true",
+                    help="short run for profilers: prefill, 32 greedy steps, then --steps LLMA decodes of 32 tokens")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -185,7 +187,22 @@ def main():
     t_pre = time.perf_counter()
     eng.llma_prefill(0, prompt)
     t_pre = time.perf_counter() - t_pre
+    if args.profile_only:
+        n_new = 32
     (y_star,), g0 = eng.llma_generate(n_new, 1, 0)
+    if args.profile_only:
+        # launches so far: ceil((P-1)/32) prefill passes of (1 + 7 L) kernels (tensor-core path), then
+        # n_new greedy steps of g0.launches / n_new kernels each
+        eng.llma_set_reference(0, y_star, None)
+        tot = 0
+        for _ in range(args.steps):
+            eng.llma_rewind(0)
+            _, st = eng.llma_generate(n_new, n, k)
+            tot += st.launches
+        print(json.dumps({"profile_only": True, "launches_per_step": g0.launches // n_new,
+                          "greedy_launches": int(g0.launches), "llma_launches": int(tot),
+                          "llma_steps": int(st.steps), "llma_ms_per_step": st.device_ms / st.steps}))
+        return
     ref, offs, ref_info = build_reference(y_star, docs, f, shape.vocab, seed=0)
     ref_host = torch.from_numpy(ref.copy()).pin_memory().numpy()
 

@@ -1,0 +1,51 @@
+"""Micro-benchmark of the projection GEMM on its own (weight streaming at 32 activation rows).
+
+    python -m paper_2304_04487_b200.microbench --n-out 22016 --k-in 4096 --iters 40
+
+Cycles through several weight buffers so that every launch streams its matrix from HBM
+(one matrix may fit in the 126 MB L2), times the launches with CUDA events on the launching
+stream and prints achieved GB/s of weight bytes.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+
+def main():
+    import torch
+    from . import llma_gemm_rows32_bf16_noalloc
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--n-out", type=int, default=22016)
+    ap.add_argument("--k-in", type=int, default=4096)
+    ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--buffers", type=int, default=4)
+    a = ap.parse_args()
+    torch.manual_seed(0)
+    Ws = [(torch.randn(a.n_out, a.k_in, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(a.buffers)]
+    act = torch.randn(32, a.k_in, device="cuda").to(torch.bfloat16)
+    out = torch.empty(32, a.n_out, device="cuda")
+    st = torch.cuda.current_stream()
+    for i in range(3):
+        llma_gemm_rows32_bf16_noalloc(Ws[i % a.buffers], act, out)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(a.iters + 1)]
+    # each call is synchronous (it reads back its error word), so the event pairs bracket
+    # exactly one launch plus its small clears; the clears are a few microseconds
+    times = []
+    for i in range(a.iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        llma_gemm_rows32_bf16_noalloc(Ws[i % a.buffers], act, out)
+        e1.record(st)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    times.sort()
+    med = times[len(times) // 2]
+    nbytes = a.n_out * a.k_in * 2
+    print(json.dumps({"n_out": a.n_out, "k_in": a.k_in, "bytes": nbytes, "median_us": 1e3 * med,
+                      "min_us": 1e3 * times[0], "gbs_median": nbytes / (med / 1e3) / 1e9,
+                      "gbs_best": nbytes / (times[0] / 1e3) / 1e9}))
+
+
+if __name__ == "__main__":
+    main()
