@@ -59,6 +59,8 @@ template <int HD>
 __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
     using L = AttnSmem<HD>;
+    pdl_trigger();
+    pdl_wait();  // row descriptors, q and the K/V rows of this step come from the kernels before
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
@@ -290,9 +292,9 @@ cudaError_t init_attention_mma() {
 void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v) {
     dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
     if (a.dims.head_dim == 128)
-        attention_mma_kernel<128><<<grid, 128, AttnSmem<128>::kBytes + 1024, st>>>(a, map_k, map_v);
+        launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024, attention_mma_kernel<128>, a, map_k, map_v);
     else
-        attention_mma_kernel<64><<<grid, 128, AttnSmem<64>::kBytes + 1024, st>>>(a, map_k, map_v);
+        launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64>, a, map_k, map_v);
 }
 
 }  // namespace llma

@@ -12,6 +12,8 @@ template <typename T>
 __global__ void qkv_post_kernel(ModelDims dims, int layer, const RowDesc* __restrict__ rows, float* __restrict__ qkv,
                                 const float* __restrict__ rope_cos, const float* __restrict__ rope_sin,
                                 T* __restrict__ kcache, T* __restrict__ vcache) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x, head = blockIdx.y;
     const int pos = rows->pos[r];
     if (pos < 0) return;
@@ -41,6 +43,8 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(ModelDims dims, int
                                                              const T* __restrict__ kcache,
                                                              const T* __restrict__ vcache, void* __restrict__ attn_out,
                                                              int act_layout) {
+    pdl_trigger();
+    pdl_wait();
     const int head = blockIdx.x, r = blockIdx.y;
     const int pos = rows->pos[r];
     if (pos < 0) return;
@@ -98,11 +102,9 @@ void launch_qkv_post(cudaStream_t st, bool bf16, const ModelDims& dims, int laye
                      const float* rope_cos, const float* rope_sin, void* kcache, void* vcache) {
     dim3 grid(kMaxRows, dims.n_heads);
     if (bf16)
-        qkv_post_kernel<__nv_bfloat16><<<grid, 64, 0, st>>>(dims, layer, rows, qkv, rope_cos, rope_sin,
-                                                             (__nv_bfloat16*)kcache, (__nv_bfloat16*)vcache);
+        launch_pdl(st, true, grid, dim3(64), 0, qkv_post_kernel<__nv_bfloat16>, dims, layer, rows, qkv, rope_cos, rope_sin, (__nv_bfloat16*)kcache, (__nv_bfloat16*)vcache);
     else
-        qkv_post_kernel<float><<<grid, 64, 0, st>>>(dims, layer, rows, qkv, rope_cos, rope_sin, (float*)kcache,
-                                                     (float*)vcache);
+        launch_pdl(st, true, grid, dim3(64), 0, qkv_post_kernel<float>, dims, layer, rows, qkv, rope_cos, rope_sin, (float*)kcache, (float*)vcache);
 }
 
 void launch_attention_simt(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, const RowDesc* rows,
@@ -111,12 +113,12 @@ void launch_attention_simt(cudaStream_t st, bool bf16, const ModelDims& dims, in
     const bool hd128 = dims.head_dim == 128;
     if (bf16) {
         auto K = (const __nv_bfloat16*)kcache; auto V = (const __nv_bfloat16*)vcache;
-        if (hd128) attention_simt_kernel<__nv_bfloat16, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
-        else attention_simt_kernel<__nv_bfloat16, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        if (hd128) launch_pdl(st, true, grid, dim3(128), 0, attention_simt_kernel<__nv_bfloat16, 4>, dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        else launch_pdl(st, true, grid, dim3(128), 0, attention_simt_kernel<__nv_bfloat16, 2>, dims, layer, rows, qkv, K, V, attn_out, act_layout);
     } else {
         auto K = (const float*)kcache; auto V = (const float*)vcache;
-        if (hd128) attention_simt_kernel<float, 4><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
-        else attention_simt_kernel<float, 2><<<grid, 128, 0, st>>>(dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        if (hd128) launch_pdl(st, true, grid, dim3(128), 0, attention_simt_kernel<float, 4>, dims, layer, rows, qkv, K, V, attn_out, act_layout);
+        else launch_pdl(st, true, grid, dim3(128), 0, attention_simt_kernel<float, 2>, dims, layer, rows, qkv, K, V, attn_out, act_layout);
     }
 }
 

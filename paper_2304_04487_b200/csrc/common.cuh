@@ -73,6 +73,25 @@ __device__ __forceinline__ void store_act(void* buf, int layout, int r, int64_t 
     }
 }
 
+// Every kernel of a decoding step is launched with programmatic stream serialization: it may
+// start while its predecessor is still running, so it must call pdl_wait() before it touches
+// anything an earlier kernel wrote (or anything an earlier kernel may still be reading).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(cudaStream_t st, bool pdl, dim3 grid, dim3 block, size_t smem, void (*kernel)(KArgs...),
+                       Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // K/V cache addressing: [layer][seq][head][max_seq][head_dim]; returns the row index
 __host__ __device__ __forceinline__ int64_t kv_row_index(const ModelDims& d, int layer, int seq, int head, int pos) {
     return ((((int64_t)layer * d.max_batch + seq) * d.n_heads + head) * d.max_seq + pos);

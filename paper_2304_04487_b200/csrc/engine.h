@@ -37,7 +37,11 @@ struct llma_engine {
     // tensor-core GEMM path (bf16): TMA descriptors of weights and activation buffers, work buffers
     struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };
     std::vector<LayerMaps> maps;
-    CUtensorMap map_lm_head, map_x_hat, map_attn, map_h;
+    CUtensorMap map_lm_head;
+    // activation operands: [0] = 16-row boxes (decode when a step holds <= 16 rows), [1] = 64-row boxes
+    CUtensorMap map_x_hat[2], map_attn[2], map_h[2];
+    int decode_nr = 32;             // rows per half used by decoding steps (16 or 32); prefill always uses 32
+    int cur_nr = 32;                // what the launches being enqueued use
     int num_sms = 0;
     float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
     int32_t* gemm_cnt = nullptr;    // per-tile arrival counters

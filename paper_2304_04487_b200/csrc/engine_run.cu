@@ -35,9 +35,10 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
 }
 
 static void run_gemm(llma_engine* e, const GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1,
-                     const CUtensorMap& a2, const CUtensorMap& b) {
+                     const CUtensorMap& a2, const CUtensorMap (&bmaps)[2]) {
+    const CUtensorMap& b = bmaps[e->cur_nr == 16 ? 0 : 1];
     const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
-    launch_gemm_tcgen05(e->stream, grid, a, a0, a1, a2, b);
+    launch_gemm_tcgen05(e->stream, grid, e->cur_nr, true, a, a0, a1, a2, b);
 }
 
 // Tensor-core path (bf16): 7 kernels per layer, every projection fused with what follows it.
@@ -85,7 +86,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
         run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
         mark(e, LLMA_K_GEMM_LMHEAD);
-        launch_argmax_final(st, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
+        launch_argmax_final(st, true, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
         mark(e, LLMA_K_ARGMAX);
         e->launch_counter += 3;
     }
@@ -139,6 +140,7 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
 // plan (trigger search + copy) -> embedding gather -> forward -> accept + K/V commit
 static void enqueue_step(llma_engine* e, int n, int k) {
     const ModelDims& d = e->dims;
+    e->cur_nr = e->decode_nr;
     launch_plan(e->stream, d, e->seq_state, e->rows, e->ref, e->doc_start, e->doc_end, e->y, e->y_cap, n, k,
                 e->dev_err);
     mark(e, LLMA_K_PLAN);
@@ -199,6 +201,7 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
         R->rows_used = cnt;
         R->max_pos = p0 + cnt - 1;
         CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));
+        e->cur_nr = 32;  // prompt chunks fill all 32 rows
         launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
         mark(e, LLMA_K_EMBED);
         enqueue_forward(e, false);

@@ -18,7 +18,7 @@ int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, 
     g.mode = kGemmStore; g.n_out = n_out; g.n_tiles = (n_out + 127) / 128; g.chunks = k_in / 64;
     g.tiles_per_map = g.n_tiles; g.rows = nullptr; g.ws = ws; g.cnt = cnt; g.dev_err = dev_err;
     g.out_f32 = out; g.ld = n_out;
-    launch_gemm_tcgen05(st, grid, g, ma, ma, ma, mb);
+    launch_gemm_tcgen05(st, grid, 32, false, g, ma, ma, ma, mb);
     CU_TRY(cudaGetLastError());
     return LLMA_OK;
 }

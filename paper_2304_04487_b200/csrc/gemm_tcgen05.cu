@@ -5,9 +5,16 @@
 //   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue
 //   warp  4    producer: one thread issues the TMA loads of weight and activation tiles
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
-// Two accumulators (2 x 64 TMEM columns: 32 for the hi half of the activations, 32 for lo) let the epilogue of one tile overlap the MMAs of
-// the next.  Every wait is bounded: when one runs out the kernel raises the device error
-// word, stops issuing work, lets its outstanding copies land, frees TMEM and returns.
+// Two accumulators in TMEM let the epilogue of one tile overlap the MMAs of the next.
+//
+// Programmatic dependent launch: the kernel lets its successor start at once, and itself
+// starts streaming WEIGHT tiles (which no earlier kernel writes) before it waits for its
+// predecessor; only the activation tiles and every global access of the epilogue come after
+// that wait.  So the prologue and pipeline fill of one projection overlap the tail of the
+// kernel before it.
+//
+// Every wait is bounded: when one runs out the kernel raises the device error word, stops
+// issuing work, lets its outstanding copies land, frees TMEM and returns.
 #include <cuda.h>
 
 #include "gemm_epilogue.cuh"
@@ -21,26 +28,29 @@ using namespace ptx;
 // Range of flat (tile, chunk) work items owned by CTA b of G.
 __device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
 
+// NR = activation rows per half (hi / lo): 16 or 32.  MMA N = 2 * NR.
+template <int NR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b) {
-    const int rows_used = g.rows ? g.rows->rows_used : kMaxRows;
-    if (rows_used <= 0) return;  // uniform over the grid: nothing to verify this step
+    using Cfg = GemmCfg<NR>;
+    constexpr int S = Cfg::kStages;
+    constexpr uint32_t kBBytes = Cfg::kBBytes;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t sA = base, sB = base + kGemmStages * kGemmABytes;
-    float (*stage)[33] = reinterpret_cast<float (*)[33]>(gen_base + kGemmStages * (kGemmABytes + kGemmBBytes));
+    const uint32_t sA = base, sB = base + S * kGemmABytes;
+    float (*stage)[33] = reinterpret_cast<float (*)[33]>(gen_base + S * (kGemmABytes + kBBytes));
     uint8_t* tail = reinterpret_cast<uint8_t*>(stage) + 128 * 33 * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full[S], empty[S], acc_full[2], acc_empty[2]
-    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + (2 * kGemmStages + 4) * 8);
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + (2 * S + 4) * 8);
     // sh[0] = TMEM base, sh[1] = abort flag, sh[2] = epilogue broadcast word
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kGemmStages + s); };
-    auto accf_bar = [&](int i) { return bar0 + 8u * (2 * kGemmStages + i); };
-    auto acce_bar = [&](int i) { return bar0 + 8u * (2 * kGemmStages + 2 + i); };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+    auto accf_bar = [&](int i) { return bar0 + 8u * (2 * S + i); };
+    auto acce_bar = [&](int i) { return bar0 + 8u * (2 * S + 2 + i); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, b = blockIdx.x;
@@ -48,14 +58,15 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     const int64_t work = (int64_t)g.n_tiles * C;
     const int64_t w_beg = cta_begin(work, b, G), w_end = cta_begin(work, b + 1, G);
 
+    grid_launch_dependents();  // the next kernel may begin its own prologue now
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kGemmStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(accf_bar(i), 1); mbar_init(acce_bar(i), 4); }
         sh[1] = 0; sh[2] = 0;
         fence_mbar_init();
     }
     if (warp == 5) {
-        tmem_alloc(smem_u32((const void*)&sh[0]), 2 * kGemmN);
+        tmem_alloc(smem_u32((const void*)&sh[0]), 4 * NR);
         tmem_relinquish();
     }
     if (warp == 4 && lane == 0) {
@@ -71,13 +82,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     if (warp == 4) {
         // ------------------------------- producer ---------------------------------------------
         if (lane == 0) {
-            int64_t it = 0;
-            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w, ++it) {
+            auto load_a = [&](int64_t w, int s) {
                 const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
-                const int s = (int)(it % kGemmStages);
-                const uint32_t ph = (uint32_t)((it / kGemmStages) & 1);
-                if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                mbar_arrive_expect_tx(full_bar(s), kGemmABytes + kGemmBBytes);
                 const uint32_t dstA = sA + s * kGemmABytes;
                 if (g.mode == kGemmSwiGLU) {
                     tma_load_2d(dstA, &map_a0, full_bar(s), c * 64, tile * 64);
@@ -87,19 +93,46 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
                     tma_load_2d(dstA, mp, full_bar(s), c * 64, r0);
                 }
-                tma_load_2d(sB + s * kGemmBBytes, &map_b, full_bar(s), c * 64, 0);
+            };
+            auto load_b = [&](int64_t w, int s) {
+                const int c = (int)(w % C);
+                const uint32_t dstB = sB + s * kBBytes;
+                if (NR == kMaxRows) {
+                    tma_load_2d(dstB, &map_b, full_bar(s), c * 64, 0);            // 64 rows: hi then lo
+                } else {
+                    tma_load_2d(dstB, &map_b, full_bar(s), c * 64, 0);            // hi rows 0..NR-1
+                    tma_load_2d(dstB + kBBytes / 2, &map_b, full_bar(s), c * 64, kMaxRows);  // lo rows
+                }
+            };
+            // weights of the first ring-full of items do not depend on any earlier kernel
+            const int64_t n_items = w_end - w_beg;
+            const int n_pre = (int)(n_items < S ? n_items : S);
+            for (int i = 0; i < n_pre; ++i) {
+                mbar_arrive_expect_tx(full_bar(i), kGemmABytes + kBBytes);
+                load_a(w_beg + i, i);
+            }
+            grid_dependency_wait();  // activations are written by the kernel before this one
+            for (int i = 0; i < n_pre; ++i) load_b(w_beg + i, i);
+            int64_t it = n_pre;
+            for (int64_t w = w_beg + n_pre; w < w_end && !sh[1]; ++w, ++it) {
+                const int s = (int)(it % S);
+                const uint32_t ph = (uint32_t)((it / S) & 1);
+                if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                mbar_arrive_expect_tx(full_bar(s), kGemmABytes + kBBytes);
+                load_a(w, s);
+                load_b(w, s);
             }
             if (sh[1]) {
                 // give up: let the copies already issued land before the CTA's memory goes away
-                const int64_t first = it > kGemmStages ? it - kGemmStages : 0;
+                const int64_t first = it > S ? it - S : 0;
                 for (int64_t j = first; j < it; ++j)
-                    (void)mbar_wait(full_bar((int)(j % kGemmStages)), (uint32_t)((j / kGemmStages) & 1), 100000000ull);
+                    (void)mbar_wait(full_bar((int)(j % S)), (uint32_t)((j / S) & 1), 100000000ull);
             }
         }
     } else if (warp == 5) {
         // ------------------------------- MMA issuer ---------------------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_m128(kGemmN);
+            constexpr uint32_t idesc = idesc_bf16_m128(2 * NR);
             int64_t it = 0;
             int seg = 0;
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
@@ -109,14 +142,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const uint32_t use = (uint32_t)(seg >> 1);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kGemmN;
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (2 * NR);
                 for (int c = c0; c < c1; ++c, ++it) {
-                    const int s = (int)(it % kGemmStages);
-                    const uint32_t ph = (uint32_t)((it / kGemmStages) & 1);
+                    const int s = (int)(it % S);
+                    const uint32_t ph = (uint32_t)((it / S) & 1);
                     if (!mbar_wait(full_bar(s), ph)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                     tc_fence_after();
                     const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
-                    const uint64_t db = smem_desc_sw128(sB + s * kGemmBBytes);
+                    const uint64_t db = smem_desc_sw128(sB + s * kBBytes);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
                         umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0) ? 1u : 0u);
@@ -129,6 +162,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
+        grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
+        const int rows_used = g.rows ? g.rows->rows_used : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
@@ -149,12 +184,18 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             tc_fence_after();
             float acc[32];
             {
-                float lo[32];
-                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * kGemmN;
-                tmem_ld_32cols(t0, acc);
-                tmem_ld_32cols(t0 + kMaxRows, lo);
+                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (2 * NR);
+                if (NR == 32) {
+                    float lo[32];
+                    tmem_ld_32cols(t0, acc);
+                    tmem_ld_32cols(t0 + 32, lo);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+                    for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+                } else {
+                    tmem_ld_32cols(t0, acc);  // columns 0..15 hi, 16..31 lo
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { acc[j] += acc[16 + j]; acc[16 + j] = 0.f; }
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -172,7 +213,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const int my_slot = (w_beg >= t_lo) ? 0 : 1;  // first segment of my range, or its last
                 float4* dst = reinterpret_cast<float4*>(g.ws + (((int64_t)b * 2 + my_slot) * 128 + row) * 32);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                for (int q = 0; q < NR / 4; ++q) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
                 __threadfence();
                 epi_sync();
                 if (threadIdx.x == 0) {
@@ -192,7 +233,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const int slot = (cta_begin(work, bb, G) >= t_lo) ? 0 : 1;
                     const float4* src = reinterpret_cast<const float4*>(g.ws + (((int64_t)bb * 2 + slot) * 128 + row) * 32);
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
+                    for (int q = 0; q < NR / 4; ++q) {
                         const float4 p = __ldcg(src + q);
                         acc[4 * q] += p.x; acc[4 * q + 1] += p.y; acc[4 * q + 2] += p.z; acc[4 * q + 3] += p.w;
                     }
@@ -211,7 +252,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * kGemmN);
+        tmem_dealloc(tmem_base, 4 * NR);
     }
 }
 
@@ -220,6 +261,8 @@ __global__ void __launch_bounds__(128) argmax_final_kernel(const RowDesc* __rest
                                                            const float* __restrict__ part_max,
                                                            const int32_t* __restrict__ part_idx, int n_tiles,
                                                            int32_t* __restrict__ out_tok) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int r = blockIdx.x;
     if (rows->pos[r] < 0) { if (threadIdx.x == 0) out_tok[r] = -1; return; }
     float bv = -INFINITY; int bi = 0x7fffffff;
@@ -272,17 +315,32 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 }
 
 cudaError_t init_gemm_tcgen05() {
-    return cudaFuncSetAttribute(gemm_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)GemmCfg<16>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(gemm_ws_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)GemmCfg<32>::kSmemBytes);
 }
 
-void launch_gemm_tcgen05(cudaStream_t st, int grid, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
-                         const CUtensorMap& a2, const CUtensorMap& b) {
-    gemm_ws_kernel<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(args, a0, a1, a2, b);
+void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+                         const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = nr == 16 ? GemmCfg<16>::kSmemBytes : GemmCfg<32>::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    if (nr == 16) cudaLaunchKernelEx(&cfg, gemm_ws_kernel<16>, args, a0, a1, a2, b);
+    else cudaLaunchKernelEx(&cfg, gemm_ws_kernel<32>, args, a0, a1, a2, b);
 }
 
-void launch_argmax_final(cudaStream_t st, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
+void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
                          int32_t n_tiles, int32_t* out_tok) {
-    argmax_final_kernel<<<kMaxRows, 128, 0, st>>>(rows, part_max, part_idx, n_tiles, out_tok);
+    launch_pdl(st, pdl, dim3(kMaxRows), dim3(128), 0, argmax_final_kernel, rows, part_max, part_idx, (int)n_tiles, out_tok);
 }
 
 }  // namespace llma

@@ -49,12 +49,17 @@ struct GemmArgs {
     int32_t* part_idx;
 };
 
-constexpr int kGemmStages = 7;
-constexpr int kGemmN = 2 * kMaxRows;  // MMA N: hi rows then lo rows
+constexpr int kGemmN = 2 * kMaxRows;  // rows of a split activation buffer: hi rows then lo rows
 constexpr int kGemmThreads = 192;
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
-constexpr uint32_t kGemmBBytes = kGemmN * 64 * 2;
-constexpr size_t kGemmSmemBytes = 1024 + (size_t)kGemmStages * (kGemmABytes + kGemmBBytes) + 128 * 33 * 4 + 256;
+
+// The kernel exists for NR = 16 or 32 activation rows per half (MMA N = 2 NR).  Fewer rows
+// mean a smaller activation tile per stage, hence more weight bytes in flight per SM.
+template <int NR> struct GemmCfg {
+    static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
+    static constexpr int kStages = NR == 16 ? 10 : 8;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 256;
+};
 
 // grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)
 int gemm_grid_for(int64_t work, int num_sms);
@@ -66,11 +71,13 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-void launch_gemm_tcgen05(cudaStream_t st, int grid, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
-                         const CUtensorMap& a2, const CUtensorMap& b);
+// nr = 16 or 32 (the B descriptor's box must hold nr rows for 16, 64 rows for 32); pdl = launch with
+// programmatic stream serialization (the kernel before it must be one of this library's)
+void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+                         const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b);
 
 // out_tok[r] = index of the largest logit over all tiles (lowest index on ties)
-void launch_argmax_final(cudaStream_t st, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
+void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
                          int32_t n_tiles, int32_t* out_tok);
 
 }  // namespace llma

@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(256) plan_kernel(ModelDims dims, SeqState* __r
                                                    const int32_t* __restrict__ doc_end,
                                                    const int32_t* __restrict__ y, int32_t y_cap, int32_t n,
                                                    int32_t k, int32_t* __restrict__ dev_err) {
+    pdl_trigger();
+    pdl_wait();
     const int s = blockIdx.x;
     SeqState& S = st[s];
     __shared__ unsigned long long best;  // (ext << 32) | (0x7fffffff - pos): max = longest, then earliest
@@ -92,6 +94,8 @@ __global__ void __launch_bounds__(256) plan_kernel(ModelDims dims, SeqState* __r
 
 // rows_used / max_pos after all sequences are planned (one small CTA)
 __global__ void finish_plan_kernel(ModelDims dims, const SeqState* __restrict__ st, RowDesc* __restrict__ rows) {
+    pdl_trigger();
+    pdl_wait();
     if (threadIdx.x == 0) {
         int used = 0, mp = -1;
         for (int s = 0; s < dims.max_batch; ++s) {
@@ -114,6 +118,8 @@ __global__ void finish_plan_kernel(ModelDims dims, const SeqState* __restrict__ 
 template <typename T>
 __global__ void embed_kernel(ModelDims dims, const RowDesc* __restrict__ rows, const T* __restrict__ emb,
                              float* __restrict__ x, int32_t* __restrict__ dev_err) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
     const int d = dims.d_model;
     float* xr = x + (int64_t)r * d;
@@ -133,6 +139,8 @@ __global__ void embed_kernel(ModelDims dims, const RowDesc* __restrict__ rows, c
 // --------------------------------------------------------------------------------------
 __global__ void accept_kernel(ModelDims dims, SeqState* __restrict__ st, const int32_t* __restrict__ ref,
                               const int32_t* __restrict__ out_tok, int32_t* __restrict__ y, int32_t y_cap) {
+    pdl_trigger();
+    pdl_wait();
     const int s = blockIdx.x;
     if (threadIdx.x != 0) return;
     SeqState& S = st[s];
@@ -168,21 +176,21 @@ __global__ void accept_kernel(ModelDims dims, SeqState* __restrict__ st, const i
 void launch_plan(cudaStream_t st, const ModelDims& dims, SeqState* seq, RowDesc* rows, const int32_t* ref,
                  const int32_t* doc_start, const int32_t* doc_end, const int32_t* y, int32_t y_cap, int32_t n,
                  int32_t k, int32_t* dev_err) {
-    plan_kernel<<<dims.max_batch, 256, 0, st>>>(dims, seq, rows, ref, doc_start, doc_end, y, y_cap, n, k, dev_err);
-    finish_plan_kernel<<<1, 32, 0, st>>>(dims, seq, rows);
+    launch_pdl(st, true, dim3(dims.max_batch), dim3(256), 0, plan_kernel, dims, seq, rows, ref, doc_start, doc_end, y, y_cap, n, k, dev_err);
+    launch_pdl(st, true, dim3(1), dim3(32), 0, finish_plan_kernel, dims, seq, rows);
 }
 
 void launch_embed(cudaStream_t st, const ModelDims& dims, bool bf16, const RowDesc* rows, const void* emb, float* x,
                   int32_t* dev_err) {
     if (bf16)
-        embed_kernel<__nv_bfloat16><<<kMaxRows, 256, 0, st>>>(dims, rows, (const __nv_bfloat16*)emb, x, dev_err);
+        launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, embed_kernel<__nv_bfloat16>, dims, rows, (const __nv_bfloat16*)emb, x, dev_err);
     else
-        embed_kernel<float><<<kMaxRows, 256, 0, st>>>(dims, rows, (const float*)emb, x, dev_err);
+        launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, embed_kernel<float>, dims, rows, (const float*)emb, x, dev_err);
 }
 
 void launch_accept(cudaStream_t st, const ModelDims& dims, SeqState* seq, const int32_t* ref, const int32_t* out_tok,
                    int32_t* y, int32_t y_cap) {
-    accept_kernel<<<dims.max_batch, 32, 0, st>>>(dims, seq, ref, out_tok, y, y_cap);
+    launch_pdl(st, true, dim3(dims.max_batch), dim3(32), 0, accept_kernel, dims, seq, ref, out_tok, y, y_cap);
 }
 
 }  // namespace llma

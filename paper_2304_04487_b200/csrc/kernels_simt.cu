@@ -13,6 +13,8 @@ namespace llma {
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ x,
                                                       const float* __restrict__ g, void* __restrict__ out, int layout,
                                                       int d, float eps) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
     const float* xr = x + (int64_t)r * d;
     if (rows->pos[r] < 0) {
@@ -59,6 +61,8 @@ template <typename T, int RB>  // RB rows handled per pass over the weight row
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const RowDesc* __restrict__ rows, const T* __restrict__ W,
                                                         const float* __restrict__ a, float* __restrict__ out, int n_out,
                                                         int k_in, int ld_out, int accumulate) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int V = Vec16<T>::N;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -101,6 +105,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const RowDesc* __restric
 // ---- SiLU gating ----------------------------------------------------------------------------
 __global__ void silu_mul_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ gate_up,
                                 float* __restrict__ h, int d_ffn) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.y;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= d_ffn) return;
@@ -116,6 +122,8 @@ __global__ void silu_mul_kernel(const RowDesc* __restrict__ rows, const float* _
 // ---- per-row argmax, lowest index on ties --------------------------------------------------
 __global__ void __launch_bounds__(256) argmax_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ logits,
                                                      int vocab, int32_t* __restrict__ out_tok) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
     if (rows->pos[r] < 0) { if (threadIdx.x == 0) out_tok[r] = -1; return; }
     const float* lr = logits + (int64_t)r * vocab;
@@ -142,27 +150,25 @@ __global__ void __launch_bounds__(256) argmax_kernel(const RowDesc* __restrict__
 // ---- launchers -------------------------------------------------------------------------------
 void launch_rmsnorm(cudaStream_t st, int act_layout, const RowDesc* rows, const float* x, const float* g, void* x_hat,
                     int32_t d, float eps) {
-    rmsnorm_kernel<<<kMaxRows, 256, 0, st>>>(rows, x, g, x_hat, act_layout, d, eps);
+    launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, rmsnorm_kernel, rows, x, g, x_hat, act_layout, d, eps);
 }
 
 void launch_gemm_simt(cudaStream_t st, bool bf16, const RowDesc* rows, const void* W, const float* a, float* out,
                       int32_t n_out, int32_t k_in, int32_t ld_out, bool accumulate) {
     const int blocks = (n_out + 7) / 8;
     if (bf16)
-        gemm_simt_kernel<__nv_bfloat16, 8><<<blocks, 256, 0, st>>>(rows, (const __nv_bfloat16*)W,
-                                                                    a, out, n_out, k_in, ld_out, accumulate ? 1 : 0);
+        launch_pdl(st, true, dim3(blocks), dim3(256), 0, gemm_simt_kernel<__nv_bfloat16, 8>, rows, (const __nv_bfloat16*)W, a, out, n_out, k_in, ld_out, accumulate ? 1 : 0);
     else
-        gemm_simt_kernel<float, 8><<<blocks, 256, 0, st>>>(rows, (const float*)W, a, out, n_out, k_in,
-                                                           ld_out, accumulate ? 1 : 0);
+        launch_pdl(st, true, dim3(blocks), dim3(256), 0, gemm_simt_kernel<float, 8>, rows, (const float*)W, a, out, n_out, k_in, ld_out, accumulate ? 1 : 0);
 }
 
 void launch_silu_mul(cudaStream_t st, const RowDesc* rows, const float* gate_up, float* h, int32_t d_ffn) {
     dim3 grid((d_ffn + 255) / 256, kMaxRows);
-    silu_mul_kernel<<<grid, 256, 0, st>>>(rows, gate_up, h, d_ffn);
+    launch_pdl(st, true, grid, dim3(256), 0, silu_mul_kernel, rows, gate_up, h, d_ffn);
 }
 
 void launch_argmax(cudaStream_t st, const RowDesc* rows, const float* logits, int32_t vocab, int32_t* out_tok) {
-    argmax_kernel<<<kMaxRows, 256, 0, st>>>(rows, logits, vocab, out_tok);
+    launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, argmax_kernel, rows, logits, vocab, out_tok);
 }
 
 }  // namespace llma
