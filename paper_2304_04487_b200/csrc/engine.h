@@ -45,6 +45,7 @@ struct llma_engine {
     int num_sms = 0;
     float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
     int32_t* gemm_cnt = nullptr;    // per-tile arrival counters
+    float* norm_ss = nullptr;       // per-tile sums of squares of the residual rows [d/128][32]
     float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
     int32_t* part_idx = nullptr;
 

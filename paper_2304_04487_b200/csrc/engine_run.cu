@@ -41,16 +41,23 @@ static void run_gemm(llma_engine* e, const GemmArgs& a, const CUtensorMap& a0, c
     launch_gemm_tcgen05(e->stream, grid, e->cur_nr, true, a, a0, a1, a2, b);
 }
 
-// Tensor-core path (bf16): 7 kernels per layer, every projection fused with what follows it.
+// Tensor-core path (bf16): 5 kernels per layer.  Every projection is fused with what follows
+// it, and the RMSNorms are folded into the projections around them: the producer of the
+// residual stream emits split(x * gain) and per-tile sums of squares, the consumer scales its
+// accumulators by rsqrt(mean square + eps).
+static void with_norm(llma_engine* e, GemmArgs& a) {
+    a.ss_in = e->norm_ss; a.ss_tiles = (e->dims.d_model + 127) / 128;
+    a.norm_dim = e->dims.d_model; a.norm_eps = e->dims.rms_eps;
+}
+
 static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const ModelDims& d = e->dims;
     cudaStream_t st = e->stream;
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
     for (int l = 0; l < d.n_layers; ++l) {
         const llma_engine::LayerMaps& m = e->maps[l];
-        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
-        mark(e, LLMA_K_NORM);
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
+        with_norm(e, q);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
         run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
@@ -62,33 +69,32 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
-        o.out_f32 = e->x; o.ld = D;
+        o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
         run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
         mark(e, LLMA_K_GEMM_O);
-        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
-        mark(e, LLMA_K_NORM);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
+        with_norm(e, gu);
         gu.out_act = e->h;
         run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
         mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
-        dn.out_f32 = e->x; dn.ld = D;
+        dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
+        dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
         run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->map_h);
         mark(e, LLMA_K_GEMM_DOWN);
-        e->launch_counter += 7;
+        e->launch_counter += 5;
     }
     if (lm_head) {
         const int vt = (d.vocab + 127) / 128;
-        launch_rmsnorm(st, kActSplit, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
-        mark(e, LLMA_K_NORM);
         GemmArgs lm = gemm_args(e, kGemmLmHead, d.vocab, vt, D, vt);
+        with_norm(e, lm);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
         run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
         mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax_final(st, true, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
         mark(e, LLMA_K_ARGMAX);
-        e->launch_counter += 3;
+        e->launch_counter += 2;
     }
 }
 
@@ -137,6 +143,13 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
     }
 }
 
+static void enqueue_embed(llma_engine* e) {
+    if (e->gemm_impl == LLMA_GEMM_TCGEN05)
+        launch_embed_norm(e->stream, e->dims, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat, e->norm_ss, e->dev_err);
+    else
+        launch_embed(e->stream, e->dims, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+}
+
 // plan (trigger search + copy) -> embedding gather -> forward -> accept + K/V commit
 static void enqueue_step(llma_engine* e, int n, int k) {
     const ModelDims& d = e->dims;
@@ -144,7 +157,7 @@ static void enqueue_step(llma_engine* e, int n, int k) {
     launch_plan(e->stream, d, e->seq_state, e->rows, e->ref, e->doc_start, e->doc_end, e->y, e->y_cap, n, k,
                 e->dev_err);
     mark(e, LLMA_K_PLAN);
-    launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+    enqueue_embed(e);
     mark(e, LLMA_K_EMBED);
     e->launch_counter += 3;
     enqueue_forward(e, true);
@@ -202,8 +215,7 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
         R->max_pos = p0 + cnt - 1;
         CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));
         e->cur_nr = 32;  // prompt chunks fill all 32 rows
-        launch_embed(e->stream, d, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
-        mark(e, LLMA_K_EMBED);
+        enqueue_embed(e);
         enqueue_forward(e, false);
         CU_TRY(cudaGetLastError());
         CU_TRY(cudaStreamSynchronize(e->stream));  // h_rows is reused by the next chunk

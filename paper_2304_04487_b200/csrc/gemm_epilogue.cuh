@@ -11,14 +11,37 @@ constexpr uint32_t kEpiBar = 1;  // named barrier of the 128 epilogue threads
 
 __device__ __forceinline__ void epi_sync() { ptx::named_bar_sync(kEpiBar, 128); }
 
-// x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32)
+// x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
+// When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
+// per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
 __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                               int rows_used) {
+                                               int rows_used, float (*stage)[33]) {
     const int col = tile * 128 + row;
-    if (col >= g.n_out) return;
+    const bool valid = col < g.n_out;
+    float xn[32];
 #pragma unroll
-    for (int j = 0; j < 32; ++j)
-        if (j < rows_used) g.out_f32[(int64_t)j * g.ld + col] += acc[j];
+    for (int j = 0; j < 32; ++j) {
+        xn[j] = 0.f;
+        if (j < rows_used && valid) {
+            xn[j] = g.out_f32[(int64_t)j * g.ld + col] + acc[j];
+            g.out_f32[(int64_t)j * g.ld + col] = xn[j];
+        }
+    }
+    if (!g.xs_out) return;
+    const float gain = valid ? g.gain_next[col] : 0.f;
+    const int warp = row >> 5, lane = row & 31;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (j < rows_used) {
+            if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn[j] * gain);
+            float sq = xn[j] * xn[j];
+            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            if (lane == 0) stage[warp][j] = sq;
+        }
+    }
+    epi_sync();
+    if (row < rows_used) g.ss_out[(int64_t)tile * 32 + row] = ((stage[0][row] + stage[1][row]) + stage[2][row]) + stage[3][row];
+    epi_sync();
 }
 
 // out[r, n] = acc

@@ -45,6 +45,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     uint8_t* tail = reinterpret_cast<uint8_t*>(stage) + 128 * 33 * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full[S], empty[S], acc_full[2], acc_empty[2]
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + (2 * S + 4) * 8);
+    float* rscale = reinterpret_cast<float*>(tail + (2 * S + 4) * 8 + 16);  // [32] per-row norm scales
     // sh[0] = TMEM base, sh[1] = abort flag, sh[2] = epilogue broadcast word
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -165,6 +166,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
         const int rows_used = g.rows ? g.rows->rows_used : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
+        if (g.ss_in) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
+            if (row < 32) {
+                float ssum = 0.f;
+                for (int t = 0; t < g.ss_tiles; ++t) ssum += g.ss_in[(int64_t)t * 32 + row];
+                rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
+            }
+            epi_sync();
+        }
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
             const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
@@ -239,9 +248,13 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     }
                 }
             }
+            if (g.ss_in) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] *= rscale[j];
+            }
             switch (g.mode) {
                 case kGemmQKV: epilogue_qkv(g, tile, row, acc, rows_used, stage); break;
-                case kGemmResid: epilogue_resid(g, tile, row, acc, rows_used); break;
+                case kGemmResid: epilogue_resid(g, tile, row, acc, rows_used, stage); break;
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, acc, rows_used, stage); break;
                 case kGemmStore: epilogue_store(g, tile, row, acc, rows_used); break;
                 default: epilogue_lmhead(g, tile, row, acc, rows_used, stage); break;

@@ -39,6 +39,17 @@ struct GemmArgs {
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
     int32_t ld;             // leading dimension of out_f32
     void* out_act;          // SwiGLU: h in ActLayout kActSplit [64][d_ffn]
+    // RMSNorm folded into the projections: the producer of the residual stream x writes
+    // xs = split(x * gain) and, per 128-column tile, the rows' sums of squares; the consumer
+    // multiplies its accumulators by rsqrt(sum / norm_dim + eps), which equals projecting the
+    // normalised row because the scale is one number per row.
+    const float* ss_in;     // consumer: [ss_tiles][32] partial sums of squares, or nullptr
+    int32_t ss_tiles;
+    int32_t norm_dim;
+    float norm_eps;
+    const float* gain_next; // Resid producer: gain of the next norm [n_out], with xs_out / ss_out
+    void* xs_out;           // ActLayout kActSplit [64][n_out], or nullptr
+    float* ss_out;          // [n_tiles][32]
     // QKV
     ModelDims dims;
     int32_t layer;
@@ -58,7 +69,7 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 template <int NR> struct GemmCfg {
     static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
     static constexpr int kStages = NR == 16 ? 10 : 8;
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 256;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 512;
 };
 
 // grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)
