@@ -263,21 +263,61 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     __syncthreads();
     if (!flag[1]) return;
     __threadfence();
+    // The K/V tiles are no longer needed: reuse their shared memory for the chunk statistics.
     const int64_t head_base = ((int64_t)seq * d.n_heads + head) * a.n_chunks * kMaxRows;
-    for (int idx = threadIdx.x; idx < cnt * HD; idx += blockDim.x) {
-        const int r = idx / HD, i = idx - r * HD;
+    float* c_m = reinterpret_cast<float*>(gbase + L::offK);   // [n_active][32] chunk maxima, then weights
+    float* c_l = c_m + (size_t)a.n_chunks * kMaxRows;         // [n_active][32] chunk sums
+    float* r_den = reinterpret_cast<float*>(gbase + L::offO);  // [32]
+    for (int idx = threadIdx.x; idx < n_active * cnt; idx += blockDim.x) {
+        const int c = idx / cnt, r = idx - c * cnt;
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * kMaxRows + r);
+        c_m[c * kMaxRows + r] = ml.x;
+        c_l[c * kMaxRows + r] = ml.y;
+    }
+    __syncthreads();
+    if (threadIdx.x < cnt) {  // one thread per row: weights of its chunks, in ascending chunk order
+        const int r = threadIdx.x;
         const int nc = a.rows->pos[first + r] / kAttnChunk + 1;
         float M = -INFINITY;
-        for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(&a.ws_ml[(head_base + (int64_t)c * kMaxRows + r) * 2]));
-        float num = 0.f, den = 0.f;
+        for (int c = 0; c < nc; ++c) M = fmaxf(M, c_m[c * kMaxRows + r]);
+        float den = 0.f;
         for (int c = 0; c < nc; ++c) {
-            const int64_t pr = head_base + (int64_t)c * kMaxRows + r;
-            const float mc = __ldcg(&a.ws_ml[pr * 2]);
+            const float mc = c_m[c * kMaxRows + r];
             const float f = mc == -INFINITY ? 0.f : expf(mc - M);
-            den += f * __ldcg(&a.ws_ml[pr * 2 + 1]);
-            num += f * __ldcg(&a.ws_o[pr * HD + i]);
+            den += f * c_l[c * kMaxRows + r];
+            c_m[c * kMaxRows + r] = f;
         }
-        store_act(a.attn_out, kActSplit, first + r, (int64_t)head * HD + i, d.hd_total, num / den);
+        for (int c = nc; c < n_active; ++c) c_m[c * kMaxRows + r] = 0.f;
+        r_den[r] = den;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < cnt * (HD / 4); idx += blockDim.x) {
+        const int r = idx / (HD / 4), i4 = idx - r * (HD / 4);
+        const int nc = a.rows->pos[first + r] / kAttnChunk + 1;
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + i4;
+        int c = 0;
+        for (; c + 4 <= nc; c += 4) {  // four independent loads in flight, summed in ascending order
+            float4 p[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) p[u] = __ldcg(src + (int64_t)(c + u) * kMaxRows * (HD / 4));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float f = c_m[(c + u) * kMaxRows + r];
+                num.x += f * p[u].x; num.y += f * p[u].y; num.z += f * p[u].z; num.w += f * p[u].w;
+            }
+        }
+        for (; c < nc; ++c) {
+            const float4 p = __ldcg(src + (int64_t)c * kMaxRows * (HD / 4));
+            const float f = c_m[c * kMaxRows + r];
+            num.x += f * p.x; num.y += f * p.y; num.z += f * p.z; num.w += f * p.w;
+        }
+        const float den = r_den[r];
+        const int64_t col = (int64_t)head * HD + i4 * 4;
+        store_act(a.attn_out, kActSplit, first + r, col, d.hd_total, num.x / den);
+        store_act(a.attn_out, kActSplit, first + r, col + 1, d.hd_total, num.y / den);
+        store_act(a.attn_out, kActSplit, first + r, col + 2, d.hd_total, num.z / den);
+        store_act(a.attn_out, kActSplit, first + r, col + 3, d.hd_total, num.w / den);
     }
 }
 

@@ -190,6 +190,11 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
         CREATE_TRY(init_gemm_tcgen05());
         e->attn_chunks = (d.max_seq + kAttnChunk - 1) / kAttnChunk;
+        // the chunk merge keeps 2 floats per (chunk, row) in the shared memory of the K/V tiles
+        if ((size_t)e->attn_chunks * kMaxRows * 8 > (size_t)2 * (d.head_dim / 64) * kAttnChunk * 128) {
+            free_engine(e);
+            return LLMA_ERR_CONFIG;
+        }
         const size_t parts = (size_t)B * d.n_heads * e->attn_chunks * kMaxRows;
         CREATE_TRY(dalloc(&e->attn_ws_o, parts * d.head_dim));
         CREATE_TRY(dalloc(&e->attn_ws_ml, parts * 2));

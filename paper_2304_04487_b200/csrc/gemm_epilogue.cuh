@@ -1,6 +1,11 @@
 // Epilogues of the weight-streaming GEMM: what happens to a finished 128 x 32 fp32 tile.
-// Called by the 128 epilogue threads; thread `row` holds acc[0..31] = the 32 activation
-// rows' results for output feature (tile, row).  `stage` is a [128][33] fp32 shared buffer.
+// Called by the 128 epilogue threads after the tile has been staged in shared memory:
+// stage[f][j] is the result for output feature f of the tile (thread `row` staged its own
+// feature) and activation row j.  red_f / red_i are [4][32] scratch for per-warp reductions.
+//
+// The loops over activation rows are deliberately NOT unrolled over all 32 rows: this code
+// runs once per tile, so its cost is dominated by instruction fetch, and compact loops
+// with a few independent loads in flight beat long straight-line code.
 #pragma once
 #include "gemm_tcgen05.cuh"
 #include "ptx_sm100.cuh"
@@ -11,56 +16,59 @@ constexpr uint32_t kEpiBar = 1;  // named barrier of the 128 epilogue threads
 
 __device__ __forceinline__ void epi_sync() { ptx::named_bar_sync(kEpiBar, 128); }
 
+__device__ __forceinline__ float warp_sum(float v) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
 // When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
 // per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
-__device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                               int rows_used, float (*stage)[33]) {
+__device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int rows_used,
+                                               float (*stage)[33], float* red_f) {
     const int col = tile * 128 + row;
     const bool valid = col < g.n_out;
-    float xn[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        xn[j] = 0.f;
-        if (j < rows_used && valid) {
-            xn[j] = g.out_f32[(int64_t)j * g.ld + col] + acc[j];
-            g.out_f32[(int64_t)j * g.ld + col] = xn[j];
-        }
-    }
-    if (!g.xs_out) return;
-    const float gain = valid ? g.gain_next[col] : 0.f;
+    const bool fold = g.xs_out != nullptr;
+    const float gain = (fold && valid) ? __ldg(&g.gain_next[col]) : 0.f;
     const int warp = row >> 5, lane = row & 31;
+    for (int j0 = 0; j0 < rows_used; j0 += 4) {
+        float xv[4];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        if (j < rows_used) {
-            if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn[j] * gain);
-            float sq = xn[j] * xn[j];
-            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-            if (lane == 0) stage[warp][j] = sq;
+        for (int u = 0; u < 4; ++u)
+            xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u;
+            if (j < rows_used) {
+                const float xn = valid ? xv[u] + stage[row][j] : 0.f;
+                if (valid) g.out_f32[(int64_t)j * g.ld + col] = xn;
+                if (fold) {
+                    if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn * gain);
+                    const float sq = warp_sum(xn * xn);
+                    if (lane == 0) red_f[warp * 32 + j] = sq;
+                }
+            }
         }
     }
+    if (!fold) return;
     epi_sync();
-    if (row < rows_used) g.ss_out[(int64_t)tile * 32 + row] = ((stage[0][row] + stage[1][row]) + stage[2][row]) + stage[3][row];
+    if (row < rows_used)
+        g.ss_out[(int64_t)tile * 32 + row] = ((red_f[row] + red_f[32 + row]) + red_f[64 + row]) + red_f[96 + row];
     epi_sync();
 }
 
 // out[r, n] = acc
-__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                               int rows_used) {
+__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int row, int rows_used,
+                                               float (*stage)[33]) {
     const int col = tile * 128 + row;
     if (col >= g.n_out) return;
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-        if (j < rows_used) g.out_f32[(int64_t)j * g.ld + col] = acc[j];
+    for (int j = 0; j < rows_used; ++j) g.out_f32[(int64_t)j * g.ld + col] = stage[row][j];
 }
 
 // QKV: rotary embedding on q and k (pair (i, i + hd/2)), q to the fp32 qkv buffer, k and v
 // rows into the bf16 cache at (sequence, position) of every used row.
-__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                             int rows_used, float (*stage)[33]) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
-    epi_sync();
+__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, int rows_used,
+                                             float (*stage)[33]) {
     const ModelDims& d = g.dims;
     const int mat = tile / g.tiles_per_map;
     const int col = (tile % g.tiles_per_map) * 128 + row;
@@ -68,22 +76,39 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
     const int head = col / hd, idx = col % hd;
     const bool lower = idx < half;
     const int prow = lower ? row + half : row - half;
+    const int fi = idx % half;
     if (col < g.n_out) {
-        for (int j = 0; j < rows_used; ++j) {
-            const int pos = g.rows->pos[j];
-            if (pos < 0) continue;
-            float val = stage[row][j];
-            if (mat < 2) {
-                const float other = stage[prow][j];
-                const float c = g.rope_cos[(int64_t)pos * half + (idx % half)];
-                const float s = g.rope_sin[(int64_t)pos * half + (idx % half)];
-                val = lower ? (val * c - other * s) : (other * s + val * c);
+        for (int j0 = 0; j0 < rows_used; j0 += 2) {
+            int pos[2], sq[2];
+            float c[2], sn[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                pos[u] = j0 + u < rows_used ? __ldcg(&g.rows->pos[j0 + u]) : -1;
+                sq[u] = j0 + u < rows_used ? __ldcg(&g.rows->seq[j0 + u]) : 0;
             }
-            if (mat == 0) {
-                g.out_f32[(int64_t)j * g.ld + col] = val;
-            } else {
-                __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
-                cache[kv_row_index(d, g.layer, g.rows->seq[j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                c[u] = 1.f; sn[u] = 0.f;
+                if (pos[u] >= 0 && mat < 2) {
+                    c[u] = __ldg(&g.rope_cos[(int64_t)pos[u] * half + fi]);
+                    sn[u] = __ldg(&g.rope_sin[(int64_t)pos[u] * half + fi]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int j = j0 + u;
+                if (pos[u] < 0) continue;
+                float val = stage[row][j];
+                if (mat < 2) {
+                    const float other = stage[prow][j];
+                    val = lower ? (val * c[u] - other * sn[u]) : (other * sn[u] + val * c[u]);
+                }
+                if (mat == 0) {
+                    g.out_f32[(int64_t)j * g.ld + col] = val;
+                } else {
+                    __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
+                    cache[kv_row_index(d, g.layer, sq[u], head, pos[u]) * hd + idx] = __float2bfloat16_rn(val);
+                }
             }
         }
     }
@@ -91,11 +116,8 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
 }
 
 // SwiGLU: tile rows 0..63 are gate features, 64..127 the matching up features.
-__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                                int rows_used, float (*stage)[33]) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
-    epi_sync();
+__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, int rows_used,
+                                                float (*stage)[33]) {
     const int fi = row & 63, f = tile * 64 + fi;
     if (f < g.n_out) {
         for (int j = row >> 6; j < rows_used; j += 2) {
@@ -107,36 +129,28 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
 }
 
 // LM head: optional logits store, then the tile's (max, lowest argmax) for every used row.
-__device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, const float (&acc)[32],
-                                                int rows_used, float (*stage)[33]) {
+__device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, int rows_used,
+                                                float (*stage)[33], float* red_f, int* red_i) {
     const int v = tile * 128 + row;
     const bool valid = v < g.n_out;
-    if (g.out_f32 && valid) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (j < rows_used) g.out_f32[(int64_t)j * g.ld + v] = acc[j];
-    }
     const int warp = row >> 5, lane = row & 31;
-    float* red_v = &stage[0][0];                       // [4][32] values
-    int* red_i = reinterpret_cast<int*>(&stage[8][0]);  // [4][32] indices
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        if (j < rows_used) {
-            float bv = valid ? acc[j] : -INFINITY;
-            int bi = valid ? v : 0x7fffffff;
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-            }
-            if (lane == 0) { red_v[warp * 32 + j] = bv; red_i[warp * 32 + j] = bi; }
+    for (int j = 0; j < rows_used; ++j) {
+        const float a = stage[row][j];
+        if (g.out_f32 && valid) g.out_f32[(int64_t)j * g.ld + v] = a;
+        float bv = valid ? a : -INFINITY;
+        int bi = valid ? v : 0x7fffffff;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
+        if (lane == 0) { red_f[warp * 32 + j] = bv; red_i[warp * 32 + j] = bi; }
     }
     epi_sync();
     if (row < rows_used) {
-        float bv = red_v[row]; int bi = red_i[row];
+        float bv = red_f[row]; int bi = red_i[row];
         for (int w = 1; w < 4; ++w) {
-            const float ov = red_v[w * 32 + row]; const int oi = red_i[w * 32 + row];
+            const float ov = red_f[w * 32 + row]; const int oi = red_i[w * 32 + row];
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
         g.part_max[(int64_t)tile * 32 + row] = bv;

@@ -46,6 +46,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full[S], empty[S], acc_full[2], acc_empty[2]
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + (2 * S + 4) * 8);
     float* rscale = reinterpret_cast<float*>(tail + (2 * S + 4) * 8 + 16);  // [32] per-row norm scales
+    float* red_f = rscale + 32;                                             // [4][32] reduction scratch
+    int* red_i = reinterpret_cast<int*>(red_f + 128);                       // [4][32]
     // sh[0] = TMEM base, sh[1] = abort flag, sh[2] = epilogue broadcast word
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -238,26 +240,47 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 __threadfence();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                for (int bb = b_first; bb <= b_last; ++bb) {  // ascending k: a fixed summation order
-                    const int slot = (cta_begin(work, bb, G) >= t_lo) ? 0 : 1;
-                    const float4* src = reinterpret_cast<const float4*>(g.ws + (((int64_t)bb * 2 + slot) * 128 + row) * 32);
+                // ascending k: a fixed summation order; loads of several partials are issued together
+                constexpr int kBatch = NR == 16 ? 4 : 2;
+                for (int bb = b_first; bb <= b_last; bb += kBatch) {
+                    float4 p[kBatch][NR / 4];
 #pragma unroll
-                    for (int q = 0; q < NR / 4; ++q) {
-                        const float4 p = __ldcg(src + q);
-                        acc[4 * q] += p.x; acc[4 * q + 1] += p.y; acc[4 * q + 2] += p.z; acc[4 * q + 3] += p.w;
+                    for (int u = 0; u < kBatch; ++u) {
+                        if (bb + u <= b_last) {
+                            const int slot = (cta_begin(work, bb + u, G) >= t_lo) ? 0 : 1;
+                            const float4* src =
+                                reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + slot) * 128 + row) * 32);
+#pragma unroll
+                            for (int q = 0; q < NR / 4; ++q) p[u][q] = __ldcg(src + q);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u) {
+                        if (bb + u <= b_last) {
+#pragma unroll
+                            for (int q = 0; q < NR / 4; ++q) {
+                                acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
+                                acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
+                            }
+                        }
                     }
                 }
             }
+            // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
             if (g.ss_in) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] *= rscale[j];
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[j];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
             }
+            epi_sync();
             switch (g.mode) {
-                case kGemmQKV: epilogue_qkv(g, tile, row, acc, rows_used, stage); break;
-                case kGemmResid: epilogue_resid(g, tile, row, acc, rows_used, stage); break;
-                case kGemmSwiGLU: epilogue_swiglu(g, tile, row, acc, rows_used, stage); break;
-                case kGemmStore: epilogue_store(g, tile, row, acc, rows_used); break;
-                default: epilogue_lmhead(g, tile, row, acc, rows_used, stage); break;
+                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage); break;
+                case kGemmResid: epilogue_resid(g, tile, row, rows_used, stage, red_f); break;
+                case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
+                case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
+                default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
             }
         }
     }

@@ -69,7 +69,7 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 template <int NR> struct GemmCfg {
     static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
     static constexpr int kStages = NR == 16 ? 10 : 8;
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 512;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536;
 };
 
 // grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)
