@@ -136,7 +136,7 @@ class Engine:
 
     def __init__(self, shape, weights: Dict[str, np.ndarray], max_seq: int, max_ref: int, max_k: int,
                  max_batch: int = 1, eos_id: int = -1, gemm_impl: int = LLMA_GEMM_AUTO, keep_logits: bool = False,
-                 device: str = "cuda:0", stream=None):
+                 device: str = "cuda:0", stream=None, share_weights_with: "Engine" = None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the LLMA engine has no CPU path")
@@ -147,6 +147,9 @@ class Engine:
         torch.cuda.set_device(self.device)
         bf16 = shape.dtype == "bf16"
         self._dev: Dict[str, "torch.Tensor"] = {}
+        if share_weights_with is not None:        # a second engine over the same device copies of the weights
+            self._dev = share_weights_with._dev
+            weights = {}
         for name, arr in weights.items():
             if arr.ndim == 1:
                 t = torch.from_numpy(np.ascontiguousarray(arr, np.float32)).to(self.device)
