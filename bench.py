@@ -41,6 +41,23 @@ METRIC = "tokens_per_s_llma_b1"
 UNIT = "tokens/s"
 
 
+def measured_traffic_ratio():
+    """DRAM traffic / algorithmic bytes of the GEMM kernel from the committed ncu summary, or None
+    when the kernel's sources have changed since those counters were taken."""
+    import hashlib
+    prof = os.path.join(ROOT, "profiles", "gemm_ws_kernel_ncu_full_22016x4096.md")
+    src = [os.path.join(ROOT, "paper_2304_04487_b200", "csrc", f)
+           for f in ("gemm_tcgen05.cu", "gemm_epilogue.cuh", "gemm_tcgen05.cuh", "ptx_sm100.cuh")]
+    try:
+        h = hashlib.sha256(b"".join(open(f, "rb").read() for f in src)).hexdigest()[:16]
+        kv = dict(l.strip().split("=", 1) for l in open(prof) if "=" in l and not l.startswith("|") and " " not in l.strip())
+        if kv.get("kernel_sources_sha256_16") == h:
+            return float(kv["traffic_ratio"])
+    except Exception:
+        pass
+    return None
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -272,7 +289,10 @@ def main():
     achieved = wbytes / (gemm_ms / 1e3) / 1e9
     step_ms = dev_ms / max(steps_taken, 1)
     roofline = {"bound": "hbm", "kernel": "gemm_ws_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                # per launch, scaled from the ncu capture of a 180 MB launch (traffic grows with the matrix size)
+                "traffic": (None if measured_traffic_ratio() is None
+                            else measured_traffic_ratio() * wbytes / max(gemm_launches, 1)),
                 "bytes_per_launch": wbytes / max(gemm_launches, 1), "us_per_launch": 1e3 * gemm_ms / max(gemm_launches, 1),
                 "launches_per_step": gemm_launches,
                 "whole_step": {"bytes": wbytes + kvbytes, "ms": step_ms,
