@@ -188,3 +188,25 @@ def test_two_sequences_ragged():
     assert st.tokens == 2 * N and st.copied_accepted > 0
     infos = eng.llma_last_step_info()
     assert len(infos) == 2
+
+
+def test_llama7b_shape_sampled_parity():
+    """Full-size check in the configuration the benchmark times (7B-shaped bf16 decoder, engine created
+    for k = 8): a short prompt, then LLMA steps whose every logits row is compared with the oracle.  The
+    oracle needs about a second per position at this size, so only a few dozen positions are sampled."""
+    shape = SHAPES["llama7b-shape"]
+    w = _weights(shape)
+    prompt = make_prompt(20, shape.vocab, seed=11)
+    max_seq = 64
+    om = OM.OracleModel(shape, w, max_seq=max_seq)
+    y_star = D.greedy_decode(om, prompt, 10).tokens                     # 29 oracle positions
+    ref = y_star[:8] + [shape.vocab - 1, shape.vocab - 2]                 # one span that is accepted, then junk
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=32, max_k=8, keep_logits=True)
+    assert eng.llma_gemm_impl() == 2
+    om2 = OM.OracleModel(shape, w, max_seq=max_seq)
+    rep = step_parity(eng, om2, prompt, ref, None, 1, 8, 10, "bf16")
+    assert rep.max_logit_err <= 2e-2
+    assert rep.rows_compared >= 12 and rep.trigger_steps >= 1 and rep.copied_accepted >= 4
+    assert rep.tokens[:10] == y_star or rep.near_ties > 0
+    print(f"7B-shape parity: rows {rep.rows_compared}, max |dlogit| {rep.max_logit_err:.2e}, near ties {rep.near_ties}")
+    _cache.clear()                                                        # 13 GB of host weights
