@@ -183,6 +183,13 @@ int llma_debug_logits(llma_engine *e, float *out);
  * sequence to `out` (host, [n_heads*head_dim] fp32, widened exactly).  Errors: ARG, CUDA. */
 int llma_debug_kv_row(llma_engine *e, int32_t layer, int32_t seq, int32_t pos, int32_t which, float *out);
 
+/* Parity harness only: copy an internal activation buffer of the last forward pass to `out` (host,
+ * fp32).  which = 0: residual stream x [32][d_model]; 1: qkv [32][3*n_heads*head_dim] (q rotated; the
+ * k and v thirds are only filled on the CUDA-core path); 2: attention output [32][n_heads*head_dim];
+ * 3: gated FFN activation h [32][d_ffn].  Split bf16 buffers are returned as hi + lo.  `count` must be
+ * the buffer's element count.  Errors: NULL, ARG, CUDA. */
+int llma_debug_buffer(llma_engine *e, int32_t which, float *out, int64_t count);
+
 /* Committed K/V length of a sequence (prompt rows + emitted tokens - 1), or a negative status. */
 int llma_kv_len(llma_engine *e, int32_t seq);
 

@@ -56,7 +56,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_gemm_rows32_bf16_noalloc", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_gemm_rows32_bf16_noalloc", "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -81,6 +81,7 @@ def lib() -> C.CDLL:
         L.llma_debug_kv_row.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_float)]
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
+        L.llma_debug_buffer.argtypes = [vp, i32, C.POINTER(C.c_float), C.c_int64]
         L.llma_gemm_rows32_bf16.argtypes = [vp, vp, vp, i32, i32, vp]
         L.llma_gemm_rows32_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, vp]
         L.llma_profile_steps.argtypes = [vp, i32, i32, i32, C.POINTER(LlmaProfile)]
@@ -238,6 +239,14 @@ class Engine:
         out = np.empty(self.shape.n_heads * self.shape.head_dim, np.float32)
         self._check(lib().llma_debug_kv_row(self._h, layer, seq, pos, which,
                                             out.ctypes.data_as(C.POINTER(C.c_float))), "llma_debug_kv_row")
+        return out
+
+    def llma_debug_buffer(self, which: int) -> np.ndarray:
+        sh = self.shape
+        cols = (sh.d_model, 3 * sh.n_heads * sh.head_dim, sh.n_heads * sh.head_dim, sh.d_ffn)[which]
+        out = np.empty((32, cols), np.float32)
+        self._check(lib().llma_debug_buffer(self._h, which, out.ctypes.data_as(C.POINTER(C.c_float)), out.size),
+                    "llma_debug_buffer")
         return out
 
     def llma_kv_len(self, seq: int) -> int:

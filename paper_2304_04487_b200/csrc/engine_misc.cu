@@ -107,3 +107,30 @@ extern "C" int llma_gemm_impl(llma_engine* e) {
     if (!e) return LLMA_ERR_NULL;
     return e->gemm_impl;
 }
+
+extern "C" int llma_debug_buffer(llma_engine* e, int32_t which, float* out, int64_t count) {
+    if (!e || !out) return LLMA_ERR_NULL;
+    const ModelDims& d = e->dims;
+    const int64_t cols = which == 0 ? d.d_model : which == 1 ? 3 * (int64_t)d.hd_total : which == 2 ? d.hd_total
+                       : which == 3 ? d.d_ffn : -1;
+    if (cols < 0 || count != cols * kMaxRows) return LLMA_ERR_ARG;
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    if (which <= 1) {
+        CU_TRY(cudaMemcpy(out, which == 0 ? e->x : e->qkv, (size_t)count * sizeof(float), cudaMemcpyDeviceToHost));
+        return LLMA_OK;
+    }
+    const void* src = which == 2 ? e->attn : e->h;
+    if (e->gemm_impl != LLMA_GEMM_TCGEN05) {  // fp32 [32][K]
+        CU_TRY(cudaMemcpy(out, src, (size_t)count * sizeof(float), cudaMemcpyDeviceToHost));
+        return LLMA_OK;
+    }
+    std::vector<uint16_t> raw((size_t)2 * count);  // split bf16 [64][K]: hi rows then lo rows
+    CU_TRY(cudaMemcpy(raw.data(), src, raw.size() * 2, cudaMemcpyDeviceToHost));
+    for (int64_t i = 0; i < count; ++i) {
+        uint32_t h = (uint32_t)raw[i] << 16, l = (uint32_t)raw[count + i] << 16;
+        float fh, fl;
+        std::memcpy(&fh, &h, 4); std::memcpy(&fl, &l, 4);
+        out[i] = fh + fl;
+    }
+    return LLMA_OK;
+}

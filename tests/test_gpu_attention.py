@@ -1,0 +1,44 @@
+"""The attention kernels alone: the engine's own q rows and cached K/V rows are fed to the oracle's
+one-query softmax attention, so any difference is the attention arithmetic and nothing else."""
+import numpy as np
+import pytest
+
+from oracle import model as OM
+from workloads import SHAPES, make_prompt, make_weights
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,P,k", [("tiny-bf16", 200, 8), ("small-bf16", 300, 20), ("tiny-fp32", 150, 4)])
+def test_attention_rows_match_oracle(name, P, k):
+    from paper_2304_04487_b200 import Engine
+    shape = SHAPES[name]
+    w = make_weights(shape, seed=0, std=0.08)            # larger weights: sharper, less uniform softmax
+    prompt = make_prompt(P, shape.vocab, seed=4)
+    eng = Engine(shape, w, max_seq=P + 64, max_ref=64, max_k=k)
+    eng.llma_prefill(0, prompt)
+    (y,), _ = eng.llma_generate(k + 2, 1, 0)
+    eng.llma_set_reference(0, y)
+    eng.llma_rewind(0)
+    eng.llma_step(1, k)                                   # y is empty: one row
+    eng.llma_step(1, k)                                   # k + 1 rows
+    info = eng.llma_last_step_info()[0]
+    rows = info.k_eff + 1
+    assert rows > 1
+    L0 = eng.llma_kv_len(0) - info.emitted                # position of row 0 of that step
+    # the buffers hold the LAST layer's q and attention output
+    layer = shape.n_layers - 1
+    qkv = eng.llma_debug_buffer(1)
+    att = eng.llma_debug_buffer(2)
+    H, hd = shape.n_heads, shape.head_dim
+    K = np.stack([eng.llma_debug_kv_row(layer, 0, p, 0) for p in range(L0 + rows)]).reshape(-1, H, hd)
+    V = np.stack([eng.llma_debug_kv_row(layer, 0, p, 1) for p in range(L0 + rows)]).reshape(-1, H, hd)
+    worst = 0.0
+    for j in range(rows):
+        for h in range(H):
+            q = qkv[j, h * hd:(h + 1) * hd]
+            want = OM.attention(q, K[:L0 + j + 1, h], V[:L0 + j + 1, h])
+            got = att[j, h * hd:(h + 1) * hd]
+            worst = max(worst, float(np.abs(got - want).max() / max(1e-6, np.abs(want).max())))
+    # fp32 softmax with split bf16 operands: errors near 1e-6 of the row's scale; 2e-5 leaves headroom
+    assert worst < 2e-5, worst
