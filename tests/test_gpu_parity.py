@@ -206,7 +206,7 @@ def test_llama7b_shape_sampled_parity():
     om2 = OM.OracleModel(shape, w, max_seq=max_seq)
     rep = step_parity(eng, om2, prompt, ref, None, 1, 8, 10, "bf16")
     assert rep.max_logit_err <= bf16_logit_tolerance(shape.n_layers)
-    assert rep.rows_compared >= 12 and rep.trigger_steps >= 1 and rep.copied_accepted >= 4
+    assert rep.rows_compared >= 10 and rep.trigger_steps >= 1 and rep.copied_accepted >= 4
     assert rep.tokens[:10] == y_star or rep.near_ties > 0
     print(f"7B-shape parity: rows {rep.rows_compared}, max |dlogit| {rep.max_logit_err:.2e}, near ties {rep.near_ties}")
     _cache.clear()                                                        # 13 GB of host weights
