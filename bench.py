@@ -58,6 +58,23 @@ def measured_traffic_ratio():
     return None
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (identity without one): multi-GPU numbers are timed per rank and reported as the slowest."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replica_throughput(tokens_per_replica: int, world: int, slowest_seconds: float) -> float:
+    """Whole-job tokens/s of `world` independent replicas (weak scaling: same work per GPU)."""
+    return tokens_per_replica * world / slowest_seconds
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -265,14 +282,10 @@ def main():
     clocks = sampler.stop()
     assert toks == y_star
 
-    if world > 1:
-        t = torch.tensor([dev_ms, wall_s, g_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dev_ms, wall_s, g_ms = t.tolist()
-    total_tokens = args.steps * n_new * world
-    value = total_tokens / (dev_ms / 1e3)
-    e2e_value = total_tokens / wall_s
-    greedy_value = total_tokens / (g_ms / 1e3)
+    dev_ms, wall_s, g_ms = max_over_ranks([dev_ms, wall_s, g_ms], device="cuda")
+    value = replica_throughput(args.steps * n_new, world, dev_ms / 1e3)
+    e2e_value = replica_throughput(args.steps * n_new, world, wall_s)
+    greedy_value = replica_throughput(args.steps * n_new, world, g_ms / 1e3)
 
     # ---- roofline of the dominant kernel: the weight-streaming GEMM -----------------------------
     peak, peak_kind = load_peaks()
