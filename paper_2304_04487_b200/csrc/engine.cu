@@ -51,8 +51,7 @@ static void free_engine(llma_engine* e) {
     cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
     cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
     cudaFree(e->attn_ws_o); cudaFree(e->attn_ws_ml); cudaFree(e->attn_cnt);
-    cudaFree(e->gemm_ws); cudaFree(e->gemm_cnt); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss); cudaFree(e->x_hat2); cudaFree(e->norm_ss2); cudaFree(e->gemm_ws2); cudaFree(e->gemm_cnt2);
-    cudaFree(e->flags);
+    cudaFree(e->gemm_ws); cudaFree(e->gemm_cnt); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss);
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
     if (e->h_err) cudaFreeHost(e->h_err);
@@ -167,12 +166,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         CREATE_TRY(dalloc(&e->part_max, (size_t)vt * 32));
         CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * 32));
         CREATE_TRY(dalloc(&e->norm_ss, (size_t)((d.d_model + 127) / 128) * 32));
-        CREATE_TRY(dalloc(&e->norm_ss2, (size_t)((d.d_model + 127) / 128) * 32));
-        CREATE_TRY(dalloc((char**)&e->x_hat2, (size_t)kMaxRows * d.d_model * 4));
-        CREATE_TRY(dalloc(&e->gemm_ws2, (size_t)e->num_sms * 2 * 128 * 32));
-        CREATE_TRY(dalloc(&e->gemm_cnt2, (size_t)max_tiles));
-        e->flag_stride = std::max((d.d_model + 127) / 128, (d.d_ffn + 63) / 64);
-        CREATE_TRY(dalloc(&e->flags, (size_t)3 * e->flag_stride));
         e->maps.resize(L);
         int bad = 0;
         for (int l = 0; l < L; ++l) {
@@ -189,7 +182,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         for (int v = 0; v < 2; ++v) {
             const uint32_t box = v == 0 ? 16 : kGemmN;
             bad |= make_tensor_map_bf16(&e->map_x_hat[v], e->x_hat, kGemmN, d.d_model, box);
-            bad |= make_tensor_map_bf16(&e->map_x_hat2[v], e->x_hat2, kGemmN, d.d_model, box);
             bad |= make_tensor_map_bf16(&e->map_attn[v], e->attn, kGemmN, HD, box);
             bad |= make_tensor_map_bf16(&e->map_h[v], e->h, kGemmN, d.d_ffn, box);
         }

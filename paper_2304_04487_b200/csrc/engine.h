@@ -45,14 +45,6 @@ struct llma_engine {
     int num_sms = 0;
     float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
     int32_t* gemm_cnt = nullptr;    // per-tile arrival counters
-    // tile-granular hand-over between consecutive projections: two copies of what alternates
-    void* x_hat2 = nullptr;         // split(x * gain) written by the down projection (x_hat: by the output projection)
-    float* norm_ss2 = nullptr;
-    float* gemm_ws2 = nullptr;
-    int32_t* gemm_cnt2 = nullptr;
-    int32_t* flags = nullptr;       // [3][flag_stride]: x_hat tiles, x_hat2 tiles, h tiles
-    int flag_stride = 0;
-    CUtensorMap map_x_hat2[2];
     float* norm_ss = nullptr;       // per-tile sums of squares of the residual rows [d/128][32]
     float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
     int32_t* part_idx = nullptr;

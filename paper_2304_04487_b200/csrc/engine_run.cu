@@ -45,36 +45,22 @@ static void run_gemm(llma_engine* e, const GemmArgs& a, const CUtensorMap& a0, c
 // it, and the RMSNorms are folded into the projections around them: the producer of the
 // residual stream emits split(x * gain) and per-tile sums of squares, the consumer scales its
 // accumulators by rsqrt(mean square + eps).
-// Buffers that alternate between consecutive projections (two kernels can be in flight):
-//   set 0: QKV, gate/up, LM head      set 1: output projection, down projection
-static void use_set(llma_engine* e, GemmArgs& a, int set) {
-    a.ws = set ? e->gemm_ws2 : e->gemm_ws;
-    a.cnt = set ? e->gemm_cnt2 : e->gemm_cnt;
-}
-// consumer of split(x * gain) + sums of squares written by the output projection (which = 0: x_hat)
-// or by the down projection / embedding (which = 1: x_hat2)
-static void with_norm(llma_engine* e, GemmArgs& a, int which) {
-    a.ss_in = which ? e->norm_ss2 : e->norm_ss; a.ss_tiles = (e->dims.d_model + 127) / 128;
+static void with_norm(llma_engine* e, GemmArgs& a) {
+    a.ss_in = e->norm_ss; a.ss_tiles = (e->dims.d_model + 127) / 128;
     a.norm_dim = e->dims.d_model; a.norm_eps = e->dims.rms_eps;
 }
-static int32_t* flag_array(llma_engine* e, int i) { return e->flags + (size_t)i * e->flag_stride; }
 
 static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const ModelDims& d = e->dims;
     cudaStream_t st = e->stream;
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
-    const int d_tiles = (D + 127) / 128;
     for (int l = 0; l < d.n_layers; ++l) {
         const llma_engine::LayerMaps& m = e->maps[l];
-        // QKV: reads x_hat2 (embedding for layer 0: whole-kernel dependency; else the previous down
-        // projection, tile by tile)
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
-        use_set(e, q, 0);
-        with_norm(e, q, 1);
-        if (l > 0) { q.wait_flags = flag_array(e, 1); q.wait_shift = 1; q.wait_tiles = d_tiles; q.tag = l; }
+        with_norm(e, q);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
-        run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat2);
+        run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
         mark(e, LLMA_K_GEMM_QKV);
         AttnArgs at;
         at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
@@ -82,29 +68,18 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         at.dev_err = e->dev_err;
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
-        // output projection: whole-kernel dependency on attention; publishes x_hat tiles
-        GemmArgs o = gemm_args(e, kGemmResid, D, d_tiles, HD, d_tiles);
-        use_set(e, o, 1);
+        GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
-        o.set_flags = flag_array(e, 0); o.tag = l + 1;
         run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
         mark(e, LLMA_K_GEMM_O);
-        // gate/up: consumes x_hat tile by tile, publishes h tiles (64 features = one k-chunk of down)
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
-        use_set(e, gu, 0);
-        with_norm(e, gu, 0);
-        gu.wait_flags = flag_array(e, 0); gu.wait_shift = 1; gu.wait_tiles = d_tiles; gu.tag = l + 1;
-        gu.set_flags = flag_array(e, 2);
+        with_norm(e, gu);
         gu.out_act = e->h;
         run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
         mark(e, LLMA_K_GEMM_GATEUP);
-        // down: consumes h chunk by chunk, publishes x_hat2 tiles for the next layer (or the LM head)
-        GemmArgs dn = gemm_args(e, kGemmResid, D, d_tiles, F, d_tiles);
-        use_set(e, dn, 1);
-        dn.wait_flags = flag_array(e, 2); dn.wait_shift = 0; dn.wait_tiles = 0; dn.tag = l + 1;
-        dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat2; dn.ss_out = e->norm_ss2;
+        GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
+        dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
-        dn.set_flags = flag_array(e, 1);
         run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->map_h);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 5;
@@ -112,12 +87,10 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     if (lm_head) {
         const int vt = (d.vocab + 127) / 128;
         GemmArgs lm = gemm_args(e, kGemmLmHead, d.vocab, vt, D, vt);
-        use_set(e, lm, 0);
-        with_norm(e, lm, 1);
-        lm.wait_flags = flag_array(e, 1); lm.wait_shift = 1; lm.wait_tiles = d_tiles; lm.tag = d.n_layers;
+        with_norm(e, lm);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
-        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat2);
+        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
         mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax_final(st, true, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
         mark(e, LLMA_K_ARGMAX);
@@ -172,8 +145,7 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
 
 static void enqueue_embed(llma_engine* e) {
     if (e->gemm_impl == LLMA_GEMM_TCGEN05)
-        launch_embed_norm(e->stream, e->dims, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat2, e->norm_ss2, e->flags,
-                          3 * e->flag_stride, e->dev_err);
+        launch_embed_norm(e->stream, e->dims, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat, e->norm_ss, e->dev_err);
     else
         launch_embed(e->stream, e->dims, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
 }

@@ -97,17 +97,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     tma_load_2d(dstA, mp, full_bar(s), c * 64, r0);
                 }
             };
-            int ready_flag = -1;  // last flag index known to carry the tag (chunks are visited in order)
             auto load_b = [&](int64_t w, int s) {
                 const int c = (int)(w % C);
-                if (g.wait_flags) {
-                    const int f = c >> g.wait_shift;
-                    if (f != ready_flag) {
-                        if (!flag_wait(g.wait_flags + f, g.tag)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
-                        fence_proxy_async();
-                        ready_flag = f;
-                    }
-                }
                 const uint32_t dstB = sB + s * kBBytes;
                 if (NR == kMaxRows) {
                     tma_load_2d(dstB, &map_b, full_bar(s), c * 64, 0);            // 64 rows: hi then lo
@@ -123,7 +114,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 mbar_arrive_expect_tx(full_bar(i), kGemmABytes + kBBytes);
                 load_a(w_beg + i, i);
             }
-            if (!g.wait_flags) grid_dependency_wait();  // activations are written by the kernel before this one
+            grid_dependency_wait();  // activations are written by the kernel before this one
             for (int i = 0; i < n_pre; ++i) load_b(w_beg + i, i);
             int64_t it = n_pre;
             for (int64_t w = w_beg + n_pre; w < w_end && !sh[1]; ++w, ++it) {
@@ -174,21 +165,13 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
-        if (!g.wait_flags) grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
+        grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
         const int rows_used = g.rows ? g.rows->rows_used : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
         if (g.ss_in) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
-            if (g.wait_flags) {  // every tile of the producer must have published its sums of squares
-                if (threadIdx.x == 0) {
-                    bool ok = true;
-                    for (int t = 0; t < g.wait_tiles && ok; ++t) ok = flag_wait(g.wait_flags + t, g.tag);
-                    if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
-                }
-                epi_sync();
-            }
             if (row < 32) {
                 float ssum = 0.f;
-                for (int t = 0; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * 32 + row]);
+                for (int t = 0; t < g.ss_tiles; ++t) ssum += g.ss_in[(int64_t)t * 32 + row];
                 rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
             }
             epi_sync();
@@ -298,11 +281,6 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
                 case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
                 default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
-            }
-            if (g.set_flags) {  // publish the finished tile to the kernel running behind this one
-                __threadfence();
-                epi_sync();
-                if (threadIdx.x == 0) flag_publish(g.set_flags + tile, g.tag);
             }
         }
     }

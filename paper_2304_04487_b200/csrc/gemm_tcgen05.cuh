@@ -47,15 +47,6 @@ struct GemmArgs {
     int32_t ss_tiles;
     int32_t norm_dim;
     float norm_eps;
-    // Dependency on the kernel before this one.  wait_flags == nullptr: the whole predecessor must
-    // have finished (griddepcontrol.wait).  Otherwise the predecessor is a GEMM that publishes its
-    // output tile by tile: activation k-chunk c may be loaded once wait_flags[c >> wait_shift] == tag,
-    // and the folded-norm scales once all wait_tiles flags carry the tag.
-    const int32_t* wait_flags;
-    int32_t wait_shift;
-    int32_t wait_tiles;
-    int32_t tag;            // layer + 1: also the value this kernel publishes
-    int32_t* set_flags;     // producer: [n_tiles] flag per finished output tile, or nullptr
     const float* gain_next; // Resid producer: gain of the next norm [n_out], with xs_out / ss_out
     void* xs_out;           // ActLayout kActSplit [64][n_out], or nullptr
     float* ss_out;          // [n_tiles][32]

@@ -12,7 +12,7 @@ void launch_embed(cudaStream_t st, const ModelDims& dims, bool bf16, const RowDe
                   int32_t* dev_err);
 // bf16 embedding gather with the first RMSNorm folded in: x, xs = split(x * gain), ss[tile][row]
 void launch_embed_norm(cudaStream_t st, const ModelDims& dims, const RowDesc* rows, const void* emb, const float* gain,
-                       float* x, void* xs, float* ss, int32_t* flags, int n_flags, int32_t* dev_err);
+                       float* x, void* xs, float* ss, int32_t* dev_err);
 void launch_accept(cudaStream_t st, const ModelDims& dims, SeqState* seq, const int32_t* ref, const int32_t* out_tok,
                    int32_t* y, int32_t y_cap);
 

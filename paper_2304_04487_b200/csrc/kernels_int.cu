@@ -138,16 +138,9 @@ __global__ void __launch_bounds__(128) embed_norm_kernel(ModelDims dims, const R
                                                          const __nv_bfloat16* __restrict__ emb,
                                                          const float* __restrict__ gain, float* __restrict__ x,
                                                          void* __restrict__ xs, float* __restrict__ ss,
-                                                         int32_t* __restrict__ flags, int n_flags,
                                                          int32_t* __restrict__ dev_err) {
-    // Order matters: wait for everything before this forward pass, clear the tile hand-over flags of
-    // the projections, and only then let the next kernel exist -- no kernel of this pass can see a
-    // flag value left by an earlier pass.
-    pdl_wait();
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_flags; i += gridDim.x * blockDim.x) flags[i] = 0;
-    __threadfence();
-    __syncthreads();
     pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x, d = dims.d_model;
     const int tok = rows->tok[r];
     const bool used = rows->pos[r] >= 0;
@@ -230,9 +223,9 @@ void launch_embed(cudaStream_t st, const ModelDims& dims, bool bf16, const RowDe
 }
 
 void launch_embed_norm(cudaStream_t st, const ModelDims& dims, const RowDesc* rows, const void* emb, const float* gain,
-                       float* x, void* xs, float* ss, int32_t* flags, int n_flags, int32_t* dev_err) {
+                       float* x, void* xs, float* ss, int32_t* dev_err) {
     launch_pdl(st, true, dim3(kMaxRows), dim3(128), 0, embed_norm_kernel, dims, rows, (const __nv_bfloat16*)emb, gain, x,
-               xs, ss, flags, n_flags, dev_err);
+               xs, ss, dev_err);
 }
 
 void launch_accept(cudaStream_t st, const ModelDims& dims, SeqState* seq, const int32_t* ref, const int32_t* out_tok,

@@ -22,31 +22,6 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// ---- tile-granular hand-over between two kernels that run at the same time --------------------
-// A producer kernel publishes "tile t is written" by storing a tag into a flag word after a
-// fence; a consumer kernel launched behind it (programmatic dependent launch: it only exists once
-// every producer CTA is resident, so the producer never depends on the consumer) polls the
-// flag, bounded in time, before it reads the tile.
-__device__ __forceinline__ void flag_publish(int32_t* flag, int32_t tag) {
-    asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(flag), "r"(tag) : "memory");
-}
-__device__ __forceinline__ int32_t flag_peek(const int32_t* flag) {
-    int32_t v;
-    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    return v;
-}
-__device__ __forceinline__ bool flag_wait(const int32_t* flag, int32_t tag, uint64_t limit_ns = 2000000000ull) {
-    if (flag_peek(flag) == tag) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 32; ++i)
-            if (flag_peek(flag) == tag) return true;
-        if (globaltimer_ns() - t0 > limit_ns) return false;
-    }
-}
-// order this thread's later async-proxy operations (TMA loads) after what it has just acquired
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
 // ---- mbarrier ----------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
