@@ -65,12 +65,9 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
 
-    // rows of this sequence in the step: contiguous, found by a scan of the 32 descriptors
-    int first = -1, cnt = 0, maxpos = -1;
-    for (int r = 0; r < a.rows->rows_used; ++r) {
-        const int p = a.rows->pos[r];
-        if (p >= 0 && a.rows->seq[r] == seq) { if (first < 0) first = r; cnt = r - first + 1; maxpos = max(maxpos, p); }
-    }
+    // rows of this sequence in the step (contiguous; summarised by the planning kernel)
+    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
+    const int maxpos = __ldcg(&a.rows->seq_maxpos[seq]);
     const int c0 = chunk * kAttnChunk;
     if (cnt == 0 || c0 > maxpos) return;  // uniform over the CTA
     const int n_active = maxpos / kAttnChunk + 1;
@@ -98,7 +95,8 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     // stage Q (this head, this sequence's rows) as hi / lo bf16; rows past cnt are zero
     {
         const int HDT = d.hd_total;
-        for (int idx = threadIdx.x; idx < kMaxRows * HD; idx += blockDim.x) {
+        const int rows_staged = ((cnt + 15) >> 4) << 4;  // whole 16-row MMA tiles; rows past cnt are zero
+        for (int idx = threadIdx.x; idx < rows_staged * HD; idx += blockDim.x) {
             const int r = idx / HD, i = idx - r * HD;
             const float v = r < cnt ? a.qkv[(int64_t)(first + r) * 3 * HDT + head * HD + i] : 0.f;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);

@@ -30,6 +30,10 @@ struct RowDesc {
     int32_t pos[kMaxRows];  // absolute position in its sequence, -1 = row unused
     int32_t seq[kMaxRows];  // sequence slot
     int32_t rows_used;      // 1 + highest used row index (0 = nothing to do)
+    // per sequence slot: its rows are contiguous -- first row, row count (0 = none) and highest position
+    int32_t seq_first[kMaxRows];
+    int32_t seq_cnt[kMaxRows];
+    int32_t seq_maxpos[kMaxRows];
     int32_t max_pos;        // highest position among used rows (-1 if none)
 };
 

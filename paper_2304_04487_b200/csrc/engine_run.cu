@@ -211,6 +211,8 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
             R->pos[r] = r < cnt ? p0 + r : -1;
             R->seq[r] = seq;
         }
+        for (int s2 = 0; s2 < kMaxRows; ++s2) { R->seq_first[s2] = 0; R->seq_cnt[s2] = 0; R->seq_maxpos[s2] = -1; }
+        R->seq_first[seq] = 0; R->seq_cnt[seq] = cnt; R->seq_maxpos[seq] = p0 + cnt - 1;
         R->rows_used = cnt;
         R->max_pos = p0 + cnt - 1;
         CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));

@@ -99,6 +99,9 @@ __global__ void finish_plan_kernel(ModelDims dims, const SeqState* __restrict__ 
     if (threadIdx.x == 0) {
         int used = 0, mp = -1;
         for (int s = 0; s < dims.max_batch; ++s) {
+            rows->seq_first[s] = s * dims.kp1;
+            rows->seq_cnt[s] = st[s].nrows;
+            rows->seq_maxpos[s] = st[s].nrows > 0 ? st[s].kv_len + st[s].nrows - 1 : -1;
             if (st[s].nrows > 0) {
                 used = s * dims.kp1 + st[s].nrows;
                 mp = max(mp, st[s].kv_len + st[s].nrows - 1);
