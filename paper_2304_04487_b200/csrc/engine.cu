@@ -179,12 +179,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
             bad |= make_tensor_map_bf16(&m.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
         }
         bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
-        for (int v = 0; v < 2; ++v) {
-            const uint32_t box = v == 0 ? 16 : kGemmN;
-            bad |= make_tensor_map_bf16(&e->map_x_hat[v], e->x_hat, kGemmN, d.d_model, box);
-            bad |= make_tensor_map_bf16(&e->map_attn[v], e->attn, kGemmN, HD, box);
-            bad |= make_tensor_map_bf16(&e->map_h[v], e->h, kGemmN, d.d_ffn, box);
-        }
         // the MMA shape of decoding steps is fixed per engine (by its row capacity), never per step
         e->decode_nr = d.max_batch * d.kp1 <= 16 ? 16 : 32;
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape

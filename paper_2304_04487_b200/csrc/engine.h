@@ -38,8 +38,6 @@ struct llma_engine {
     struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };
     std::vector<LayerMaps> maps;
     CUtensorMap map_lm_head;
-    // activation operands: [0] = 16-row boxes (decode when a step holds <= 16 rows), [1] = 64-row boxes
-    CUtensorMap map_x_hat[2], map_attn[2], map_h[2];
     int decode_nr = 32;             // rows per half used by decoding steps (16 or 32); prefill always uses 32
     int cur_nr = 32;                // what the launches being enqueued use
     int num_sms = 0;

@@ -34,11 +34,11 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
     return a;
 }
 
-static void run_gemm(llma_engine* e, const GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1,
-                     const CUtensorMap& a2, const CUtensorMap (&bmaps)[2]) {
-    const CUtensorMap& b = bmaps[e->cur_nr == 16 ? 0 : 1];
+static void run_gemm(llma_engine* e, GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                     const void* act) {
+    a.act = act;
     const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
-    launch_gemm_tcgen05(e->stream, grid, e->cur_nr, true, a, a0, a1, a2, b);
+    launch_gemm_tcgen05(e->stream, grid, e->cur_nr, true, a, a0, a1, a2);
 }
 
 // Tensor-core path (bf16): 5 kernels per layer.  Every projection is fused with what follows
@@ -60,7 +60,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         with_norm(e, q);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
-        run_gemm(e, q, m.wq, m.wk, m.wv, e->map_x_hat);
+        run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat);
         mark(e, LLMA_K_GEMM_QKV);
         AttnArgs at;
         at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
@@ -70,17 +70,17 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
-        run_gemm(e, o, m.wo, m.wo, m.wo, e->map_attn);
+        run_gemm(e, o, m.wo, m.wo, m.wo, e->attn);
         mark(e, LLMA_K_GEMM_O);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         with_norm(e, gu);
         gu.out_act = e->h;
-        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->map_x_hat);
+        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat);
         mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
-        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->map_h);
+        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 5;
     }
@@ -90,7 +90,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         with_norm(e, lm);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
-        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->map_x_hat);
+        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->x_hat);
         mark(e, LLMA_K_GEMM_LMHEAD);
         launch_argmax_final(st, true, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
         mark(e, LLMA_K_ARGMAX);

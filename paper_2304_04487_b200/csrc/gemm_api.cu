@@ -10,15 +10,14 @@ namespace llma {
 // activation buffer [64][k_in] (hi rows, then lo rows).
 int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, int32_t k_in, float* ws,
                        int32_t* cnt, int32_t* dev_err, int grid, cudaStream_t st) {
-    CUtensorMap ma, mb;
+    CUtensorMap ma;
     if (make_tensor_map_bf16(&ma, W, (uint64_t)n_out, (uint64_t)k_in, 128) != 0) return LLMA_ERR_ARG;
-    if (make_tensor_map_bf16(&mb, a, kGemmN, (uint64_t)k_in, kGemmN) != 0) return LLMA_ERR_ARG;
     GemmArgs g;
     std::memset(&g, 0, sizeof(g));
     g.mode = kGemmStore; g.n_out = n_out; g.n_tiles = (n_out + 127) / 128; g.chunks = k_in / 64;
     g.tiles_per_map = g.n_tiles; g.rows = nullptr; g.ws = ws; g.cnt = cnt; g.dev_err = dev_err;
-    g.out_f32 = out; g.ld = n_out;
-    launch_gemm_tcgen05(st, grid, 32, false, g, ma, ma, ma, mb);
+    g.out_f32 = out; g.ld = n_out; g.act = a;
+    launch_gemm_tcgen05(st, grid, 32, false, g, ma, ma, ma);
     CU_TRY(cudaGetLastError());
     return LLMA_OK;
 }

@@ -3,14 +3,15 @@
 //
 // Roles inside one CTA of 192 threads:
 //   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue
-//   warp  4    producer: one thread issues the TMA loads of weight and activation tiles
+//   warp  4    producer: one thread issues the TMA loads of the weight tiles
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
+//   warps 6-9  activation loaders: warp 6 + s fills the activation tile of ring stage s with plain
+//              loads and swizzled shared-memory stores
 // Two accumulators in TMEM let the epilogue of one tile overlap the MMAs of the next.
 //
 // Programmatic dependent launch: the kernel lets its successor start at once, and itself
-// starts streaming WEIGHT tiles (which no earlier kernel writes) before it waits for its
-// predecessor; only the activation tiles and every global access of the epilogue come after
-// that wait.  So the prologue and pipeline fill of one projection overlap the tail of the
+// starts streaming WEIGHT tiles (which no earlier kernel writes) without waiting for its
+// predecessor; only the activation loaders and the epilogue warps wait for it.  So the prologue and pipeline fill of one projection overlap the tail of the
 // kernel before it.
 //
 // Every wait is bounded: when one runs out the kernel raises the device error word, stops
@@ -32,7 +33,7 @@ __device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { retur
 template <int NR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
-               const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b) {
+               const __grid_constant__ CUtensorMap map_a2) {
     using Cfg = GemmCfg<NR>;
     constexpr int S = Cfg::kStages;
     constexpr uint32_t kBBytes = Cfg::kBBytes;
@@ -63,7 +64,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 
     grid_launch_dependents();  // the next kernel may begin its own prologue now
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // a stage is full once its weight tile has landed (producer's expect_tx) and its loader warp has arrived
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(accf_bar(i), 1); mbar_init(acce_bar(i), 4); }
         sh[1] = 0; sh[2] = 0;
         fence_mbar_init();
@@ -73,7 +75,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         tmem_relinquish();
     }
     if (warp == 4 && lane == 0) {
-        tma_prefetch_desc(&map_a0); tma_prefetch_desc(&map_b);
+        tma_prefetch_desc(&map_a0);
         if (g.mode == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
         if (g.mode == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
     }
@@ -97,33 +99,15 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     tma_load_2d(dstA, mp, full_bar(s), c * 64, r0);
                 }
             };
-            auto load_b = [&](int64_t w, int s) {
-                const int c = (int)(w % C);
-                const uint32_t dstB = sB + s * kBBytes;
-                if (NR == kMaxRows) {
-                    tma_load_2d(dstB, &map_b, full_bar(s), c * 64, 0);            // 64 rows: hi then lo
-                } else {
-                    tma_load_2d(dstB, &map_b, full_bar(s), c * 64, 0);            // hi rows 0..NR-1
-                    tma_load_2d(dstB + kBBytes / 2, &map_b, full_bar(s), c * 64, kMaxRows);  // lo rows
-                }
-            };
-            // weights of the first ring-full of items do not depend on any earlier kernel
-            const int64_t n_items = w_end - w_beg;
-            const int n_pre = (int)(n_items < S ? n_items : S);
-            for (int i = 0; i < n_pre; ++i) {
-                mbar_arrive_expect_tx(full_bar(i), kGemmABytes + kBBytes);
-                load_a(w_beg + i, i);
-            }
-            grid_dependency_wait();  // activations are written by the kernel before this one
-            for (int i = 0; i < n_pre; ++i) load_b(w_beg + i, i);
-            int64_t it = n_pre;
-            for (int64_t w = w_beg + n_pre; w < w_end && !sh[1]; ++w, ++it) {
+            // weights are written by no kernel of the step: the whole range streams without waiting for
+            // the predecessor (the MMAs wait for the activation loaders, which do)
+            int64_t it = 0;
+            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w, ++it) {
                 const int s = (int)(it % S);
                 const uint32_t ph = (uint32_t)((it / S) & 1);
-                if (!mbar_wait(empty_bar(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                mbar_arrive_expect_tx(full_bar(s), kGemmABytes + kBBytes);
+                if (it >= S && !mbar_wait(empty_bar(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                mbar_arrive_expect_tx(full_bar(s), kGemmABytes);
                 load_a(w, s);
-                load_b(w, s);
             }
             if (sh[1]) {
                 // give up: let the copies already issued land before the CTA's memory goes away
@@ -162,6 +146,55 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 umma_commit(accf_bar(buf));  // accumulator complete
                 w += c1 - c0;
             }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------- activation loaders ----------------------------------------
+        // Warp 6 + s owns ring stage s.  Tile layout in shared memory (what the MMA's K-major, 128-byte
+        // swizzled descriptor reads): row r = 0..2NR-1 (hi rows, then lo rows) at r * 128 bytes, its
+        // 16-byte unit j stored at position j ^ (r & 7).  Rows past those in use are left as they are:
+        // their columns of the accumulator are never read.
+        static_assert(S == 4, "one loader warp per ring stage");
+        const int sw = warp - 6;
+        grid_dependency_wait();  // activations are written by the kernel before this one
+        const int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : NR;
+        const int64_t n_items = w_end - w_beg;
+        const int64_t ld_bytes = (int64_t)C * 128;  // one activation row: k_in bf16
+        const char* act = reinterpret_cast<const char*>(g.act);
+        constexpr int kUnits = 2 * NR * 8 / 32;     // 16-byte units per lane
+        // rows of the next tile are requested before waiting for its stage to come free, so the
+        // latency of the loads hides behind the MMAs of the tiles in between
+        uint4 v[kUnits];
+        auto fetch = [&](int64_t it) {
+            const int c = (int)((w_beg + it) % C);
+#pragma unroll
+            for (int u = 0; u < kUnits; ++u) {
+                const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
+                const int rr = r < NR ? r : r - NR;                   // row inside its half
+                const int src_row = r < NR ? r : kMaxRows + rr;       // lo rows start at kMaxRows
+                v[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (rr < rows_used)
+                    v[u] = __ldcg(reinterpret_cast<const uint4*>(act + src_row * ld_bytes + (int64_t)c * 128 + j * 16));
+            }
+        };
+        if (sw < n_items) fetch(sw);
+        for (int64_t it = sw; it < n_items && !sh[1]; it += S) {
+            const uint32_t ph = (uint32_t)((it / S) & 1);
+            if (it >= S) {
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(empty_bar(sw), ph ^ 1u);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { if (lane == 0) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; } break; }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnits; ++u) {
+                const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
+                const int rr = r < NR ? r : r - NR;
+                if (rr < rows_used) st_shared_v4(sB + sw * kBBytes + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
+            }
+            fence_proxy_async_shared();  // make the stores visible to the tensor core's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_bar(sw));
+            if (it + S < n_items) fetch(it + S);
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
@@ -359,7 +392,7 @@ cudaError_t init_gemm_tcgen05() {
 }
 
 void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
-                         const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b) {
+                         const CUtensorMap& a1, const CUtensorMap& a2) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kGemmThreads);
@@ -370,8 +403,8 @@ void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const Gemm
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (nr == 16) cudaLaunchKernelEx(&cfg, gemm_ws_kernel<16>, args, a0, a1, a2, b);
-    else cudaLaunchKernelEx(&cfg, gemm_ws_kernel<32>, args, a0, a1, a2, b);
+    if (nr == 16) cudaLaunchKernelEx(&cfg, gemm_ws_kernel<16>, args, a0, a1, a2);
+    else cudaLaunchKernelEx(&cfg, gemm_ws_kernel<32>, args, a0, a1, a2);
 }
 
 void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,

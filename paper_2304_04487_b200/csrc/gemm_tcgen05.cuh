@@ -33,6 +33,7 @@ struct GemmArgs {
     int32_t chunks;         // k_in / 64
     int32_t tiles_per_map;  // tiles per A map
     const RowDesc* rows;    // nullptr: all 32 rows are in use
+    const void* act;        // activation operand, ActLayout kActSplit [2 * kMaxRows][k_in] bf16
     float* ws;              // partial tiles [grid][2][128][32] fp32
     int32_t* cnt;           // arrival counters [n_tiles], zero between launches
     int32_t* dev_err;
@@ -61,14 +62,18 @@ struct GemmArgs {
 };
 
 constexpr int kGemmN = 2 * kMaxRows;  // rows of a split activation buffer: hi rows then lo rows
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;  // 4 epilogue warps, TMA producer, MMA issuer, 4 activation-loader warps
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 
 // The kernel exists for NR = 16 or 32 activation rows per half (MMA N = 2 NR).  Four ring stages
-// (64 KB of weights in flight per SM) measured fastest: deeper rings only lengthen the queues that
-// the activation loads and the epilogue's traffic also wait in.  The request is padded to more than
-// half an SM's shared memory so that the CTAs of two consecutive projections never share an SM
-// (measured 10 % slower when they do).
+// (64 KB of weights in flight per SM) measured fastest inside a decoding step: deeper rings only
+// lengthen the queues that the epilogue's traffic also waits in.  The activation tile of a stage
+// is NOT fetched by TMA: a second, small TMA copy per stage slowed the weight stream by a
+// quarter wherever it came from (shared buffer, per-CTA replica, one hot 4 KB block), whereas
+// plain loads by otherwise idle warps cost almost nothing.  One loader warp per stage copies the
+// rows from global memory into the 128-byte-swizzled layout the MMA expects.
+// The request is padded to more than half an SM's shared memory so that the CTAs of two
+// consecutive projections never share an SM (measured 10 % slower when they do).
 template <int NR> struct GemmCfg {
     static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
     static constexpr int kStages = 4;
@@ -86,10 +91,10 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-// nr = 16 or 32 (the B descriptor's box must hold nr rows for 16, 64 rows for 32); pdl = launch with
-// programmatic stream serialization (the kernel before it must be one of this library's)
+// nr = 16 or 32 activation rows per half; pdl = launch with programmatic stream serialization (the
+// kernel before it must be one of this library's)
 void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
-                         const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b);
+                         const CUtensorMap& a1, const CUtensorMap& a2);
 
 // out_tok[r] = index of the largest logit over all tiles (lowest index on ties)
 void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
