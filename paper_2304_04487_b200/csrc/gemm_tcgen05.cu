@@ -5,8 +5,8 @@
 //   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue
 //   warp  4    producer: one thread issues the TMA loads of the weight tiles
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
-//   warps 6-9  activation loaders: warp 6 + s fills the activation tile of ring stage s with plain
-//              loads and swizzled shared-memory stores
+//   warps 6-9  activation loaders: they take turns filling the activation tile of a ring stage with
+//              plain loads and swizzled shared-memory stores
 // Two accumulators in TMEM let the epilogue of one tile overlap the MMAs of the next.
 //
 // Programmatic dependent launch: the kernel lets its successor start at once, and itself
@@ -149,11 +149,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         }
     } else if (warp >= 6) {
         // ------------------------------- activation loaders ----------------------------------------
-        // Warp 6 + s owns ring stage s.  Tile layout in shared memory (what the MMA's K-major, 128-byte
+        // Tile layout in shared memory (what the MMA's K-major, 128-byte
         // swizzled descriptor reads): row r = 0..2NR-1 (hi rows, then lo rows) at r * 128 bytes, its
         // 16-byte unit j stored at position j ^ (r & 7).  Rows past those in use are left as they are:
         // their columns of the accumulator are never read.
-        static_assert(S == 4, "one loader warp per ring stage");
+        constexpr int NW = 4;  // loader warps: warp 6 + i takes items i, i + NW, ...
         const int sw = warp - 6;
         grid_dependency_wait();  // activations are written by the kernel before this one
         const int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : NR;
@@ -177,11 +177,12 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
         };
         if (sw < n_items) fetch(sw);
-        for (int64_t it = sw; it < n_items && !sh[1]; it += S) {
+        for (int64_t it = sw; it < n_items && !sh[1]; it += NW) {
+            const int st = (int)(it % S);
             const uint32_t ph = (uint32_t)((it / S) & 1);
             if (it >= S) {
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(empty_bar(sw), ph ^ 1u);
+                if (lane == 0) ok = mbar_wait(empty_bar(st), ph ^ 1u);
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { if (lane == 0) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; } break; }
             }
@@ -189,12 +190,12 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             for (int u = 0; u < kUnits; ++u) {
                 const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
                 const int rr = r < NR ? r : r - NR;
-                if (rr < rows_used) st_shared_v4(sB + sw * kBBytes + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
+                if (rr < rows_used) st_shared_v4(sB + st * kBBytes + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
             }
             fence_proxy_async_shared();  // make the stores visible to the tensor core's reads
             __syncwarp();
-            if (lane == 0) mbar_arrive(full_bar(sw));
-            if (it + S < n_items) fetch(it + S);
+            if (lane == 0) mbar_arrive(full_bar(st));
+            if (it + NW < n_items) fetch(it + NW);
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------

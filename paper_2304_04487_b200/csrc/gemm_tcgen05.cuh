@@ -65,18 +65,18 @@ constexpr int kGemmN = 2 * kMaxRows;  // rows of a split activation buffer: hi r
 constexpr int kGemmThreads = 320;  // 4 epilogue warps, TMA producer, MMA issuer, 4 activation-loader warps
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 
-// The kernel exists for NR = 16 or 32 activation rows per half (MMA N = 2 NR).  Four ring stages
-// (64 KB of weights in flight per SM) measured fastest inside a decoding step: deeper rings only
-// lengthen the queues that the epilogue's traffic also waits in.  The activation tile of a stage
+// The kernel exists for NR = 16 or 32 activation rows per half (MMA N = 2 NR).  Ring depths are the
+// ones measured fastest inside a decoding step (8 stages at NR 16, 6 at NR 32; deeper rings only
+// lengthen the queues that the epilogue's traffic also waits in).  The activation tile of a stage
 // is NOT fetched by TMA: a second, small TMA copy per stage slowed the weight stream by a
 // quarter wherever it came from (shared buffer, per-CTA replica, one hot 4 KB block), whereas
-// plain loads by otherwise idle warps cost almost nothing.  One loader warp per stage copies the
-// rows from global memory into the 128-byte-swizzled layout the MMA expects.
+// plain loads by otherwise idle warps cost almost nothing.  Four loader warps take turns copying
+// the rows from global memory into the 128-byte-swizzled layout the MMA expects.
 // The request is padded to more than half an SM's shared memory so that the CTAs of two
 // consecutive projections never share an SM (measured 10 % slower when they do).
 template <int NR> struct GemmCfg {
     static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
-    static constexpr int kStages = 4;
+    static constexpr int kStages = NR == 16 ? 8 : 6;
     static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
