@@ -5,7 +5,10 @@
 // the step, which is what makes verification of k+1 positions cost the K/V traffic of one.
 // Each of the 4 warps takes 32 of the positions: S = Q K^T and O = P V on the tensor cores
 // (mma.sync m16n8k16, bf16 in, fp32 accumulate), softmax statistics by warp shuffles.
-// Q and P enter the MMAs as hi + lo bf16 pairs, so they keep 16 mantissa bits.
+// Q and P enter the MMAs as hi + lo bf16 pairs, so they keep 16 mantissa bits; Q is loaded
+// from global memory directly into operand registers with all loads in flight at once.  The
+// shared-memory request is padded so that two CTAs share an SM, not three: two waves whose loads
+// overlap the other wave's arithmetic measured faster than one wave of everything at once.
 // The warps' partial (max, sum, O) are merged in warp order, the chunk's partial goes to an
 // fp32 workspace, and the last CTA of a (sequence, head) to finish merges the chunks in
 // ascending order.  For a query at absolute position p every one of these decompositions
@@ -47,16 +50,14 @@ struct AttnSmem {
     static constexpr int kBoxes = HD / 64;                    // 64-column TMA boxes per K (or V) tile
     static constexpr uint32_t kBoxBytes = kAttnChunk * 128;   // 128 rows x 128 bytes
     static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;
-    static constexpr uint32_t kQStride = HD * 2 + 16;         // bytes per Q row (padded: conflict-free ldmatrix)
     static constexpr uint32_t offK = 0, offV = kTileBytes;
-    static constexpr uint32_t offQhi = 2 * kTileBytes, offQlo = offQhi + kMaxRows * kQStride;
-    static constexpr uint32_t offO = offQlo + kMaxRows * kQStride;      // fp32 [16][HD] merged tile
+    static constexpr uint32_t offO = 2 * kTileBytes;                     // fp32 [16][HD] merged tile
     static constexpr uint32_t offStat = offO + 16 * HD * 4;              // m_w[4][16], l_w[4][16], misc
-    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64;
+    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kMaxRows * 4;  // + row positions
 };
 
 template <int HD>
-__global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__(128, 2) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
     using L = AttnSmem<HD>;
     pdl_trigger();
@@ -82,7 +83,9 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 1);
     const uint32_t bar_u = smem_u32(bar);
 
+    int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);  // [32] positions of this sequence's rows
     if (threadIdx.x == 0) { mbar_init(bar_u, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0; }
+    if (threadIdx.x < kMaxRows) s_pos[threadIdx.x] = (int)threadIdx.x < cnt ? __ldcg(&a.rows->pos[first + threadIdx.x]) : -1;
     __syncthreads();
     if (threadIdx.x == 0) {
         const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0);
@@ -92,19 +95,32 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
             tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_u, b * 64, row0);
         }
     }
-    // stage Q (this head, this sequence's rows) as hi / lo bf16; rows past cnt are zero
-    {
-        const int HDT = d.hd_total;
-        const int rows_staged = ((cnt + 15) >> 4) << 4;  // whole 16-row MMA tiles; rows past cnt are zero
-        for (int idx = threadIdx.x; idx < rows_staged * HD; idx += blockDim.x) {
-            const int r = idx / HD, i = idx - r * HD;
-            const float v = r < cnt ? a.qkv[(int64_t)(first + r) * 3 * HDT + head * HD + i] : 0.f;
-            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-            *reinterpret_cast<__nv_bfloat16*>(gbase + L::offQhi + r * L::kQStride + i * 2) = hi;
-            *reinterpret_cast<__nv_bfloat16*>(gbase + L::offQlo + r * L::kQStride + i * 2) = lo;
+    // Q (this head, 16 of this sequence's rows) goes straight from global memory into the MMA's
+    // A-operand registers as hi / lo bf16 pairs: lane (g, t) holds rows g and g + 8, columns
+    // 16 ks + 2t, +1, +8, +9.  All loads are issued before any is used; rows past cnt are zero.
+    const int g8 = lane >> 2, t4 = lane & 3;
+    uint32_t qh[HD / 16][4], ql[HD / 16][4];
+    auto load_q = [&](int mt) {
+        const int r0 = mt * 16 + g8, r1 = r0 + 8;
+        const int64_t ldq = 3 * (int64_t)d.hd_total;
+        const float* q0 = a.qkv + (first + r0) * ldq + head * HD + 2 * t4;
+        const float* q1 = q0 + 8 * ldq;
+        float2 x[HD / 16][4];
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+            const float2 z = make_float2(0.f, 0.f);
+            x[ks][0] = r0 < cnt ? __ldcg(reinterpret_cast<const float2*>(q0 + ks * 16)) : z;
+            x[ks][1] = r1 < cnt ? __ldcg(reinterpret_cast<const float2*>(q1 + ks * 16)) : z;
+            x[ks][2] = r0 < cnt ? __ldcg(reinterpret_cast<const float2*>(q0 + ks * 16 + 8)) : z;
+            x[ks][3] = r1 < cnt ? __ldcg(reinterpret_cast<const float2*>(q1 + ks * 16 + 8)) : z;
         }
-    }
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) split_pack(x[ks][i].x, x[ks][i].y, qh[ks][i], ql[ks][i]);
+        }
+    };
+    load_q(0);
     if (threadIdx.x == 0) {
         const bool ok = mbar_wait(bar_u, 0);
         if (!ok) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
@@ -118,6 +134,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     const int64_t part_base = (((int64_t)seq * d.n_heads + head) * a.n_chunks + chunk) * kMaxRows;
 
     for (int mt = 0; mt < n_mt; ++mt) {
+        if (mt > 0) load_q(mt);
         // ---------------- S = Q K^T over this warp's 32 positions ----------------------------
         float s[4][4];
 #pragma unroll
@@ -125,10 +142,8 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
         const int mi = lane >> 3, t8 = lane & 7;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
-            uint32_t ah[4], al[4];
-            const uint32_t qoff = (uint32_t)(mt * 16 + (mi & 1) * 8 + t8) * L::kQStride + (uint32_t)(ks * 16 + (mi >> 1) * 8) * 2;
-            ldsm_x4(base + L::offQhi + qoff, ah);
-            ldsm_x4(base + L::offQlo + qoff, al);
+            const uint32_t (&ah)[4] = qh[ks];
+            const uint32_t (&al)[4] = ql[ks];
 #pragma unroll
             for (int np = 0; np < 2; ++np) {
                 const int row = wpos0 + np * 16 + (mi >> 1) * 8 + t8;
@@ -145,8 +160,8 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
         }
         // ---------------- causal mask, softmax statistics of the warp's span --------------------
         const int r_lo = mt * 16 + (lane >> 2), r_hi = r_lo + 8;
-        const int lim_lo = r_lo < cnt ? a.rows->pos[first + r_lo] : -1;
-        const int lim_hi = r_hi < cnt ? a.rows->pos[first + r_hi] : -1;
+        const int lim_lo = r_lo < cnt ? s_pos[r_lo] : -1;
+        const int lim_hi = r_hi < cnt ? s_pos[r_hi] : -1;
         float m_lo = -INFINITY, m_hi = -INFINITY;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
@@ -275,7 +290,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     __syncthreads();
     if (threadIdx.x < cnt) {  // one thread per row: weights of its chunks, in ascending chunk order
         const int r = threadIdx.x;
-        const int nc = a.rows->pos[first + r] / kAttnChunk + 1;
+        const int nc = s_pos[r] / kAttnChunk + 1;
         float M = -INFINITY;
         for (int c = 0; c < nc; ++c) M = fmaxf(M, c_m[c * kMaxRows + r]);
         float den = 0.f;
@@ -289,26 +304,25 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
         r_den[r] = den;
     }
     __syncthreads();
+    // Output element group (row r, 4 columns): its chunks' partials are requested sixteen at a time
+    // and summed in ascending chunk order.
     for (int idx = threadIdx.x; idx < cnt * (HD / 4); idx += blockDim.x) {
         const int r = idx / (HD / 4), i4 = idx - r * (HD / 4);
-        const int nc = a.rows->pos[first + r] / kAttnChunk + 1;
+        const int nc = s_pos[r] / kAttnChunk + 1;
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
         const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + i4;
-        int c = 0;
-        for (; c + 4 <= nc; c += 4) {  // four independent loads in flight, summed in ascending order
-            float4 p[4];
+        for (int c = 0; c < nc; c += 16) {
+            float4 p[16];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) p[u] = __ldcg(src + (int64_t)(c + u) * kMaxRows * (HD / 4));
+            for (int u = 0; u < 16; ++u)
+                if (c + u < nc) p[u] = __ldcg(src + (int64_t)(c + u) * kMaxRows * (HD / 4));
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float f = c_m[(c + u) * kMaxRows + r];
-                num.x += f * p[u].x; num.y += f * p[u].y; num.z += f * p[u].z; num.w += f * p[u].w;
+            for (int u = 0; u < 16; ++u) {
+                if (c + u < nc) {
+                    const float f = c_m[(c + u) * kMaxRows + r];
+                    num.x += f * p[u].x; num.y += f * p[u].y; num.z += f * p[u].z; num.w += f * p[u].w;
+                }
             }
-        }
-        for (; c < nc; ++c) {
-            const float4 p = __ldcg(src + (int64_t)c * kMaxRows * (HD / 4));
-            const float f = c_m[c * kMaxRows + r];
-            num.x += f * p.x; num.y += f * p.y; num.z += f * p.z; num.w += f * p.w;
         }
         const float den = r_den[r];
         const int64_t col = (int64_t)head * HD + i4 * 4;
@@ -319,9 +333,11 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const AttnArgs a, co
     }
 }
 
+constexpr size_t kAttnPad = 20 * 1024;  // see the header comment: keeps the 128-wide-head kernel at two CTAs per SM
+
 cudaError_t init_attention_mma() {
     cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(AttnSmem<128>::kBytes + 1024));
+                                         (int)(AttnSmem<128>::kBytes + 1024 + kAttnPad));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)(AttnSmem<64>::kBytes + 1024));
@@ -330,7 +346,7 @@ cudaError_t init_attention_mma() {
 void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v) {
     dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
     if (a.dims.head_dim == 128)
-        launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024, attention_mma_kernel<128>, a, map_k, map_v);
+        launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128>, a, map_k, map_v);
     else
         launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64>, a, map_k, map_v);
 }

@@ -31,13 +31,13 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
     const bool fold = g.xs_out != nullptr;
     const float gain = (fold && valid) ? __ldg(&g.gain_next[col]) : 0.f;
     const int warp = row >> 5, lane = row & 31;
-    for (int j0 = 0; j0 < rows_used; j0 += 4) {
-        float xv[4];
+    for (int j0 = 0; j0 < rows_used; j0 += 8) {
+        float xv[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < 8; ++u)
             xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const int j = j0 + u;
             if (j < rows_used) {
                 const float xn = valid ? xv[u] + stage[row][j] : 0.f;
@@ -68,7 +68,8 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int 
 // QKV: rotary embedding on q and k (pair (i, i + hd/2)), q to the fp32 qkv buffer, k and v
 // rows into the bf16 cache at (sequence, position) of every used row.
 __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, int rows_used,
-                                             float (*stage)[33]) {
+                                             float (*stage)[33], const int* rowinfo) {
+    // rowinfo[j] = position of activation row j (-1: unused), rowinfo[32 + j] = its sequence slot
     const ModelDims& d = g.dims;
     const int mat = tile / g.tiles_per_map;
     const int col = (tile % g.tiles_per_map) * 128 + row;
@@ -78,26 +79,22 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
     const int prow = lower ? row + half : row - half;
     const int fi = idx % half;
     if (col < g.n_out) {
-        for (int j0 = 0; j0 < rows_used; j0 += 2) {
-            int pos[2], sq[2];
-            float c[2], sn[2];
+        for (int j0 = 0; j0 < rows_used; j0 += 8) {  // the rotary factors of eight rows are requested together
+            float c[8], sn[8];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                pos[u] = j0 + u < rows_used ? __ldcg(&g.rows->pos[j0 + u]) : -1;
-                sq[u] = j0 + u < rows_used ? __ldcg(&g.rows->seq[j0 + u]) : 0;
-            }
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < 8; ++u) {
+                const int pos = j0 + u < rows_used ? rowinfo[j0 + u] : -1;
                 c[u] = 1.f; sn[u] = 0.f;
-                if (pos[u] >= 0 && mat < 2) {
-                    c[u] = __ldg(&g.rope_cos[(int64_t)pos[u] * half + fi]);
-                    sn[u] = __ldg(&g.rope_sin[(int64_t)pos[u] * half + fi]);
+                if (pos >= 0 && mat < 2) {
+                    c[u] = __ldg(&g.rope_cos[(int64_t)pos * half + fi]);
+                    sn[u] = __ldg(&g.rope_sin[(int64_t)pos * half + fi]);
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 const int j = j0 + u;
-                if (pos[u] < 0) continue;
+                const int pos = j < rows_used ? rowinfo[j] : -1;
+                if (pos < 0) continue;
                 float val = stage[row][j];
                 if (mat < 2) {
                     const float other = stage[prow][j];
@@ -107,7 +104,7 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
                     g.out_f32[(int64_t)j * g.ld + col] = val;
                 } else {
                     __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
-                    cache[kv_row_index(d, g.layer, sq[u], head, pos[u]) * hd + idx] = __float2bfloat16_rn(val);
+                    cache[kv_row_index(d, g.layer, rowinfo[32 + j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
                 }
             }
         }

@@ -202,14 +202,24 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
         const int rows_used = g.rows ? g.rows->rows_used : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
-        if (g.ss_in) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
-            if (row < 32) {
-                float ssum = 0.f;
-                for (int t = 0; t < g.ss_tiles; ++t) ssum += g.ss_in[(int64_t)t * 32 + row];
-                rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
+        if (g.ss_in && row < 32) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
+            float ssum = 0.f;
+            int t = 0;
+            for (; t + 8 <= g.ss_tiles; t += 8) {  // eight loads in flight
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __ldcg(&g.ss_in[(int64_t)(t + u) * 32 + row]);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) ssum += v[u];
             }
-            epi_sync();
+            for (; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * 32 + row]);
+            rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
         }
+        if (g.mode == kGemmQKV) {  // the rows' positions and sequence slots, read once per CTA
+            if (row < 32) red_i[row] = __ldcg(&g.rows->pos[row]);
+            else if (row < 64) red_i[row] = __ldcg(&g.rows->seq[row - 32]);
+        }
+        epi_sync();
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
             const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
@@ -258,7 +268,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const int my_slot = (w_beg >= t_lo) ? 0 : 1;  // first segment of my range, or its last
                 float4* dst = reinterpret_cast<float4*>(g.ws + (((int64_t)b * 2 + my_slot) * 128 + row) * 32);
 #pragma unroll
-                for (int q = 0; q < NR / 4; ++q) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                for (int q = 0; q < NR / 4; ++q)  // only the columns of rows in use travel
+                    if (4 * q < rows_used) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
                 __threadfence();
                 epi_sync();
                 if (threadIdx.x == 0) {
@@ -285,7 +296,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                             const float4* src =
                                 reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + slot) * 128 + row) * 32);
 #pragma unroll
-                            for (int q = 0; q < NR / 4; ++q) p[u][q] = __ldcg(src + q);
+                            for (int q = 0; q < NR / 4; ++q)
+                                if (4 * q < rows_used) p[u][q] = __ldcg(src + q);
                         }
                     }
 #pragma unroll
@@ -293,8 +305,10 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                         if (bb + u <= b_last) {
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q) {
-                                acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
-                                acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
+                                if (4 * q < rows_used) {
+                                    acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
+                                    acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
+                                }
                             }
                         }
                     }
@@ -310,7 +324,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
             epi_sync();
             switch (g.mode) {
-                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage); break;
+                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i); break;
                 case kGemmResid: epilogue_resid(g, tile, row, rows_used, stage, red_f); break;
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
                 case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
