@@ -24,8 +24,10 @@ __device__ __forceinline__ float warp_sum(float v) {
 // x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
 // When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
 // per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
+// With kHavePre, xpre holds x[0..7, col], read earlier by the caller.
+template <bool kHavePre>
 __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int rows_used,
-                                               float (*stage)[33], float* red_f) {
+                                               float (*stage)[33], float* red_f, const float (&xpre)[8]) {
     const int col = tile * 128 + row;
     const bool valid = col < g.n_out;
     const bool fold = g.xs_out != nullptr;
@@ -34,8 +36,10 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
     for (int j0 = 0; j0 < rows_used; j0 += 8) {
         float xv[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
+        for (int u = 0; u < 8; ++u) {
+            if (kHavePre && j0 == 0) xv[u] = xpre[u];
+            else xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
+        }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int j = j0 + u;

@@ -227,6 +227,16 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             w += c1 - c0;
             const int buf = seg & 1;
             const uint32_t use = (uint32_t)(seg >> 1);
+            // residual rows of this tile: requested now, so their latency hides behind the accumulator wait
+            // and the cross-CTA sum (only this tile's final owner ever writes them, in its epilogue below)
+            float xpre[8];
+            constexpr bool kPrefetchX = NR == 16;  // at 32 rows the extra registers spill
+            if (kPrefetchX && g.mode == kGemmResid) {
+                const int col = tile * 128 + row;
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    xpre[u] = (col < g.n_out && u < rows_used) ? __ldcg(&g.out_f32[(int64_t)u * g.ld + col]) : 0.f;
+            }
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
                 if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
@@ -325,7 +335,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             epi_sync();
             switch (g.mode) {
                 case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i); break;
-                case kGemmResid: epilogue_resid(g, tile, row, rows_used, stage, red_f); break;
+                case kGemmResid: epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre); break;
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
                 case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
                 default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
