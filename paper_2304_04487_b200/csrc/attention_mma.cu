@@ -9,8 +9,8 @@
 // from global memory directly into operand registers with all loads in flight at once.  The
 // shared-memory request is padded so that two CTAs share an SM, not three: two waves whose loads
 // overlap the other wave's arithmetic measured faster than one wave of everything at once.
-// The warps' partial (max, sum, O) are merged in warp order, the chunk's partial goes to an
-// fp32 workspace, and the last CTA of a (sequence, head) to finish merges the chunks in
+// The warps' partial (max, sum, O) are merged in warp order and the chunk's partial goes to an
+// fp32 workspace; a second small kernel merges the chunks of every (sequence, head, row) in
 // ascending order.  For a query at absolute position p every one of these decompositions
 // is a function of p alone (chunks and warp spans are fixed position ranges, later positions
 // are masked to exact zeros), so a row's result does not depend on the other rows.
@@ -71,7 +71,6 @@ __global__ void __launch_bounds__(128, 2) attention_mma_kernel(const AttnArgs a,
     const int maxpos = __ldcg(&a.rows->seq_maxpos[seq]);
     const int c0 = chunk * kAttnChunk;
     if (cnt == 0 || c0 > maxpos) return;  // uniform over the CTA
-    const int n_active = maxpos / kAttnChunk + 1;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -263,55 +262,46 @@ __global__ void __launch_bounds__(128, 2) attention_mma_kernel(const AttnArgs a,
         }
         __syncthreads();
     }
+}
 
-    // ---------------- last CTA of this (sequence, head): merge the chunks in ascending order ----------
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(&a.cnt[seq * d.n_heads + head], 1);
-        const bool last = old == n_active - 1;
-        if (last) a.cnt[seq * d.n_heads + head] = 0;
-        flag[1] = last ? 1u : 0u;
-    }
-    __syncthreads();
-    if (!flag[1]) return;
-    __threadfence();
-    // The K/V tiles are no longer needed: reuse their shared memory for the chunk statistics.
+// Second pass: one warp per (sequence, head, row) combines the row's chunk partials in ascending chunk
+// order.  A kernel of its own, so that every head is merged at once instead of by whichever CTA of the
+// head happened to finish last; a row's result still depends on its own position only.
+template <int HD>
+__global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ float s_w[];  // [4 warps][n_chunks] weights, then [4][n_chunks] weighted sums
+    const int head = blockIdx.x, seq = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const ModelDims& d = a.dims;
+    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
+    const int r = blockIdx.y * 4 + warp;
+    if (r >= cnt) return;
+    const int nc = __ldcg(&a.rows->pos[first + r]) / kAttnChunk + 1;
     const int64_t head_base = ((int64_t)seq * d.n_heads + head) * a.n_chunks * kMaxRows;
-    float* c_m = reinterpret_cast<float*>(gbase + L::offK);   // [n_active][32] chunk maxima, then weights
-    float* c_l = c_m + (size_t)a.n_chunks * kMaxRows;         // [n_active][32] chunk sums
-    float* r_den = reinterpret_cast<float*>(gbase + L::offO);  // [32]
-    for (int idx = threadIdx.x; idx < n_active * cnt; idx += blockDim.x) {
-        const int c = idx / cnt, r = idx - c * cnt;
+    float* w_c = s_w + warp * a.n_chunks;
+    float* wl_c = s_w + (4 + warp) * a.n_chunks;
+    float M = -INFINITY;
+    for (int c = lane; c < nc; c += 32) {
         const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * kMaxRows + r);
-        c_m[c * kMaxRows + r] = ml.x;
-        c_l[c * kMaxRows + r] = ml.y;
+        w_c[c] = ml.x; wl_c[c] = ml.y;
+        M = fmaxf(M, ml.x);
     }
-    __syncthreads();
-    if (threadIdx.x < cnt) {  // one thread per row: weights of its chunks, in ascending chunk order
-        const int r = threadIdx.x;
-        const int nc = s_pos[r] / kAttnChunk + 1;
-        float M = -INFINITY;
-        for (int c = 0; c < nc; ++c) M = fmaxf(M, c_m[c * kMaxRows + r]);
-        float den = 0.f;
-        for (int c = 0; c < nc; ++c) {
-            const float mc = c_m[c * kMaxRows + r];
-            const float f = mc == -INFINITY ? 0.f : expf(mc - M);
-            den += f * c_l[c * kMaxRows + r];
-            c_m[c * kMaxRows + r] = f;
-        }
-        for (int c = nc; c < n_active; ++c) c_m[c * kMaxRows + r] = 0.f;
-        r_den[r] = den;
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    __syncwarp();
+    for (int c = lane; c < nc; c += 32) {
+        const float mc = w_c[c];
+        const float f = mc == -INFINITY ? 0.f : expf(mc - M);
+        w_c[c] = f; wl_c[c] = f * wl_c[c];
     }
-    __syncthreads();
-    // Output element group (row r, 4 columns): its chunks' partials are requested sixteen at a time
-    // and summed in ascending chunk order.
-    for (int idx = threadIdx.x; idx < cnt * (HD / 4); idx += blockDim.x) {
-        const int r = idx / (HD / 4), i4 = idx - r * (HD / 4);
-        const int nc = s_pos[r] / kAttnChunk + 1;
+    __syncwarp();
+    float den = 0.f;
+    for (int c = 0; c < nc; ++c) den += wl_c[c];  // ascending order, the same in every lane
+    if (lane < HD / 4) {
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + i4;
-        for (int c = 0; c < nc; c += 16) {
+        const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + lane;
+        for (int c = 0; c < nc; c += 16) {  // sixteen partials requested together
             float4 p[16];
 #pragma unroll
             for (int u = 0; u < 16; ++u)
@@ -319,13 +309,12 @@ __global__ void __launch_bounds__(128, 2) attention_mma_kernel(const AttnArgs a,
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
                 if (c + u < nc) {
-                    const float f = c_m[(c + u) * kMaxRows + r];
+                    const float f = w_c[c + u];
                     num.x += f * p[u].x; num.y += f * p[u].y; num.z += f * p[u].z; num.w += f * p[u].w;
                 }
             }
         }
-        const float den = r_den[r];
-        const int64_t col = (int64_t)head * HD + i4 * 4;
+        const int64_t col = (int64_t)head * HD + lane * 4;
         store_act(a.attn_out, kActSplit, first + r, col, d.hd_total, num.x / den);
         store_act(a.attn_out, kActSplit, first + r, col + 1, d.hd_total, num.y / den);
         store_act(a.attn_out, kActSplit, first + r, col + 2, d.hd_total, num.z / den);
@@ -345,10 +334,15 @@ cudaError_t init_attention_mma() {
 
 void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v) {
     dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
-    if (a.dims.head_dim == 128)
+    dim3 mgrid(a.dims.n_heads, kMaxRows / 4, a.dims.max_batch);
+    const size_t msmem = (size_t)8 * a.n_chunks * sizeof(float);
+    if (a.dims.head_dim == 128) {
         launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128>, a, map_k, map_v);
-    else
+        launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<128>, a);
+    } else {
         launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64>, a, map_k, map_v);
+        launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<64>, a);
+    }
 }
 
 }  // namespace llma

@@ -82,7 +82,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
         run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h);
         mark(e, LLMA_K_GEMM_DOWN);
-        e->launch_counter += 5;
+        e->launch_counter += 6;
     }
     if (lm_head) {
         const int vt = (d.vocab + 127) / 128;
