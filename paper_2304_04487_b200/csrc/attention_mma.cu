@@ -6,14 +6,9 @@
 // Each of the 4 warps takes 32 of the positions: S = Q K^T and O = P V on the tensor cores
 // (mma.sync m16n8k16, bf16 in, fp32 accumulate), softmax statistics by warp shuffles.
 // Q and P enter the MMAs as hi + lo bf16 pairs, so they keep 16 mantissa bits; Q is loaded
-// from global memory directly into operand registers with all loads in flight at once.  The
-// shared-memory request is padded so that two CTAs share an SM, not three: two waves whose loads
-// overlap the other wave's arithmetic measured faster than one wave of everything at once.
-// The warps' partial (max, sum, O) are merged in warp order and the chunk's partial goes to an
-// fp32 workspace; a second small kernel merges the chunks of every (sequence, head, row) in
-// ascending order.  For a query at absolute position p every one of these decompositions
-// is a function of p alone (chunks and warp spans are fixed position ranges, later positions
-// are masked to exact zeros), so a row's result does not depend on the other rows.
+// from global memory directly into operand registers with all loads in flight at once, which
+// keeps a CTA at 73 KB of shared memory: three CTAs per SM, one wave up to about 1.8 k cached
+// positions at 32 heads.
 #include <cuda.h>
 
 #include "attention_mma.cuh"
@@ -57,7 +52,7 @@ struct AttnSmem {
 };
 
 template <int HD>
-__global__ void __launch_bounds__(128, 2) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
     using L = AttnSmem<HD>;
     pdl_trigger();
@@ -322,7 +317,7 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
     }
 }
 
-constexpr size_t kAttnPad = 20 * 1024;  // see the header comment: keeps the 128-wide-head kernel at two CTAs per SM
+constexpr size_t kAttnPad = 0;  // extra shared memory per CTA (a knob for the number of CTAs per SM)
 
 cudaError_t init_attention_mma() {
     cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
