@@ -162,6 +162,8 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         const int vt = (d.vocab + 127) / 128;
         const int max_tiles = std::max(std::max(vt, 3 * HD / 128), std::max((d.d_ffn + 63) / 64, (d.d_model + 127) / 128));
         CREATE_TRY(dalloc(&e->gemm_ws, (size_t)e->num_sms * 2 * 128 * 32));
+        // hand-over slots start out empty: every word the all-ones pattern (see gemm_ws_kernel)
+        if (cudaMemset(e->gemm_ws, 0xFF, (size_t)e->num_sms * 2 * 128 * 32 * sizeof(float)) != cudaSuccess) { free_engine(e); return LLMA_ERR_CUDA; }
         CREATE_TRY(dalloc(&e->gemm_cnt, (size_t)max_tiles));
         CREATE_TRY(dalloc(&e->part_max, (size_t)vt * 32));
         CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * 32));

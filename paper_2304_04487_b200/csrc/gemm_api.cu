@@ -47,6 +47,7 @@ extern "C" int llma_gemm_rows32_bf16(const void* W, const void* a, float* out, i
     int rc = LLMA_OK;
     int32_t err = 0;
     ce = cudaMemsetAsync(cnt, 0, ((size_t)n_tiles + 1) * sizeof(int32_t), st);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(ws, 0xFF, (size_t)grid * 2 * 128 * 32 * sizeof(float), st);  // hand-over slots empty
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(a2, a, a_bytes, cudaMemcpyDeviceToDevice, st);
     if (ce == cudaSuccess) ce = cudaMemsetAsync((char*)a2 + a_bytes, 0, a_bytes, st);
     if (ce == cudaSuccess) rc = gemm_rows32_launch(W, a2, out, n_out, k_in, ws, cnt, cnt + n_tiles, grid, st);

@@ -72,6 +72,8 @@ extern "C" int llma_gemm_rows32_bf16_noalloc(const void* W, const void* a, float
     // the array keeps the previous call's contents: counters and the error word must start at
     // zero, and the low half of the operand must be zero (this entry point takes plain bf16 rows)
     CU_TRY(cudaMemsetAsync(cnt, 0, ((size_t)n_tiles + 1) * sizeof(int32_t), st));
+    // the partial-tile hand-over slots must read as empty (all-ones words) when the kernel starts
+    CU_TRY(cudaMemsetAsync(ws, 0xFF, (size_t)grid * 2 * 128 * 32 * sizeof(float), st));
     CU_TRY(cudaMemcpyAsync(operand, a, a_bytes, cudaMemcpyDeviceToDevice, st));
     CU_TRY(cudaMemsetAsync(reinterpret_cast<char*>(operand) + a_bytes, 0, a_bytes, st));
     int rc = gemm_rows32_launch(W, operand, out, n_out, k_in, ws, cnt, cnt + n_tiles, grid, st);

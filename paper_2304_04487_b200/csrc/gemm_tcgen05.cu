@@ -220,6 +220,45 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             else if (row < 64) red_i[row] = __ldcg(&g.rows->seq[row - 32]);
         }
         epi_sync();
+        constexpr bool kPrefetchX = NR == 16;  // at 32 rows the extra registers spill
+        // residual rows of a tile: requested early, so their latency hides behind the accumulator wait
+        // and the cross-CTA sum (only the tile's owner ever writes them, in its epilogue)
+        auto prefetch_x = [&](int tile, float (&xpre)[8]) {
+            if (kPrefetchX && g.mode == kGemmResid) {
+                const int col = tile * 128 + row;
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    xpre[u] = (col < g.n_out && u < rows_used) ? __ldcg(&g.out_f32[(int64_t)u * g.ld + col]) : 0.f;
+            }
+        };
+        // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
+        auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[8]) {
+            if (g.ss_in) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[j];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
+            }
+            epi_sync();
+            switch (g.mode) {
+                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i); break;
+                case kGemmResid: epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre); break;
+                case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
+                case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
+                default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
+            }
+        };
+        // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks
+        // its own partial (slot 0 of its workspace) and completes the tile after its last segment.  Every
+        // other CTA of the tile hands its partial over through slot 1, whose words hold the bit pattern
+        // kEmpty (a NaN no arithmetic here produces) while nothing has been handed over: the owner polls
+        // the words it needs until none is kEmpty, adds the partials in ascending k order, and puts kEmpty
+        // back.  No fence, counter or second pass: one store and one load stand between the last MMA of a
+        // neighbour and the owner's epilogue.
+        constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+        int own_tile = -1, own_first = 0;
+        bool aborted = false;
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
             const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
@@ -227,16 +266,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             w += c1 - c0;
             const int buf = seg & 1;
             const uint32_t use = (uint32_t)(seg >> 1);
-            // residual rows of this tile: requested now, so their latency hides behind the accumulator wait
-            // and the cross-CTA sum (only this tile's final owner ever writes them, in its epilogue below)
             float xpre[8];
-            constexpr bool kPrefetchX = NR == 16;  // at 32 rows the extra registers spill
-            if (kPrefetchX && g.mode == kGemmResid) {
-                const int col = tile * 128 + row;
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    xpre[u] = (col < g.n_out && u < rows_used) ? __ldcg(&g.out_f32[(int64_t)u * g.ld + col]) : 0.f;
-            }
+            prefetch_x(tile, xpre);
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
                 if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
@@ -245,7 +276,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             epi_sync();
             const bool ok = sh[2] != 0;
             epi_sync();
-            if (!ok) break;
+            if (!ok) { aborted = true; break; }
             tc_fence_after();
             float acc[32];
             {
@@ -266,45 +297,41 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             __syncwarp();
             if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
 
-            // ---- tiles shared by several CTAs: write the partial, the last arriver sums all ----
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
-            int b_first = (int)(t_lo * G / work);
-            while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
-            while (cta_begin(work, b_first, G) > t_lo) --b_first;
-            int b_last = (int)((t_hi - 1) * G / work);
-            while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
-            while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
-            if (b_first != b_last) {
-                const int my_slot = (w_beg >= t_lo) ? 0 : 1;  // first segment of my range, or its last
-                float4* dst = reinterpret_cast<float4*>(g.ws + (((int64_t)b * 2 + my_slot) * 128 + row) * 32);
+            if (w_beg > t_lo || w_end < t_hi) {  // the tile is shared with a neighbour
+                const bool owner = w_end >= t_hi;
+                float4* dst = reinterpret_cast<float4*>(g.ws + (((int64_t)b * 2 + (owner ? 0 : 1)) * 128 + row) * 32);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q)  // only the columns of rows in use travel
                     if (4 * q < rows_used) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-                __threadfence();
-                epi_sync();
-                if (threadIdx.x == 0) {
-                    const int old = atomicAdd(&g.cnt[tile], 1);
-                    const bool last = old == (b_last - b_first);
-                    if (last) g.cnt[tile] = 0;
-                    sh[2] = last ? 1u : 0u;
+                if (owner) {
+                    int b_first = (int)(t_lo * G / work);
+                    while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
+                    while (cta_begin(work, b_first, G) > t_lo) --b_first;
+                    own_tile = tile; own_first = b_first;
                 }
-                epi_sync();
-                const bool last = sh[2] != 0;
-                epi_sync();
-                if (!last) continue;
-                __threadfence();
+                continue;
+            }
+            finish_tile(tile, acc, xpre);
+        }
+        if (own_tile >= 0 && !aborted) {
+            float xpre[8];
+            prefetch_x(own_tile, xpre);
+            float acc[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                // ascending k: a fixed summation order; loads of several partials are issued together
-                constexpr int kBatch = NR == 16 ? 4 : 2;
-                for (int bb = b_first; bb <= b_last; bb += kBatch) {
-                    float4 p[kBatch][NR / 4];
+            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
+            constexpr int kBatch = NR == 16 ? 4 : 2;
+            for (int bb = own_first; bb < b; bb += kBatch) {  // ascending k: a fixed summation order
+                float4 p[kBatch][NR / 4];
+                bool valid;
+                do {
+                    valid = true;
 #pragma unroll
                     for (int u = 0; u < kBatch; ++u) {
-                        if (bb + u <= b_last) {
-                            const int slot = (cta_begin(work, bb + u, G) >= t_lo) ? 0 : 1;
+                        if (bb + u < b) {
                             const float4* src =
-                                reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + slot) * 128 + row) * 32);
+                                reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + 1) * 128 + row) * 32);
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q)
                                 if (4 * q < rows_used) p[u][q] = __ldcg(src + q);
@@ -312,34 +339,47 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     }
 #pragma unroll
                     for (int u = 0; u < kBatch; ++u) {
-                        if (bb + u <= b_last) {
+                        if (bb + u < b) {
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q) {
                                 if (4 * q < rows_used) {
-                                    acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
-                                    acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
+                                    valid = valid && __float_as_uint(p[u][q].x) != kEmpty;
+                                    if (4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[u][q].y) != kEmpty;
+                                    if (4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[u][q].z) != kEmpty;
+                                    if (4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[u][q].w) != kEmpty;
                                 }
+                            }
+                        }
+                    }
+                    if (!valid && globaltimer_ns() > give_up) { atomicExch(g.dev_err, kDevErrTimeout); break; }
+                } while (!valid);
+                const float e = __uint_as_float(kEmpty);
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    if (bb + u < b) {
+                        float4* src = reinterpret_cast<float4*>(g.ws + (((int64_t)(bb + u) * 2 + 1) * 128 + row) * 32);
+#pragma unroll
+                        for (int q = 0; q < NR / 4; ++q) {
+                            if (4 * q < rows_used) {
+                                src[q] = make_float4(e, e, e, e);  // empty again for the next projection
+                                acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
+                                acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
                             }
                         }
                     }
                 }
             }
-            // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
-            if (g.ss_in) {
+            {   // this CTA's own partial comes last (it holds the highest k)
+                const float4* src = reinterpret_cast<const float4*>(g.ws + (((int64_t)b * 2) * 128 + row) * 32);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[j];
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
+                for (int q = 0; q < NR / 4; ++q) {
+                    if (4 * q < rows_used) {
+                        const float4 v = src[q];
+                        acc[4 * q] += v.x; acc[4 * q + 1] += v.y; acc[4 * q + 2] += v.z; acc[4 * q + 3] += v.w;
+                    }
+                }
             }
-            epi_sync();
-            switch (g.mode) {
-                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i); break;
-                case kGemmResid: epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre); break;
-                case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
-                case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
-                default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
-            }
+            finish_tile(own_tile, acc, xpre);
         }
     }
     tc_fence_before();
