@@ -33,6 +33,7 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
     const bool fold = g.xs_out != nullptr;
     const float gain = (fold && valid) ? __ldg(&g.gain_next[col]) : 0.f;
     const int warp = row >> 5, lane = row & 31;
+    // x is added into the staged tile with a few loads in flight; the per-row work is a rolled loop
     for (int j0 = 0; j0 < rows_used; j0 += 8) {
         float xv[8];
 #pragma unroll
@@ -41,17 +42,17 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
             else xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int j = j0 + u;
-            if (j < rows_used) {
-                const float xn = valid ? xv[u] + stage[row][j] : 0.f;
-                if (valid) g.out_f32[(int64_t)j * g.ld + col] = xn;
-                if (fold) {
-                    if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn * gain);
-                    const float sq = warp_sum(xn * xn);
-                    if (lane == 0) red_f[warp * 32 + j] = sq;
-                }
-            }
+        for (int u = 0; u < 8; ++u)
+            if (j0 + u < rows_used) stage[row][j0 + u] += xv[u];
+    }
+#pragma unroll 1
+    for (int j = 0; j < rows_used; ++j) {
+        const float xn = valid ? stage[row][j] : 0.f;
+        if (valid) g.out_f32[(int64_t)j * g.ld + col] = xn;
+        if (fold) {
+            if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn * gain);
+            const float sq = warp_sum(xn * xn);
+            if (lane == 0) red_f[warp * 32 + j] = sq;
         }
     }
     if (!fold) return;
