@@ -73,8 +73,9 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int 
 // QKV: rotary embedding on q and k (pair (i, i + hd/2)), q to the fp32 qkv buffer, k and v
 // rows into the bf16 cache at (sequence, position) of every used row.
 __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, int rows_used,
-                                             float (*stage)[33], const int* rowinfo) {
-    // rowinfo[j] = position of activation row j (-1: unused), rowinfo[32 + j] = its sequence slot
+                                             float (*stage)[33], const int* rowinfo, const float2* rope_s) {
+    // rowinfo[j] = position of activation row j (-1: unused), rowinfo[32 + j] = its sequence slot;
+    // rope_s[j * hd/2 + i] = (cos, sin) of row j's position for rotary pair i
     const ModelDims& d = g.dims;
     const int mat = tile / g.tiles_per_map;
     const int col = (tile % g.tiles_per_map) * 128 + row;
@@ -84,33 +85,21 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
     const int prow = lower ? row + half : row - half;
     const int fi = idx % half;
     if (col < g.n_out) {
-        for (int j0 = 0; j0 < rows_used; j0 += 8) {  // the rotary factors of eight rows are requested together
-            float c[8], sn[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int pos = j0 + u < rows_used ? rowinfo[j0 + u] : -1;
-                c[u] = 1.f; sn[u] = 0.f;
-                if (pos >= 0 && mat < 2) {
-                    c[u] = __ldg(&g.rope_cos[(int64_t)pos * half + fi]);
-                    sn[u] = __ldg(&g.rope_sin[(int64_t)pos * half + fi]);
-                }
+#pragma unroll 1
+        for (int j = 0; j < rows_used; ++j) {
+            const int pos = rowinfo[j];
+            if (pos < 0) continue;
+            float val = stage[row][j];
+            if (mat < 2) {
+                const float2 cs = rope_s[j * half + fi];
+                const float other = stage[prow][j];
+                val = lower ? (val * cs.x - other * cs.y) : (other * cs.y + val * cs.x);
             }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int j = j0 + u;
-                const int pos = j < rows_used ? rowinfo[j] : -1;
-                if (pos < 0) continue;
-                float val = stage[row][j];
-                if (mat < 2) {
-                    const float other = stage[prow][j];
-                    val = lower ? (val * c[u] - other * sn[u]) : (other * sn[u] + val * c[u]);
-                }
-                if (mat == 0) {
-                    g.out_f32[(int64_t)j * g.ld + col] = val;
-                } else {
-                    __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
-                    cache[kv_row_index(d, g.layer, rowinfo[32 + j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
-                }
+            if (mat == 0) {
+                g.out_f32[(int64_t)j * g.ld + col] = val;
+            } else {
+                __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
+                cache[kv_row_index(d, g.layer, rowinfo[32 + j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
             }
         }
     }

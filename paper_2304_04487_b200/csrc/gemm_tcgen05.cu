@@ -49,6 +49,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     float* rscale = reinterpret_cast<float*>(tail + (2 * S + 4) * 8 + 16);  // [32] per-row norm scales
     float* red_f = rscale + 32;                                             // [4][32] reduction scratch
     int* red_i = reinterpret_cast<int*>(red_f + 128);                       // [4][32]
+    float2* rope_s = reinterpret_cast<float2*>(tail + 1536);                // [32][head_dim / 2] (QKV mode)
     // sh[0] = TMEM base, sh[1] = abort flag, sh[2] = epilogue broadcast word
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -220,6 +221,18 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             else if (row < 64) red_i[row] = __ldcg(&g.rows->seq[row - 32]);
         }
         epi_sync();
+        if (g.mode == kGemmQKV) {
+            // rotary factors of every row in use, once per CTA: the tile epilogues then read shared memory only
+            const int half = g.dims.head_dim >> 1;
+            for (int idx = row; idx < rows_used * half; idx += 128) {
+                const int j = idx / half, fi = idx - j * half;
+                const int pos = red_i[j];
+                float2 cs = make_float2(1.f, 0.f);
+                if (pos >= 0) cs = make_float2(__ldg(&g.rope_cos[(int64_t)pos * half + fi]), __ldg(&g.rope_sin[(int64_t)pos * half + fi]));
+                rope_s[j * half + fi] = cs;
+            }
+            epi_sync();
+        }
         constexpr bool kPrefetchX = NR == 16;  // at 32 rows the extra registers spill
         // residual rows of a tile: requested early, so their latency hides behind the accumulator wait
         // and the cross-CTA sum (only the tile's owner ever writes them, in its epilogue)
@@ -242,7 +255,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
             epi_sync();
             switch (g.mode) {
-                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i); break;
+                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i, rope_s); break;
                 case kGemmResid: epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre); break;
                 case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
                 case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;

@@ -77,7 +77,8 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 template <int NR> struct GemmCfg {
     static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
     static constexpr int kStages = NR == 16 ? 8 : 6;
-    static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536;
+    static constexpr size_t kRopeBytes = kMaxRows * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
+    static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
 
