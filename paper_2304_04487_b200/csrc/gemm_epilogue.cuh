@@ -67,6 +67,7 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int 
                                                float (*stage)[33]) {
     const int col = tile * 128 + row;
     if (col >= g.n_out) return;
+#pragma unroll 1
     for (int j = 0; j < rows_used; ++j) g.out_f32[(int64_t)j * g.ld + col] = stage[row][j];
 }
 
@@ -111,6 +112,7 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
                                                 float (*stage)[33]) {
     const int fi = row & 63, f = tile * 64 + fi;
     if (f < g.n_out) {
+#pragma unroll 1
         for (int j = row >> 6; j < rows_used; j += 2) {
             const float gate = stage[fi][j], up = stage[64 + fi][j];
             store_act(g.out_act, kActSplit, j, f, g.n_out, gate / (1.f + expf(-gate)) * up);
@@ -125,6 +127,7 @@ __device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int
     const int v = tile * 128 + row;
     const bool valid = v < g.n_out;
     const int warp = row >> 5, lane = row & 31;
+#pragma unroll 1
     for (int j = 0; j < rows_used; ++j) {
         const float a = stage[row][j];
         if (g.out_f32 && valid) g.out_f32[(int64_t)j * g.ld + v] = a;

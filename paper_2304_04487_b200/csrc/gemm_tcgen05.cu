@@ -248,10 +248,10 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[8]) {
             if (g.ss_in) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[j];
+                for (int j = 0; j < NR; ++j) stage[row][j] = acc[j] * rscale[j];
             } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
+                for (int j = 0; j < NR; ++j) stage[row][j] = acc[j];
             }
             epi_sync();
             switch (g.mode) {
