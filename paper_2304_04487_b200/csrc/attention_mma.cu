@@ -48,7 +48,7 @@ struct AttnSmem {
     static constexpr uint32_t offK = 0, offV = kTileBytes;
     static constexpr uint32_t offO = 2 * kTileBytes;                     // fp32 [16][HD] merged tile
     static constexpr uint32_t offStat = offO + 16 * HD * 4;              // m_w[4][16], l_w[4][16], misc
-    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kMaxRows * 4;  // + row positions
+    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kMaxRows * 4 + 16;  // + row positions, barriers
 };
 
 template <int HD>
@@ -74,20 +74,20 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     float* s_m = reinterpret_cast<float*>(gbase + L::offStat);   // [4][16]
     float* s_l = s_m + 64;                                        // [4][16]
     uint64_t* bar = reinterpret_cast<uint64_t*>(s_l + 64);
-    volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 1);
-    const uint32_t bar_u = smem_u32(bar);
+    volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 2);
+    const uint32_t bar_u = smem_u32(bar), bar_v = bar_u + 8;  // K tile, V tile
 
     int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);  // [32] positions of this sequence's rows
-    if (threadIdx.x == 0) { mbar_init(bar_u, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0; }
+    if (threadIdx.x == 0) { mbar_init(bar_u, 1); mbar_init(bar_v, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0; }
     if (threadIdx.x < kMaxRows) s_pos[threadIdx.x] = (int)threadIdx.x < cnt ? __ldcg(&a.rows->pos[first + threadIdx.x]) : -1;
     __syncthreads();
     if (threadIdx.x == 0) {
         const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0);
-        mbar_arrive_expect_tx(bar_u, 2 * L::kTileBytes);
-        for (int b = 0; b < L::kBoxes; ++b) {
-            tma_load_2d(base + L::offK + b * L::kBoxBytes, &map_k, bar_u, b * 64, row0);
-            tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_u, b * 64, row0);
-        }
+        // K first, on a barrier of its own: S = Q K^T and the softmax run while V is still arriving
+        mbar_arrive_expect_tx(bar_u, L::kTileBytes);
+        for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offK + b * L::kBoxBytes, &map_k, bar_u, b * 64, row0);
+        mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+        for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_v, b * 64, row0);
     }
     // Q (this head, 16 of this sequence's rows) goes straight from global memory into the MMA's
     // A-operand registers as hi / lo bf16 pairs: lane (g, t) holds rows g and g + 8, columns
@@ -185,6 +185,11 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
 
         // ---------------- O = P V ----------------------------------------------------------------
+        if (mt == 0) {
+            if (threadIdx.x == 0 && !mbar_wait(bar_v, 0)) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
+            __syncthreads();
+            if (flag[0]) return;  // uniform: the copy never landed (error word is set)
+        }
         float o[HD / 8][4];
 #pragma unroll
         for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
