@@ -136,7 +136,7 @@ __global__ void embed_kernel(ModelDims dims, const RowDesc* __restrict__ rows, c
 
 // Embedding gather for the tensor-core path, with the first RMSNorm folded in: besides x it
 // writes xs = split(x * gain) and, per 128-column tile, each row's sum of squares (the
-// projections multiply by rsqrt(mean square + eps) afterwards).  One CTA of 128 threads per row.
+// projections multiply by rsqrt(mean square + eps) afterwards).  One CTA of 128 threads per (row, 128-column tile).
 __global__ void __launch_bounds__(128) embed_norm_kernel(ModelDims dims, const RowDesc* __restrict__ rows,
                                                          const __nv_bfloat16* __restrict__ emb,
                                                          const float* __restrict__ gain, float* __restrict__ x,
@@ -144,28 +144,25 @@ __global__ void __launch_bounds__(128) embed_norm_kernel(ModelDims dims, const R
                                                          int32_t* __restrict__ dev_err) {
     pdl_trigger();
     pdl_wait();
-    const int r = blockIdx.x, d = dims.d_model;
+    const int r = blockIdx.x, t = blockIdx.y, d = dims.d_model;
     const int tok = rows->tok[r];
     const bool used = rows->pos[r] >= 0;
     const bool ok = used && tok >= 0 && tok < dims.vocab;
-    if (used && !ok && threadIdx.x == 0) atomicExch(dev_err, kDevErrToken);
+    if (used && !ok && t == 0 && threadIdx.x == 0) atomicExch(dev_err, kDevErrToken);
     const __nv_bfloat16* er = emb + (int64_t)(ok ? tok : 0) * d;
     __shared__ float red[4];
-    for (int t = 0; t * 128 < d; ++t) {
-        const int col = t * 128 + threadIdx.x;
-        float v = 0.f;
-        if (col < d) {
-            v = ok ? __bfloat162float(er[col]) : 0.f;
-            x[(int64_t)r * d + col] = v;
-            store_act(xs, kActSplit, r, col, d, v * gain[col]);
-        }
-        float sq = v * v;
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
-        __syncthreads();
-        if (threadIdx.x == 0) ss[(int64_t)t * 32 + r] = ((red[0] + red[1]) + red[2]) + red[3];
-        __syncthreads();
+    const int col = t * 128 + threadIdx.x;
+    float v = 0.f;
+    if (col < d) {
+        v = ok ? __bfloat162float(er[col]) : 0.f;
+        x[(int64_t)r * d + col] = v;
+        store_act(xs, kActSplit, r, col, d, v * gain[col]);
     }
+    float sq = v * v;
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) ss[(int64_t)t * 32 + r] = ((red[0] + red[1]) + red[2]) + red[3];
 }
 
 // --------------------------------------------------------------------------------------
@@ -227,7 +224,7 @@ void launch_embed(cudaStream_t st, const ModelDims& dims, bool bf16, const RowDe
 
 void launch_embed_norm(cudaStream_t st, const ModelDims& dims, const RowDesc* rows, const void* emb, const float* gain,
                        float* x, void* xs, float* ss, int32_t* dev_err) {
-    launch_pdl(st, true, dim3(kMaxRows), dim3(128), 0, embed_norm_kernel, dims, rows, (const __nv_bfloat16*)emb, gain, x,
+    launch_pdl(st, true, dim3(kMaxRows, (dims.d_model + 127) / 128), dim3(128), 0, embed_norm_kernel, dims, rows, (const __nv_bfloat16*)emb, gain, x,
                xs, ss, dev_err);
 }
 
