@@ -56,16 +56,10 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
                                                             const __grid_constant__ CUtensorMap map_v) {
     using L = AttnSmem<HD>;
     pdl_trigger();
-    pdl_wait();  // row descriptors, q and the K/V rows of this step come from the kernels before
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
-
-    // rows of this sequence in the step (contiguous; summarised by the planning kernel)
-    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
-    const int maxpos = __ldcg(&a.rows->seq_maxpos[seq]);
     const int c0 = chunk * kAttnChunk;
-    if (cnt == 0 || c0 > maxpos) return;  // uniform over the CTA
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -76,19 +70,36 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     uint64_t* bar = reinterpret_cast<uint64_t*>(s_l + 64);
     volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 2);
     const uint32_t bar_u = smem_u32(bar), bar_v = bar_u + 8;  // K tile, V tile
-
     int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);  // [32] positions of this sequence's rows
-    if (threadIdx.x == 0) { mbar_init(bar_u, 1); mbar_init(bar_v, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0; }
-    if (threadIdx.x < kMaxRows) s_pos[threadIdx.x] = (int)threadIdx.x < cnt ? __ldcg(&a.rows->pos[first + threadIdx.x]) : -1;
-    __syncthreads();
-    if (threadIdx.x == 0) {
+
+    auto fetch_kv = [&]() {  // one thread
         const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0);
         // K first, on a barrier of its own: S = Q K^T and the softmax run while V is still arriving
         mbar_arrive_expect_tx(bar_u, L::kTileBytes);
         for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offK + b * L::kBoxBytes, &map_k, bar_u, b * 64, row0);
         mbar_arrive_expect_tx(bar_v, L::kTileBytes);
         for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_v, b * 64, row0);
+    };
+    // A chunk that lies wholly below the length committed before this step cannot change during the step
+    // (new K/V rows go to positions at or above that length), so its tiles are requested before waiting
+    // for the QKV projection: the loads overlap that kernel's tail.
+    const bool early = a.early_kv && c0 + kAttnChunk <= __ldcg(&a.seq_state[seq].kv_len);
+    if (threadIdx.x == 0) {
+        mbar_init(bar_u, 1); mbar_init(bar_v, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0;
+        if (early) fetch_kv();
     }
+    pdl_wait();  // row descriptors, q and the K/V rows of this step come from the kernels before
+
+    // rows of this sequence in the step (contiguous; summarised by the planning kernel)
+    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
+    const int maxpos = __ldcg(&a.rows->seq_maxpos[seq]);
+    if (cnt == 0 || c0 > maxpos) {  // uniform over the CTA; tiles already requested must land before the CTA goes
+        if (early && threadIdx.x == 0) { (void)mbar_wait(bar_u, 0); (void)mbar_wait(bar_v, 0); }
+        return;
+    }
+    if (threadIdx.x < kMaxRows) s_pos[threadIdx.x] = (int)threadIdx.x < cnt ? __ldcg(&a.rows->pos[first + threadIdx.x]) : -1;
+    __syncthreads();
+    if (!early && threadIdx.x == 0) fetch_kv();
     // Q (this head, 16 of this sequence's rows) goes straight from global memory into the MMA's
     // A-operand registers as hi / lo bf16 pairs: lane (g, t) holds rows g and g + 8, columns
     // 16 ks + 2t, +1, +8, +9.  All loads are issued before any is used; rows past cnt are zero.

@@ -13,6 +13,8 @@ struct AttnArgs {
     int32_t layer;
     int32_t n_chunks;        // grid.x = ceil(max_seq / 128); CTAs past a sequence's last position exit
     const RowDesc* rows;
+    const SeqState* seq_state;  // decode steps: kv_len here is the length committed before this step
+    int32_t early_kv;        // 1: chunks wholly below that length may be fetched before the predecessor has finished
     const float* qkv;        // [32][3*H*hd] fp32, q already rotated
     void* attn_out;          // ActLayout kActSplit [64][H*hd]
     float* ws_o;             // chunk partials [seq][head][chunk][32][hd] fp32

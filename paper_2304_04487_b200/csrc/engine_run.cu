@@ -66,6 +66,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
         at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml; at.cnt = e->attn_cnt;
         at.dev_err = e->dev_err;
+        at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0;  // prompt passes: the device-side length is stale
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
