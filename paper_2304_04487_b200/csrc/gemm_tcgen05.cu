@@ -29,8 +29,9 @@ using namespace ptx;
 // Range of flat (tile, chunk) work items owned by CTA b of G.
 __device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
 
-// NR = activation rows per half (hi / lo): 16 or 32.  MMA N = 2 * NR.
-template <int NR>
+// NR = activation rows per half (hi / lo): 16 or 32.  MMA N = 2 * NR.  MODE = GemmMode: one kernel per
+// fused epilogue, so that each carries only the code it runs (the end of a launch is instruction-fetch-bound).
+template <int NR, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2) {
@@ -77,8 +78,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     }
     if (warp == 4 && lane == 0) {
         tma_prefetch_desc(&map_a0);
-        if (g.mode == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
-        if (g.mode == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
+        if (MODE == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
+        if (MODE == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
     }
     tc_fence_before();
     __syncthreads();
@@ -91,7 +92,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             auto load_a = [&](int64_t w, int s) {
                 const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
                 const uint32_t dstA = sA + s * kGemmABytes;
-                if (g.mode == kGemmSwiGLU) {
+                if (MODE == kGemmSwiGLU) {
                     tma_load_2d(dstA, &map_a0, full_bar(s), c * 64, tile * 64);
                     tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_bar(s), c * 64, tile * 64);
                 } else {
@@ -216,12 +217,12 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             for (; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * 32 + row]);
             rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
         }
-        if (g.mode == kGemmQKV) {  // the rows' positions and sequence slots, read once per CTA
+        if (MODE == kGemmQKV) {  // the rows' positions and sequence slots, read once per CTA
             if (row < 32) red_i[row] = __ldcg(&g.rows->pos[row]);
             else if (row < 64) red_i[row] = __ldcg(&g.rows->seq[row - 32]);
         }
         epi_sync();
-        if (g.mode == kGemmQKV) {
+        if (MODE == kGemmQKV) {
             // rotary factors of every row in use, once per CTA: the tile epilogues then read shared memory only
             const int half = g.dims.head_dim >> 1;
             for (int idx = row; idx < rows_used * half; idx += 128) {
@@ -237,7 +238,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         // residual rows of a tile: requested early, so their latency hides behind the accumulator wait
         // and the cross-CTA sum (only the tile's owner ever writes them, in its epilogue)
         auto prefetch_x = [&](int tile, float (&xpre)[8]) {
-            if (kPrefetchX && g.mode == kGemmResid) {
+            if (kPrefetchX && MODE == kGemmResid) {
                 const int col = tile * 128 + row;
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
@@ -254,13 +255,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 for (int j = 0; j < NR; ++j) stage[row][j] = acc[j];
             }
             epi_sync();
-            switch (g.mode) {
-                case kGemmQKV: epilogue_qkv(g, tile, row, rows_used, stage, red_i, rope_s); break;
-                case kGemmResid: epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre); break;
-                case kGemmSwiGLU: epilogue_swiglu(g, tile, row, rows_used, stage); break;
-                case kGemmStore: epilogue_store(g, tile, row, rows_used, stage); break;
-                default: epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i); break;
-            }
+            if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, rows_used, stage, red_i, rope_s);
+            else if constexpr (MODE == kGemmResid) epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre);
+            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, rows_used, stage);
+            else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, rows_used, stage);
+            else epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i);
         };
         // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks
         // its own partial (slot 0 of its workspace) and completes the tile after its last segment.  Every
@@ -334,7 +333,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc[j] = 0.f;
             const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
-            constexpr int kBatch = NR == 16 ? 4 : 2;
+            constexpr int kBatch = 2;
             for (int bb = own_first; bb < b; bb += kBatch) {  // ascending k: a fixed summation order
                 float4 p[kBatch][NR / 4];
                 bool valid;
@@ -461,12 +460,37 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+template <int NR, int MODE>
+static cudaError_t opt_in() {
+    return cudaFuncSetAttribute(gemm_ws_kernel<NR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)GemmCfg<NR>::kSmemBytes);
+}
+template <int NR>
+static cudaError_t opt_in_all() {
+    cudaError_t e;
+    if ((e = opt_in<NR, kGemmQKV>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmResid>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmSwiGLU>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmLmHead>()) != cudaSuccess) return e;
+    return opt_in<NR, kGemmStore>();
+}
+
 cudaError_t init_gemm_tcgen05() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_ws_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)GemmCfg<16>::kSmemBytes);
+    cudaError_t e = opt_in_all<16>();
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(gemm_ws_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)GemmCfg<32>::kSmemBytes);
+    return opt_in_all<32>();
+}
+
+template <int NR>
+static void launch_mode(cudaLaunchConfig_t* cfg, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
+                        const CUtensorMap& a2) {
+    switch (args.mode) {
+        case kGemmQKV: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmQKV>, args, a0, a1, a2); break;
+        case kGemmResid: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmResid>, args, a0, a1, a2); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmSwiGLU>, args, a0, a1, a2); break;
+        case kGemmLmHead: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmLmHead>, args, a0, a1, a2); break;
+        default: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmStore>, args, a0, a1, a2); break;
+    }
 }
 
 void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
@@ -481,8 +505,8 @@ void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const Gemm
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (nr == 16) cudaLaunchKernelEx(&cfg, gemm_ws_kernel<16>, args, a0, a1, a2);
-    else cudaLaunchKernelEx(&cfg, gemm_ws_kernel<32>, args, a0, a1, a2);
+    if (nr == 16) launch_mode<16>(&cfg, args, a0, a1, a2);
+    else launch_mode<32>(&cfg, args, a0, a1, a2);
 }
 
 void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
