@@ -12,6 +12,8 @@
 
 namespace llma {
 
+constexpr int kXPre = 13;  // residual epilogue: x rows 0..11 of the column, then the next norm's gain, requested early
+
 constexpr uint32_t kEpiBar = 1;  // named barrier of the 128 epilogue threads
 
 __device__ __forceinline__ void epi_sync() { ptx::named_bar_sync(kEpiBar, 128); }
@@ -24,23 +26,26 @@ __device__ __forceinline__ float warp_sum(float v) {
 // x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
 // When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
 // per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
-// With kHavePre, xpre holds x[0..7, col], read earlier by the caller.
+// With kHavePre, xpre holds x[0..11, col] and the gain, read earlier by the caller.
 template <bool kHavePre>
 __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int rows_used,
-                                               float (*stage)[33], float* red_f, const float (&xpre)[8]) {
+                                               float (*stage)[33], float* red_f, const float (&xpre)[kXPre]) {
     const int col = tile * 128 + row;
     const bool valid = col < g.n_out;
     const bool fold = g.xs_out != nullptr;
-    const float gain = (fold && valid) ? __ldg(&g.gain_next[col]) : 0.f;
+    const float gain = kHavePre ? xpre[kXPre - 1] : ((fold && valid) ? __ldg(&g.gain_next[col]) : 0.f);
     const int warp = row >> 5, lane = row & 31;
     // x is added into the staged tile with a few loads in flight; the per-row work is a rolled loop
-    for (int j0 = 0; j0 < rows_used; j0 += 8) {
+    if (kHavePre) {
+#pragma unroll
+        for (int u = 0; u < kXPre - 1; ++u)
+            if (u < rows_used) stage[row][u] += xpre[u];
+    }
+    for (int j0 = kHavePre ? kXPre - 1 : 0; j0 < rows_used; j0 += 8) {
         float xv[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (kHavePre && j0 == 0) xv[u] = xpre[u];
-            else xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
-        }
+        for (int u = 0; u < 8; ++u)
+            xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (j0 + u < rows_used) stage[row][j0 + u] += xv[u];

@@ -234,19 +234,20 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
             epi_sync();
         }
-        constexpr bool kPrefetchX = NR == 16;  // at 32 rows the extra registers spill
+        constexpr bool kPrefetchX = true;
         // residual rows of a tile: requested early, so their latency hides behind the accumulator wait
         // and the cross-CTA sum (only the tile's owner ever writes them, in its epilogue)
-        auto prefetch_x = [&](int tile, float (&xpre)[8]) {
+        auto prefetch_x = [&](int tile, float (&xpre)[kXPre]) {
             if (kPrefetchX && MODE == kGemmResid) {
                 const int col = tile * 128 + row;
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
+                for (int u = 0; u < kXPre - 1; ++u)
                     xpre[u] = (col < g.n_out && u < rows_used) ? __ldcg(&g.out_f32[(int64_t)u * g.ld + col]) : 0.f;
+                xpre[kXPre - 1] = (col < g.n_out && g.xs_out) ? __ldg(&g.gain_next[col]) : 0.f;  // the next norm's gain
             }
         };
         // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
-        auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[8]) {
+        auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[kXPre]) {
             if (g.ss_in) {
 #pragma unroll
                 for (int j = 0; j < NR; ++j) stage[row][j] = acc[j] * rscale[j];
@@ -278,7 +279,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             w += c1 - c0;
             const int buf = seg & 1;
             const uint32_t use = (uint32_t)(seg >> 1);
-            float xpre[8];
+            float xpre[kXPre];
             prefetch_x(tile, xpre);
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
@@ -327,7 +328,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             finish_tile(tile, acc, xpre);
         }
         if (own_tile >= 0 && !aborted) {
-            float xpre[8];
+            float xpre[kXPre];
             prefetch_x(own_tile, xpre);
             float acc[32];
 #pragma unroll
