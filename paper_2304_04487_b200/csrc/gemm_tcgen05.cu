@@ -347,7 +347,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                                 reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + 1) * 128 + row) * 32);
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q)
-                                if (4 * q < rows_used) p[u][q] = __ldcg(src + q);
+                                if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q);
                         }
                     }
 #pragma unroll
