@@ -166,7 +166,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         // rows of the next tile are requested before waiting for its stage to come free, so the
         // latency of the loads hides behind the MMAs of the tiles in between
         uint4 v[kUnits];
-        auto fetch = [&](int64_t it) {
+        auto fetch = [&](int64_t it, int row_limit) {
             const int c = (int)((w_beg + it) % C);
 #pragma unroll
             for (int u = 0; u < kUnits; ++u) {
@@ -174,11 +174,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const int rr = r < NR ? r : r - NR;                   // row inside its half
                 const int src_row = r < NR ? r : kMaxRows + rr;       // lo rows start at kMaxRows
                 v[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (rr < rows_used)
+                if (rr < row_limit)
                     v[u] = __ldcg(reinterpret_cast<const uint4*>(act + src_row * ld_bytes + (int64_t)c * 128 + j * 16));
             }
         };
-        if (sw < n_items) fetch(sw);
+        if (sw < n_items) fetch(sw, NR);  // every row: the count of rows in use is still on its way
         for (int64_t it = sw; it < n_items && !sh[1]; it += NW) {
             const int st = (int)(it % S);
             const uint32_t ph = (uint32_t)((it / S) & 1);
@@ -197,7 +197,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             fence_proxy_async_shared();  // make the stores visible to the tensor core's reads
             __syncwarp();
             if (lane == 0) mbar_arrive(full_bar(st));
-            if (it + NW < n_items) fetch(it + NW);
+            if (it + NW < n_items) fetch(it + NW, rows_used);
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
