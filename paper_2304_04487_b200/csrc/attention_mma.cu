@@ -225,39 +225,76 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
                 mma_bf16(o[2 * nn + 1], pl, b[2], b[3]);
             }
         }
-        // ---------------- merge the 4 warps in warp order ------------------------------------------
+        // ---------------- merge the 4 warps in warp order, chunk partial -> workspace -----------------
         if ((lane & 3) == 0) {
             s_m[warp * 16 + (lane >> 2)] = m_lo; s_m[warp * 16 + (lane >> 2) + 8] = m_hi;
             s_l[warp * 16 + (lane >> 2)] = l_lo; s_l[warp * 16 + (lane >> 2) + 8] = l_hi;
         }
-        __syncthreads();
-        float M_lo = -INFINITY, M_hi = -INFINITY;
+        const int rows_here = min(16, cnt - mt * 16);
+        if (n_mt == 1) {
+            // The K tile is dead (every warp passed the barrier after its scores): each warp parks its
+            // unscaled partial there, [warp][16 rows][HD] with the column XOR-ed by (row & 3) * 8 so that
+            // neither the stores nor the float4 reads below conflict; then all threads combine the four
+            // partials of their elements in warp order and write the chunk's partial straight to global memory.
+            float* buf = reinterpret_cast<float*>(gbase + L::offK) + warp * 16 * HD;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) { M_lo = fmaxf(M_lo, s_m[w * 16 + (lane >> 2)]); M_hi = fmaxf(M_hi, s_m[w * 16 + (lane >> 2) + 8]); }
-        const float f_lo = m_lo == -INFINITY ? 0.f : expf(m_lo - M_lo);
-        const float f_hi = m_hi == -INFINITY ? 0.f : expf(m_hi - M_hi);
-        for (int w = 0; w < 4; ++w) {
-            if (warp == w) {
-#pragma unroll
-                for (int nt = 0; nt < HD / 8; ++nt) {
-                    float* p_lo = sO + (lane >> 2) * HD + nt * 8 + 2 * (lane & 3);
-                    float* p_hi = p_lo + 8 * HD;
-                    if (w == 0) {
-                        p_lo[0] = f_lo * o[nt][0]; p_lo[1] = f_lo * o[nt][1];
-                        p_hi[0] = f_hi * o[nt][2]; p_hi[1] = f_hi * o[nt][3];
-                    } else {
-                        p_lo[0] += f_lo * o[nt][0]; p_lo[1] += f_lo * o[nt][1];
-                        p_hi[0] += f_hi * o[nt][2]; p_hi[1] += f_hi * o[nt][3];
-                    }
-                }
+            for (int nt = 0; nt < HD / 8; ++nt) {
+                const int col = nt * 8 + 2 * t4;
+                *reinterpret_cast<float2*>(buf + g8 * HD + (col ^ ((g8 & 3) << 3))) = make_float2(o[nt][0], o[nt][1]);
+                *reinterpret_cast<float2*>(buf + (g8 + 8) * HD + (col ^ ((g8 & 3) << 3))) = make_float2(o[nt][2], o[nt][3]);
             }
             __syncthreads();
-        }
-        // ---------------- chunk partial -> workspace -----------------------------------------------
-        const int rows_here = min(16, cnt - mt * 16);
-        for (int idx = threadIdx.x; idx < rows_here * HD; idx += blockDim.x) {
-            const int r = idx / HD, i = idx - r * HD;
-            a.ws_o[(part_base + mt * 16 + r) * HD + i] = sO[r * HD + i];
+            const float* all = reinterpret_cast<const float*>(gbase + L::offK);
+            for (int e = threadIdx.x; e < rows_here * (HD / 4); e += blockDim.x) {
+                const int r = e / (HD / 4), c4 = e - r * (HD / 4);
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) M = fmaxf(M, s_m[w * 16 + r]);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float mw = s_m[w * 16 + r];
+                    const float f = mw == -INFINITY ? 0.f : expf(mw - M);
+                    const float4 v = *reinterpret_cast<const float4*>(all + (w * 16 + r) * HD + ((c4 * 4) ^ ((r & 3) << 3)));
+                    if (w == 0) {
+                        acc = make_float4(__fmul_rn(f, v.x), __fmul_rn(f, v.y), __fmul_rn(f, v.z), __fmul_rn(f, v.w));
+                    } else {
+                        acc.x = __fmaf_rn(f, v.x, acc.x); acc.y = __fmaf_rn(f, v.y, acc.y);
+                        acc.z = __fmaf_rn(f, v.z, acc.z); acc.w = __fmaf_rn(f, v.w, acc.w);
+                    }
+                }
+                *reinterpret_cast<float4*>(a.ws_o + (part_base + r) * HD + c4 * 4) = acc;
+            }
+        } else {
+            // several 16-row tiles share the K and V tiles: accumulate in a buffer of its own, warp by warp
+            // (the same products and fused multiply-adds as above, so a row's bits do not depend on the path)
+            __syncthreads();
+            float M_lo = -INFINITY, M_hi = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) { M_lo = fmaxf(M_lo, s_m[w * 16 + (lane >> 2)]); M_hi = fmaxf(M_hi, s_m[w * 16 + (lane >> 2) + 8]); }
+            const float f_lo = m_lo == -INFINITY ? 0.f : expf(m_lo - M_lo);
+            const float f_hi = m_hi == -INFINITY ? 0.f : expf(m_hi - M_hi);
+            for (int w = 0; w < 4; ++w) {
+                if (warp == w) {
+#pragma unroll
+                    for (int nt = 0; nt < HD / 8; ++nt) {
+                        float* p_lo = sO + (lane >> 2) * HD + nt * 8 + 2 * (lane & 3);
+                        float* p_hi = p_lo + 8 * HD;
+                        if (w == 0) {
+                            p_lo[0] = __fmul_rn(f_lo, o[nt][0]); p_lo[1] = __fmul_rn(f_lo, o[nt][1]);
+                            p_hi[0] = __fmul_rn(f_hi, o[nt][2]); p_hi[1] = __fmul_rn(f_hi, o[nt][3]);
+                        } else {
+                            p_lo[0] = __fmaf_rn(f_lo, o[nt][0], p_lo[0]); p_lo[1] = __fmaf_rn(f_lo, o[nt][1], p_lo[1]);
+                            p_hi[0] = __fmaf_rn(f_hi, o[nt][2], p_hi[0]); p_hi[1] = __fmaf_rn(f_hi, o[nt][3], p_hi[1]);
+                        }
+                    }
+                }
+                __syncthreads();
+            }
+            for (int idx = threadIdx.x; idx < rows_here * HD; idx += blockDim.x) {
+                const int r = idx / HD, i = idx - r * HD;
+                a.ws_o[(part_base + mt * 16 + r) * HD + i] = sO[r * HD + i];
+            }
         }
         if (threadIdx.x < rows_here) {
             const int r = threadIdx.x;
