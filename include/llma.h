@@ -248,7 +248,7 @@ int llma_gemm_rows32_bf16(const void *W, const void *a, float *out, int32_t n_ou
  * no cudaMalloc, cudaFree or any other allocating routine.
  *
  * Arguments, layouts and results are exactly those of llma_gemm_rows32_bf16 (W, a, out are
- * caller-owned device buffers).  The split-k partial tiles, arrival counters and the operand
+ * caller-owned device buffers).  The partial tiles handed between CTAs, the error word and the operand
  * staging live in a fixed array of about 7 MiB that is part of the library image: every GPU
  * that loads the library holds it until the process exits.  Limits that follow from its size:
  * n_out <= 262144 and k_in <= 16384; larger sizes return LLMA_ERR_CAPACITY and do nothing.
@@ -256,7 +256,8 @@ int llma_gemm_rows32_bf16(const void *W, const void *a, float *out, int32_t n_ou
  * The first call on a device resolves the array's device address (with the caller's current
  * device) and opts the kernel into its shared-memory size; make that first call before any
  * stream capture is begun.  All calls on a device share the array and it keeps the previous
- * call's contents: the call clears what has to start at zero itself, but two calls that
+ * call's contents: the call itself puts the hand-over slots into their empty state and clears the
+ * error word, but two calls that
  * overlap on the GPU (different streams, or different threads) race on it and give wrong
  * results -- serialise them.  Synchronous.
  * Errors: NULL, ARG, CAPACITY, CONFIG (not an sm_100 device), CUDA, DEVICE_TIMEOUT.

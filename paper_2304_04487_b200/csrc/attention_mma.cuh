@@ -19,7 +19,7 @@ struct AttnArgs {
     void* attn_out;          // ActLayout kActSplit [64][H*hd]
     float* ws_o;             // chunk partials [seq][head][chunk][32][hd] fp32
     float* ws_ml;            // [seq][head][chunk][32][2] = (max, sum)
-    int32_t* cnt;            // arrival counters [seq][head], zero between launches
+    int32_t* cnt;            // (unused: the chunks are merged by a second kernel)
     int32_t* dev_err;
 };
 

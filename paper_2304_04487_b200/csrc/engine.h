@@ -42,12 +42,12 @@ struct llma_engine {
     int cur_nr = 32;                // what the launches being enqueued use
     int num_sms = 0;
     float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
-    int32_t* gemm_cnt = nullptr;    // per-tile arrival counters
+    int32_t* gemm_cnt = nullptr;    // (unused by the current kernels)
     float* norm_ss = nullptr;       // per-tile sums of squares of the residual rows [d/128][32]
     float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
     int32_t* part_idx = nullptr;
 
-    // tensor-core attention: TMA descriptors of the K/V cache, chunk partials, arrival counters
+    // tensor-core attention: TMA descriptors of the K/V cache, chunk partials
     CUtensorMap map_kcache, map_vcache;
     int attn_chunks = 0;
     float *attn_ws_o = nullptr, *attn_ws_ml = nullptr;

@@ -1,5 +1,5 @@
 // llma_gemm_rows32_bf16_noalloc: the stand-alone projection GEMM for callers that must not
-// allocate.  Its split-k partial tiles, arrival counters, error word and the 64-row operand
+// allocate.  Its partial tiles (handed between CTAs), error word and the 64-row operand
 // staging live in one file-scope __device__ array instead of cudaMalloc'ed memory.
 #include <cstring>
 #include <mutex>
@@ -69,7 +69,7 @@ extern "C" int llma_gemm_rows32_bf16_noalloc(const void* W, const void* a, float
     int grid = gemm_grid_for((int64_t)n_tiles * (k_in / 64), sms);
     if (grid > kMaxGrid) grid = kMaxGrid;
     const size_t a_bytes = (size_t)kMaxRows * k_in * sizeof(__nv_bfloat16);
-    // the array keeps the previous call's contents: counters and the error word must start at
+    // the array keeps the previous call's contents: the error word must start at
     // zero, and the low half of the operand must be zero (this entry point takes plain bf16 rows)
     CU_TRY(cudaMemsetAsync(cnt, 0, ((size_t)n_tiles + 1) * sizeof(int32_t), st));
     // the partial-tile hand-over slots must read as empty (all-ones words) when the kernel starts

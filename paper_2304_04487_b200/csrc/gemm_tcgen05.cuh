@@ -34,8 +34,8 @@ struct GemmArgs {
     int32_t tiles_per_map;  // tiles per A map
     const RowDesc* rows;    // nullptr: all 32 rows are in use
     const void* act;        // activation operand, ActLayout kActSplit [2 * kMaxRows][k_in] bf16
-    float* ws;              // partial tiles [grid][2][128][32] fp32
-    int32_t* cnt;           // arrival counters [n_tiles], zero between launches
+    float* ws;              // partial tiles [grid][2][128][32] fp32; slot 1 of every CTA all-ones (empty) at launch
+    int32_t* cnt;           // unused by the kernel (kept for the layout of callers' scratch)
     int32_t* dev_err;
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
     int32_t ld;             // leading dimension of out_f32
