@@ -173,6 +173,10 @@ static int check_device_error(llma_engine* e) {
     const int32_t code = *e->h_err;
     if (code == kDevErrNone) return LLMA_OK;
     CU_TRY(cudaMemsetAsync(e->dev_err, 0, sizeof(int32_t), e->stream));
+    // a kernel that gave up may have left partial tiles in the hand-over slots: empty them again, so that
+    // a caller who carries on after the error does not sum stale partials into later projections
+    if (code == kDevErrTimeout && e->gemm_ws)
+        CU_TRY(cudaMemsetAsync(e->gemm_ws, 0xFF, (size_t)e->num_sms * 2 * 128 * 32 * sizeof(float), e->stream));
     CU_TRY(cudaStreamSynchronize(e->stream));
     if (code == kDevErrTimeout) return LLMA_ERR_DEVICE_TIMEOUT;
     if (code == kDevErrCapacity) return LLMA_ERR_CAPACITY;
