@@ -34,6 +34,7 @@ WORKLOADS = {
     # name: (shape, prompt_len, doc_lengths, overlap, n, k, n_new)
     "llama7b-rag": ("llama7b-shape", 1536, [480, 480, 480], 0.8, 1, 8, 256),
     "llama13b-rag": ("llama13b-shape", 2048, [1024], 0.8, 1, 8, 256),
+    "llama7b-2layer-rag": ("llama7b-2layer", 1536, [480, 480, 480], 0.8, 1, 8, 256),   # small case for profiler captures
     "mid-rag": ("mid-bf16", 256, [128, 128], 0.8, 1, 8, 128),
     "tiny-fp32": ("tiny-fp32", 128, [256], 0.6, 2, 4, 64),
 }

@@ -65,6 +65,8 @@ SHAPES: Dict[str, ModelShape] = {
     # wide enough that every projection is split over several CTAs along k
     "mid-bf16": ModelShape("mid-bf16", 2, 1024, 8, 128, 2816, 8000, "bf16"),
     "llama7b-shape": ModelShape("llama7b-shape", 32, 4096, 32, 128, 11008, 32000, "bf16"),
+    # two layers at the 7B widths: the same kernels and tile shapes at a size a profiler capture can hold
+    "llama7b-2layer": ModelShape("llama7b-2layer", 2, 4096, 32, 128, 11008, 32000, "bf16"),
     "llama13b-shape": ModelShape("llama13b-shape", 40, 5120, 40, 128, 13824, 32000, "bf16"),
 }
 
