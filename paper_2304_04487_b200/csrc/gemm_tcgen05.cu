@@ -26,6 +26,12 @@ namespace llma {
 
 using namespace ptx;
 
+// Partial tiles in the workspace: [cta][slot][q][feature] float4, q = group of four activation rows.  The 32
+// features of a warp are 512 consecutive bytes, so one store or polling load of a warp touches four lines.
+__device__ __forceinline__ float4* ws_slot(float* ws, int cta, int slot, int feature) {
+    return reinterpret_cast<float4*>(ws) + ((int64_t)cta * 2 + slot) * (8 * 128) + feature;
+}
+
 // Range of flat (tile, chunk) work items owned by CTA b of G.
 __device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
 
@@ -313,10 +319,10 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
             if (w_beg > t_lo || w_end < t_hi) {  // the tile is shared with a neighbour
                 const bool owner = w_end >= t_hi;
-                float4* dst = reinterpret_cast<float4*>(g.ws + (((int64_t)b * 2 + (owner ? 0 : 1)) * 128 + row) * 32);
+                float4* dst = ws_slot(g.ws, b, owner ? 0 : 1, row);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q)  // only the columns of rows in use travel
-                    if (4 * q < rows_used) dst[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                    if (4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
                 if (owner) {
                     int b_first = (int)(t_lo * G / work);
                     while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
@@ -343,11 +349,10 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
                     for (int u = 0; u < kBatch; ++u) {
                         if (bb + u < b) {
-                            const float4* src =
-                                reinterpret_cast<const float4*>(g.ws + (((int64_t)(bb + u) * 2 + 1) * 128 + row) * 32);
+                            const float4* src = ws_slot(g.ws, bb + u, 1, row);
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q)
-                                if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q);
+                                if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q * 128);
                         }
                     }
 #pragma unroll
@@ -370,11 +375,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     if (bb + u < b) {
-                        float4* src = reinterpret_cast<float4*>(g.ws + (((int64_t)(bb + u) * 2 + 1) * 128 + row) * 32);
+                        float4* src = ws_slot(g.ws, bb + u, 1, row);
 #pragma unroll
                         for (int q = 0; q < NR / 4; ++q) {
                             if (4 * q < rows_used) {
-                                src[q] = make_float4(e, e, e, e);  // empty again for the next projection
+                                src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
                                 acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
                                 acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
                             }
@@ -383,11 +388,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 }
             }
             {   // this CTA's own partial comes last (it holds the highest k)
-                const float4* src = reinterpret_cast<const float4*>(g.ws + (((int64_t)b * 2) * 128 + row) * 32);
+                const float4* src = ws_slot(g.ws, b, 0, row);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q) {
                     if (4 * q < rows_used) {
-                        const float4 v = src[q];
+                        const float4 v = src[q * 128];
                         acc[4 * q] += v.x; acc[4 * q + 1] += v.y; acc[4 * q + 2] += v.z; acc[4 * q + 3] += v.w;
                     }
                 }
