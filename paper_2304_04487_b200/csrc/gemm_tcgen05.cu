@@ -339,6 +339,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             float acc[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            // this CTA's own partial (parked in slot 0 by these same threads) is requested now and added last
+            float4 own[NR / 4];
+            {
+                const float4* src = ws_slot(g.ws, b, 0, row);
+#pragma unroll
+                for (int q = 0; q < NR / 4; ++q)
+                    if (4 * q < rows_used) own[q] = src[q * 128];
+            }
             const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
             constexpr int kBatch = 2;
             for (int bb = own_first; bb < b; bb += kBatch) {  // ascending k: a fixed summation order
@@ -387,14 +395,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     }
                 }
             }
-            {   // this CTA's own partial comes last (it holds the highest k)
-                const float4* src = ws_slot(g.ws, b, 0, row);
+            // this CTA's own partial comes last (it holds the highest k)
 #pragma unroll
-                for (int q = 0; q < NR / 4; ++q) {
-                    if (4 * q < rows_used) {
-                        const float4 v = src[q * 128];
-                        acc[4 * q] += v.x; acc[4 * q + 1] += v.y; acc[4 * q + 2] += v.z; acc[4 * q + 3] += v.w;
-                    }
+            for (int q = 0; q < NR / 4; ++q) {
+                if (4 * q < rows_used) {
+                    acc[4 * q] += own[q].x; acc[4 * q + 1] += own[q].y; acc[4 * q + 2] += own[q].z; acc[4 * q + 3] += own[q].w;
                 }
             }
             finish_tile(own_tile, acc, xpre);
