@@ -7,7 +7,7 @@
  * tokens that follow it are copied into the decoder input and all k+1 positions are
  * evaluated in ONE causal forward pass (Eq. 3); the longest prefix of copied tokens that
  * agrees with the model's own argmax outputs is kept, plus one more output token
- * (Algorithm 1).  The result is token-for-token what greedy decoding (Eq. 2)
+ * (Algorithm 1, the acceptance loop).  The result is token-for-token what greedy decoding (Eq. 2)
  * produces.
  *
  * Every step of that path -- trigger search, copy + embedding gather, the decoder layers

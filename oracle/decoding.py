@@ -11,8 +11,9 @@ Readings of the paper taken here (each is a choice where the text is silent):
     from a decoding step and greedy takes exactly N steps (Algorithm 1 starts
     with y empty and calls the model inside the loop).
   * The trigger looks at generated tokens only; with fewer than n of them there
-    is no match (Section 2.2: "the previously generated n tokens").
-  * "Longest matching prefixes" = how far the match extends backwards, bounded
+    is no match (Section 2.2 matches the n tokens generated last).
+  * Section 2.2 prefers, among several matches, the one that agrees with the
+    generated text for longest: read as how far the match extends backwards, bounded
     by the start of the document and the start of y.
   * Ties go to the smallest flattened reference position (one valid instance of
     the paper's random tie-break; it cannot change y, only the trace).

@@ -90,7 +90,7 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     e->stream = (cudaStream_t)cuda_stream;
     e->bf16 = cfg->dtype == LLMA_DTYPE_BF16;
     const bool tc_ok = cfg->dtype == LLMA_DTYPE_BF16 && HD % 128 == 0 && cfg->d_model % 128 == 0;
-    if (cfg->gemm_impl == LLMA_GEMM_TCGEN05 && !tc_ok) return LLMA_ERR_CONFIG;
+    if (cfg->gemm_impl == LLMA_GEMM_TCGEN05 && !tc_ok) { delete e; return LLMA_ERR_CONFIG; }
     e->gemm_impl = cfg->gemm_impl == LLMA_GEMM_AUTO ? (tc_ok ? LLMA_GEMM_TCGEN05 : LLMA_GEMM_SIMT) : cfg->gemm_impl;
     ModelDims& d = e->dims;
     d.n_layers = L; d.d_model = cfg->d_model; d.n_heads = cfg->n_heads; d.head_dim = cfg->head_dim;

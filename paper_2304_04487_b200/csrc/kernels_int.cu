@@ -1,6 +1,6 @@
 // Integer side of an LLMA decoding step: trigger search + copy (Section 2.2 of the paper,
-// Algorithm 1 line 139 and the copy in line 146), embedding gather, and acceptance + K/V
-// commit (Algorithm 1).  All results here are exact integer work.
+// Algorithm 1's match and copy steps), embedding gather, and acceptance + K/V
+// commit (Algorithm 1's acceptance loop).  All results here are exact integer work.
 #include "kernels.h"
 
 namespace llma {

@@ -89,7 +89,12 @@ def step_parity(eng, oracle_model, prompt: Sequence[int], ref: Sequence[int], of
         assert got_tokens == gouts[:ga + 1], (rep.steps, got_tokens, gouts, ga)
         assert info.accepted == ga and info.emitted == ga + 1
         if got_tokens != want_tokens:
-            j = next(i for i in range(min(len(got_tokens), len(want_tokens))) if got_tokens[i] != want_tokens[i])
+            common = min(len(got_tokens), len(want_tokens))
+            diff = [i for i in range(common) if got_tokens[i] != want_tokens[i]]
+            # both sides apply Algorithm 1's acceptance rule to their own argmaxes on the same copied
+            # tokens, so two token lists that agree on their common prefix have the same length
+            assert diff, f"step {rep.steps}: equal prefixes but {len(got_tokens)} vs {len(want_tokens)} tokens"
+            j = diff[0]
             srt = np.sort(want_rows[j])
             margin = float(srt[-1] - srt[-2])
             assert margin < tie_margin, f"tokens differ at step {rep.steps} row {j} with oracle margin {margin:.3e}"
@@ -103,8 +108,3 @@ def step_parity(eng, oracle_model, prompt: Sequence[int], ref: Sequence[int], of
         rep.copied_accepted += len(got_tokens) - 1
     rep.tokens = y
     return rep
-
-
-def make_overlap_reference(y_star: Sequence[int], doc_lengths: Sequence[int], overlap: float, vocab: int, seed: int = 0):
-    from workloads import build_reference
-    return build_reference(y_star, doc_lengths, overlap, vocab, seed=seed)

@@ -120,6 +120,45 @@ def test_match_ngrams_edges():
     assert D.match_ngrams([1, 2], [0, 1, 2, 3], [0, 2, 4], 1) == (True, 3, 1)
 
 
+def test_copy_length_by_hand():
+    """k_eff = min(k, tokens left in the matched document, tokens still to emit - 1): every
+    expectation below is worked out by hand from that sentence (Section 2.2: the copied span
+    lies inside one reference document; Algorithm 1 emits exactly N tokens)."""
+    offs = [0, 6, 10]                                   # documents [0, 6) and [6, 10)
+    assert D.copy_length(4, 10, offs, 8, 100) == 2      # positions 4, 5 are left in the first document
+    assert D.copy_length(5, 10, offs, 8, 100) == 1
+    assert D.copy_length(6, 10, offs, 8, 100) == 4      # first position of the second document: 6..9
+    assert D.copy_length(9, 10, offs, 8, 100) == 1
+    assert D.copy_length(1, 10, offs, 3, 100) == 3      # k is the binding term
+    assert D.copy_length(1, 10, offs, 8, 3) == 2        # three tokens to go: one comes from the model anyway
+    assert D.copy_length(1, 10, offs, 8, 1) == 0        # last token: nothing to copy
+    assert D.copy_length(4, 10, None, 8, 100) == 6      # a single document runs to the end
+    assert D.copy_length(0, 10, [0, 0, 10], 20, 100) == 10   # an empty document in front changes nothing
+    assert D.copy_length(10, 10, offs, 8, 100) == 0     # past the end: no document holds the position
+
+
+def test_copy_stops_at_document_boundary_scripted():
+    """The reference continues with the CORRECT next tokens across a document boundary; a copy
+    that ran on into the second document would be accepted whole (and would still be lossless),
+    so only the hand-written trace below can tell the two readings apart."""
+    target = [11, 12, 13, 14, 15, 16, 17, 18, 19, 20]
+    ref = [11, 12, 13, 14] + [15, 16, 17, 18, 19, 20]   # same text, cut into two documents after 14
+    offs = [0, 4, 10]
+    res, model = scripted_run(target, ref, offs, n=1, k=8)
+    assert res.tokens == target
+    # step 1: y empty, no trigger: emits 11.  step 2: "11" matches at pos 1; three tokens (12, 13, 14)
+    # are left in document one: k_eff = 3, all accepted, plus the model's own 15.  step 3: "15" matches
+    # at pos 5 in document two; five tokens left there but only 10 - 5 - 1 = 4 may be copied: 16..19
+    # accepted, plus the model's own 20.
+    assert [(r.pos, r.k_eff, r.accepted, r.emitted) for r in res.trace] == [(-1, 0, 0, 1), (1, 3, 3, 4), (5, 4, 4, 5)]
+    assert D.simulate_decoding_sequence(target, ref, offs, 1, 8) == [(1, 1), (4, 4), (5, 5)]
+    # the model saw exactly those inputs, one position at a time, in order (prompt [7, 8, 9]: base 2)
+    assert model.calls[2:] == [(9, 2), (11, 3), (12, 4), (13, 5), (14, 6), (15, 7), (16, 8), (17, 9), (18, 10), (19, 11)]
+    # the same text as ONE document is copied straight through: 1 + min(8, 9, 8) + ... = two steps
+    res1, _ = scripted_run(target, ref, None, n=1, k=8)
+    assert [(r.pos, r.k_eff, r.accepted, r.emitted) for r in res1.trace] == [(-1, 0, 0, 1), (1, 8, 8, 9)]
+
+
 # --------------------------------------------------------------------------------------
 # P1/P2/P3/P4/P6 on scripted models (any target, any reference)
 # --------------------------------------------------------------------------------------
