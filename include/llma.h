@@ -57,15 +57,19 @@ enum { LLMA_GEMM_AUTO = 0, LLMA_GEMM_SIMT = 1, LLMA_GEMM_TCGEN05 = 2 };
 typedef struct {
     int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
     int32_t dtype;        /* storage type of weights and K/V cache: LLMA_DTYPE_* */
-    int32_t max_batch;    /* sequences held at once; max_batch * (max_k + 1) must be <= 32 */
+    int32_t max_batch;    /* sequences held at once (<= 256); max_batch * (max_k + 1) must be <= 256 */
     int32_t max_seq;      /* K/V rows per sequence */
     int32_t max_ref;      /* reference tokens per sequence */
-    int32_t max_k;        /* largest copy length k that will be requested (0..31) */
+    int32_t max_k;        /* largest copy length k that will be requested (0..255) */
     float rms_eps;        /* RMSNorm epsilon */
     float rope_theta;     /* rotary base; pairing is (i, i + head_dim/2) */
     int32_t eos_id;       /* -1: none.  Otherwise a sequence stops after emitting this id */
     int32_t gemm_impl;    /* LLMA_GEMM_*; AUTO = tensor-core kernels for bf16, SIMT for fp32 */
     int32_t keep_logits;  /* 1: keep the last step's logits for llma_debug_logits */
+    int32_t kv_proj_terms; /* tensor-core path: bf16 terms the normalised hidden state is split into for the
+                              Q/K/V projection: 2 (16 mantissa bits) or 3 (24 bits); 0 = default (3).  K/V rows
+                              are rounded to bf16 afterwards, so their pre-rounding accuracy decides how often
+                              the stored code differs from an exact computation's */
 } llma_config;
 
 /* Device pointers.  Per-layer arrays are HOST arrays of n_layers device pointers. */
@@ -108,7 +112,8 @@ typedef struct {
  * NULL for the default stream); all work of the engine is issued on it.  Allocates the K/V
  * cache ([layer][seq][head][max_seq][head_dim], zero-filled), reference storage and
  * workspaces.  Supported: head_dim 64 or 128; d_model, n_heads*head_dim and d_ffn multiples
- * of 64; max_batch*(max_k+1) <= 32.  Errors: NULL, CONFIG, CUDA.
+ * of 64; max_batch <= 256 and max_batch*(max_k+1) <= 256 rows per decoding step (the rows of a
+ * step are packed, so a sequence without a copy takes one row).  Errors: NULL, CONFIG, CUDA.
  */
 int llma_create(const llma_config *cfg, const llma_weights *w, void *cuda_stream, llma_engine **out);
 
@@ -117,7 +122,8 @@ int llma_destroy(llma_engine *e);
 
 /*
  * Load a prompt x (host, n_prompt >= 1 tokens) into sequence slot `seq`: positions
- * 0..n_prompt-2 are pushed through the decoder and cached; the last prompt token becomes
+ * 0..n_prompt-2 are pushed through the decoder (128 positions per pass on the tensor-core path) and
+ * cached; the last prompt token becomes
  * the pending input of the first decoding step (Algorithm 1 starts with y empty and calls
  * the model inside its loop, so prefill emits nothing).  Clears the sequence's output and
  * statistics; keeps its reference.  Synchronous.  Errors: NULL, CAPACITY, TOKEN_RANGE, CUDA.
@@ -184,18 +190,40 @@ int llma_debug_logits(llma_engine *e, float *out);
 int llma_debug_kv_row(llma_engine *e, int32_t layer, int32_t seq, int32_t pos, int32_t which, float *out);
 
 /* Parity harness only: copy an internal activation buffer of the last forward pass to `out` (host,
- * fp32).  which = 0: residual stream x [32][d_model]; 1: qkv [32][3*n_heads*head_dim] (q rotated; the
- * k and v thirds are only filled on the CUDA-core path); 2: attention output [32][n_heads*head_dim];
- * 3: gated FFN activation h [32][d_ffn].  Split bf16 buffers are returned as hi + lo.  `count` must be
- * the buffer's element count.  Errors: NULL, ARG, CUDA. */
+ * fp32), rc = llma_row_capacity rows (row r = packed row r of the step).  which = 0: residual stream
+ * x [rc][d_model]; 1: qkv [rc][3*n_heads*head_dim] (q rotated; the k and v thirds are only filled on the
+ * CUDA-core path); 2: attention output [rc][n_heads*head_dim]; 3: gated FFN activation h [rc][d_ffn].
+ * Split bf16 buffers are returned as hi + lo.  `count` must be the buffer's element count.
+ * Errors: NULL, ARG, CUDA. */
 int llma_debug_buffer(llma_engine *e, int32_t which, float *out, int64_t count);
+
+/*
+ * Replay of a given step sequence for one sequence slot, as the paper times its method (Section 3.2,
+ * "target guided simulation", Algorithm 2): step i feeds trace[2i] >= 1 input rows (the pending token and
+ * the next trace[2i]-1 tokens of `target`) through the real forward pass and then appends trace[2i+1]
+ * tokens of `target` (1 <= trace[2i+1] <= trace[2i] <= max_k+1), whatever the model's own outputs are.
+ * trace (host, [n_steps][2]); target (host, n_target ids) is the text to reproduce; the trace's emitted
+ * counts must sum to n_target.  Every other sequence must be idle or finished.  Output tokens are the
+ * target's; stats (may be NULL) carry steps, launches and device time.
+ * Errors: NULL, ARG, CAPACITY, TOKEN_RANGE, STATE, CUDA, DEVICE_TIMEOUT.
+ */
+int llma_generate_forced(llma_engine *e, int32_t seq, const int32_t *trace, int32_t n_steps,
+                         const int32_t *target, int32_t n_target, llma_stats *stats);
+
+/* Parity harness only: preset the device-side error word (0 none, 1 a bounded wait ran out, 2 capacity,
+ * 3 token range), as a kernel that gave up would have left it; the next step reports it.  Errors: ARG, CUDA. */
+int llma_debug_set_device_error(llma_engine *e, int32_t code);
+
+/* Rows the engine's activation buffers hold (the leading dimension of llma_debug_buffer), or a negative
+ * status. */
+int llma_row_capacity(llma_engine *e);
 
 /* Committed K/V length of a sequence (prompt rows + emitted tokens - 1), or a negative status. */
 int llma_kv_len(llma_engine *e, int32_t seq);
 
 /* Kernel classes reported by llma_profile_steps. */
 enum {
-    LLMA_K_PLAN = 0,      /* trigger search + copy planning */
+    LLMA_K_PLAN = 0,      /* trigger search + copy planning (the step-tail kernel launched for the plan alone) */
     LLMA_K_EMBED,         /* embedding gather */
     LLMA_K_NORM,          /* RMSNorm */
     LLMA_K_GEMM_QKV,      /* QKV projection (tensor-core path: + rotary + K/V append) */
@@ -204,8 +232,8 @@ enum {
     LLMA_K_GEMM_GATEUP,   /* gate/up projections (tensor-core path: + SiLU gating) */
     LLMA_K_GEMM_DOWN,     /* down projection + residual */
     LLMA_K_GEMM_LMHEAD,   /* LM head (tensor-core path: + per-tile argmax) */
-    LLMA_K_ARGMAX,        /* final per-row argmax */
-    LLMA_K_ACCEPT,        /* acceptance + K/V commit */
+    LLMA_K_ARGMAX,        /* final per-row argmax (CUDA-core path; folded into ACCEPT on the tensor-core path) */
+    LLMA_K_ACCEPT,        /* final argmax + acceptance + K/V commit (+ the next step's plan inside llma_generate) */
     LLMA_K_EPILOGUE,      /* separate rotary / gating kernels of the SIMT path */
     LLMA_K_COUNT
 };

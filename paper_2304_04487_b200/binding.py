@@ -17,7 +17,7 @@ class LlmaConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab", "dtype",
                                          "max_batch", "max_seq", "max_ref", "max_k")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("eos_id", C.c_int32),
-                ("gemm_impl", C.c_int32), ("keep_logits", C.c_int32)]
+                ("gemm_impl", C.c_int32), ("keep_logits", C.c_int32), ("kv_proj_terms", C.c_int32)]
 
 
 class LlmaWeights(C.Structure):
@@ -56,7 +56,9 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_gemm_rows32_bf16_noalloc", "llma_last_cuda_error", "llma_strerror")
+           "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16",
+           "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity",
+           "llma_last_cuda_error", "llma_strerror")
 
 
 def lib() -> C.CDLL:
@@ -81,6 +83,9 @@ def lib() -> C.CDLL:
         L.llma_debug_kv_row.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_float)]
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
+        L.llma_row_capacity.argtypes = [vp]
+        L.llma_debug_set_device_error.argtypes = [vp, i32]
+        L.llma_generate_forced.argtypes = [vp, i32, pi32, i32, pi32, i32, C.POINTER(LlmaStats)]
         L.llma_debug_buffer.argtypes = [vp, i32, C.POINTER(C.c_float), C.c_int64]
         L.llma_gemm_rows32_bf16.argtypes = [vp, vp, vp, i32, i32, vp]
         L.llma_gemm_rows32_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, vp]
@@ -137,7 +142,7 @@ class Engine:
 
     def __init__(self, shape, weights: Dict[str, np.ndarray], max_seq: int, max_ref: int, max_k: int,
                  max_batch: int = 1, eos_id: int = -1, gemm_impl: int = LLMA_GEMM_AUTO, keep_logits: bool = False,
-                 device: str = "cuda:0", stream=None, share_weights_with: "Engine" = None):
+                 device: str = "cuda:0", stream=None, share_weights_with: "Engine" = None, kv_proj_terms: int = 0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the LLMA engine has no CPU path")
@@ -174,7 +179,7 @@ class Engine:
                         arr_of("w_down"))
         self.cfg = LlmaConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                               LLMA_DTYPE_BF16 if bf16 else LLMA_DTYPE_F32, max_batch, max_seq, max_ref, max_k,
-                              shape.rms_eps, shape.rope_theta, eos_id, gemm_impl, int(keep_logits))
+                              shape.rms_eps, shape.rope_theta, eos_id, gemm_impl, int(keep_logits), kv_proj_terms)
         self._stream = stream if stream is not None else torch.cuda.Stream(self.device)
         h = C.c_void_p()
         torch.cuda.synchronize(self.device)
@@ -244,7 +249,7 @@ class Engine:
     def llma_debug_buffer(self, which: int) -> np.ndarray:
         sh = self.shape
         cols = (sh.d_model, 3 * sh.n_heads * sh.head_dim, sh.n_heads * sh.head_dim, sh.d_ffn)[which]
-        out = np.empty((32, cols), np.float32)
+        out = np.empty((self.llma_row_capacity(), cols), np.float32)
         self._check(lib().llma_debug_buffer(self._h, which, out.ctypes.data_as(C.POINTER(C.c_float)), out.size),
                     "llma_debug_buffer")
         return out
@@ -259,6 +264,21 @@ class Engine:
                for i, name in enumerate(K_NAMES) if pr.launches[i]}
         out["_total"] = {"ms_per_step": pr.total_ms / pr.steps, "launches_per_step": float(sum(pr.launches)) / pr.steps}
         return out
+
+    def llma_row_capacity(self) -> int:
+        return self._check(lib().llma_row_capacity(self._h), "llma_row_capacity")
+
+    def llma_debug_set_device_error(self, code: int) -> None:
+        self._check(lib().llma_debug_set_device_error(self._h, code), "llma_debug_set_device_error")
+
+    def llma_generate_forced(self, seq: int, trace: Sequence[Tuple[int, int]], target: Sequence[int]) -> LlmaStats:
+        """trace: (input rows, emitted tokens) per step, as Algorithm 2 produces them; target: the text."""
+        t = _i32(np.asarray(trace, np.int32).reshape(-1, 2))
+        g = _i32(target)
+        st = LlmaStats()
+        self._check(lib().llma_generate_forced(self._h, seq, _pi32(t), len(t), _pi32(g), len(g), C.byref(st)),
+                    "llma_generate_forced")
+        return st
 
     def llma_gemm_impl(self) -> int:
         return self._check(lib().llma_gemm_impl(self._h), "llma_gemm_impl")

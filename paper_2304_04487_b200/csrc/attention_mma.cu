@@ -48,7 +48,7 @@ struct AttnSmem {
     static constexpr uint32_t offK = 0, offV = kTileBytes;
     static constexpr uint32_t offO = 2 * kTileBytes;                     // fp32 [16][HD] merged tile
     static constexpr uint32_t offStat = offO + 16 * HD * 4;              // m_w[4][16], l_w[4][16], misc
-    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kMaxRows * 4 + 16;  // + row positions, barriers
+    static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kRowCap * 4 + 16;  // + row positions, barriers
 };
 
 template <int HD>
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     uint64_t* bar = reinterpret_cast<uint64_t*>(s_l + 64);
     volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 2);
     const uint32_t bar_u = smem_u32(bar), bar_v = bar_u + 8;  // K tile, V tile
-    int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);  // [32] positions of this sequence's rows
+    int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);  // positions of this sequence's rows
 
     auto fetch_kv = [&]() {  // one thread
         const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0);
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
         if (early && threadIdx.x == 0) { (void)mbar_wait(bar_u, 0); (void)mbar_wait(bar_v, 0); }
         return;
     }
-    if (threadIdx.x < kMaxRows) s_pos[threadIdx.x] = (int)threadIdx.x < cnt ? __ldcg(&a.rows->pos[first + threadIdx.x]) : -1;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) s_pos[i] = __ldcg(&a.rows->pos[first + i]);
     __syncthreads();
     if (!early && threadIdx.x == 0) fetch_kv();
     // Q (this head, 16 of this sequence's rows) goes straight from global memory into the MMA's
@@ -136,7 +136,8 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     const float scale = rsqrtf((float)HD);
     const int n_mt = (cnt + 15) >> 4;
     const int wpos0 = warp * 32;  // this warp's positions inside the chunk
-    const int64_t part_base = (((int64_t)seq * d.n_heads + head) * a.n_chunks + chunk) * kMaxRows;
+    // chunk partials are indexed by the row's slot in the step: [head][chunk][row][HD]
+    const int64_t part_base = ((int64_t)head * a.n_chunks + chunk) * d.row_cap + first;
 
     for (int mt = 0; mt < n_mt; ++mt) {
         if (mt > 0) load_q(mt);
@@ -312,7 +313,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     }
 }
 
-// Second pass: one warp per (sequence, head, row) combines the row's chunk partials in ascending chunk
+// Second pass: one warp per (head, row) combines the row's chunk partials in ascending chunk
 // order.  A kernel of its own, so that every head is merged at once instead of by whichever CTA of the
 // head happened to finish last; a row's result still depends on its own position only.
 template <int HD>
@@ -320,19 +321,20 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
     pdl_trigger();
     pdl_wait();
     extern __shared__ float s_w[];  // [4 warps][n_chunks] weights, then [4][n_chunks] weighted sums
-    const int head = blockIdx.x, seq = blockIdx.z;
+    const int head = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
-    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
-    const int r = blockIdx.y * 4 + warp;
-    if (r >= cnt) return;
-    const int nc = __ldcg(&a.rows->pos[first + r]) / kAttnChunk + 1;
-    const int64_t head_base = ((int64_t)seq * d.n_heads + head) * a.n_chunks * kMaxRows;
+    const int r = blockIdx.y * 4 + warp;  // row slot of the step
+    if (r >= __ldcg(&a.rows->rows_used)) return;
+    const int pos = __ldcg(&a.rows->pos[r]);
+    if (pos < 0) return;
+    const int nc = pos / kAttnChunk + 1;
+    const int64_t head_base = (int64_t)head * a.n_chunks * d.row_cap;
     float* w_c = s_w + warp * a.n_chunks;
     float* wl_c = s_w + (4 + warp) * a.n_chunks;
     float M = -INFINITY;
     for (int c = lane; c < nc; c += 32) {
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * kMaxRows + r);
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * d.row_cap + r);
         w_c[c] = ml.x; wl_c[c] = ml.y;
         M = fmaxf(M, ml.x);
     }
@@ -353,7 +355,7 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
             float4 p[16];
 #pragma unroll
             for (int u = 0; u < 16; ++u)
-                if (c + u < nc) p[u] = __ldcg(src + (int64_t)(c + u) * kMaxRows * (HD / 4));
+                if (c + u < nc) p[u] = __ldcg(src + (int64_t)(c + u) * d.row_cap * (HD / 4));
 #pragma unroll
             for (int u = 0; u < 16; ++u) {
                 if (c + u < nc) {
@@ -363,10 +365,10 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
             }
         }
         const int64_t col = (int64_t)head * HD + lane * 4;
-        store_act(a.attn_out, kActSplit, first + r, col, d.hd_total, num.x / den);
-        store_act(a.attn_out, kActSplit, first + r, col + 1, d.hd_total, num.y / den);
-        store_act(a.attn_out, kActSplit, first + r, col + 2, d.hd_total, num.z / den);
-        store_act(a.attn_out, kActSplit, first + r, col + 3, d.hd_total, num.w / den);
+        store_act(a.attn_out, kActSplit, d.row_cap, r, col, d.hd_total, num.x / den);
+        store_act(a.attn_out, kActSplit, d.row_cap, r, col + 1, d.hd_total, num.y / den);
+        store_act(a.attn_out, kActSplit, d.row_cap, r, col + 2, d.hd_total, num.z / den);
+        store_act(a.attn_out, kActSplit, d.row_cap, r, col + 3, d.hd_total, num.w / den);
     }
 }
 
@@ -382,7 +384,7 @@ cudaError_t init_attention_mma() {
 
 void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap& map_k, const CUtensorMap& map_v) {
     dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
-    dim3 mgrid(a.dims.n_heads, kMaxRows / 4, a.dims.max_batch);
+    dim3 mgrid(a.dims.n_heads, (a.n_rows + 3) / 4);
     const size_t msmem = (size_t)8 * a.n_chunks * sizeof(float);
     if (a.dims.head_dim == 128) {
         launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128>, a, map_k, map_v);

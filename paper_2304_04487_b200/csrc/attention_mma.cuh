@@ -15,11 +15,11 @@ struct AttnArgs {
     const RowDesc* rows;
     const SeqState* seq_state;  // decode steps: kv_len here is the length committed before this step
     int32_t early_kv;        // 1: chunks wholly below that length may be fetched before the predecessor has finished
-    const float* qkv;        // [32][3*H*hd] fp32, q already rotated
-    void* attn_out;          // ActLayout kActSplit [64][H*hd]
-    float* ws_o;             // chunk partials [seq][head][chunk][32][hd] fp32
-    float* ws_ml;            // [seq][head][chunk][32][2] = (max, sum)
-    int32_t* cnt;            // (unused: the chunks are merged by a second kernel)
+    int32_t n_rows;          // row slots of this pass (grid of the merge kernel)
+    const float* qkv;        // [rows][3*H*hd] fp32, q already rotated
+    void* attn_out;          // ActLayout kActSplit [2 rc][H*hd]
+    float* ws_o;             // chunk partials [head][chunk][rc][hd] fp32
+    float* ws_ml;            // [head][chunk][rc][2] = (max, sum)
     int32_t* dev_err;
 };
 

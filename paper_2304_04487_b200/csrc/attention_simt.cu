@@ -94,22 +94,23 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(ModelDims dims, int
             for (int e = 0; e < EPL; ++e) num[e] += f * sacc[w][lane * EPL + e];
         }
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) store_act(attn_out, act_layout, r, head * hd + lane * EPL + e, HD, num[e] / den);
+        for (int e = 0; e < EPL; ++e) store_act(attn_out, act_layout, dims.row_cap, r, head * hd + lane * EPL + e, HD, num[e] / den);
     }
 }
 
-void launch_qkv_post(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, const RowDesc* rows, float* qkv,
-                     const float* rope_cos, const float* rope_sin, void* kcache, void* vcache) {
-    dim3 grid(kMaxRows, dims.n_heads);
+void launch_qkv_post(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, int n_rows, const RowDesc* rows,
+                     float* qkv, const float* rope_cos, const float* rope_sin, void* kcache, void* vcache) {
+    dim3 grid(n_rows, dims.n_heads);
     if (bf16)
         launch_pdl(st, true, grid, dim3(64), 0, qkv_post_kernel<__nv_bfloat16>, dims, layer, rows, qkv, rope_cos, rope_sin, (__nv_bfloat16*)kcache, (__nv_bfloat16*)vcache);
     else
         launch_pdl(st, true, grid, dim3(64), 0, qkv_post_kernel<float>, dims, layer, rows, qkv, rope_cos, rope_sin, (float*)kcache, (float*)vcache);
 }
 
-void launch_attention_simt(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, const RowDesc* rows,
-                           const float* qkv, const void* kcache, const void* vcache, void* attn_out, int act_layout) {
-    dim3 grid(dims.n_heads, kMaxRows);
+void launch_attention_simt(cudaStream_t st, bool bf16, const ModelDims& dims, int layer, int n_rows,
+                           const RowDesc* rows, const float* qkv, const void* kcache, const void* vcache,
+                           void* attn_out, int act_layout) {
+    dim3 grid(dims.n_heads, n_rows);
     const bool hd128 = dims.head_dim == 128;
     if (bf16) {
         auto K = (const __nv_bfloat16*)kcache; auto V = (const __nv_bfloat16*)vcache;

@@ -6,7 +6,8 @@
 
 namespace llma {
 
-constexpr int kMaxRows = 32;  // query rows of one forward pass (all sequences together)
+constexpr int kRowCap = 256;  // most query rows one forward pass can hold (all sequences together)
+constexpr int kSeqCap = 256;  // most sequence slots of an engine
 
 // Per-sequence decoding state, resident in device memory.  Field order is mirrored by the
 // host when it reads the array back.
@@ -20,21 +21,25 @@ struct SeqState {
     int32_t ref_len;     // reference tokens stored for this sequence
     int32_t prompt_len;
     int32_t pos, k_eff, nrows;  // plan of the step in flight
+    int32_t forced_rows, forced_emit;  // replay of a given step shape (0 = decide as Algorithm 1 does)
+    int32_t trace_step;                // replay: index of the next step in the trace
     int32_t last_pos, last_k_eff, last_accepted, last_emitted;
     int32_t steps, trigger_steps, copied_accepted;
 };
 
-// One forward pass works on up to kMaxRows rows; these arrays say what each row is.
+// One forward pass works on up to kRowCap rows; these arrays say what each row is.  The rows of
+// the sequences that take part are packed: sequence s owns rows seq_first[s] .. +seq_cnt[s]-1
+// and rows_used is the total, so a sequence without a copy adds one row, not k+1.
 struct RowDesc {
-    int32_t tok[kMaxRows];  // input token id
-    int32_t pos[kMaxRows];  // absolute position in its sequence, -1 = row unused
-    int32_t seq[kMaxRows];  // sequence slot
-    int32_t rows_used;      // 1 + highest used row index (0 = nothing to do)
-    // per sequence slot: its rows are contiguous -- first row, row count (0 = none) and highest position
-    int32_t seq_first[kMaxRows];
-    int32_t seq_cnt[kMaxRows];
-    int32_t seq_maxpos[kMaxRows];
-    int32_t max_pos;        // highest position among used rows (-1 if none)
+    int32_t tok[kRowCap];  // input token id
+    int32_t pos[kRowCap];  // absolute position in its sequence, -1 = row unused
+    int32_t seq[kRowCap];  // sequence slot
+    int32_t rows_used;     // number of rows in use (0 = nothing to do); they are rows 0 .. rows_used-1
+    // per sequence slot: first row, row count (0 = none) and highest position
+    int32_t seq_first[kSeqCap];
+    int32_t seq_cnt[kSeqCap];
+    int32_t seq_maxpos[kSeqCap];
+    int32_t max_pos;       // highest position among used rows (-1 if none)
 };
 
 enum : int32_t {
@@ -47,7 +52,8 @@ enum : int32_t {
 struct ModelDims {
     int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
     int32_t hd_total;  // n_heads * head_dim
-    int32_t max_batch, max_seq, max_ref, kp1;  // kp1 = max_k + 1 rows reserved per sequence
+    int32_t max_batch, max_seq, max_ref, kp1;  // kp1 = max_k + 1 = most rows of one sequence in a decoding step
+    int32_t row_cap;   // rows the activation buffers hold (multiple of 16, <= kRowCap)
     float rms_eps;
     int32_t eos_id;
 };
@@ -59,21 +65,26 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-// Activations that feed a projection are kept in one of two layouts:
-//   kActF32   fp32 [kMaxRows][K]                       (CUDA-core GEMM)
-//   kActSplit bf16 [2*kMaxRows][K]: row r holds hi = bf16(v), row kMaxRows + r holds
-//             lo = bf16(v - hi), so hi + lo carries 16 mantissa bits through a bf16 tensor-core
-//             product (the two halves are summed in the GEMM's fp32 accumulator epilogue)
-enum ActLayout : int32_t { kActF32 = 0, kActSplit = 1 };
+// Activations that feed a projection are kept in one of these layouts (rc = the engine's row capacity):
+//   kActF32    fp32 [rc][K]                         (CUDA-core GEMM)
+//   kActSplit  bf16 [2 rc][K]: row r holds hi = bf16(v), row rc + r holds lo = bf16(v - hi), so
+//              hi + lo carries 16 mantissa bits through a bf16 tensor-core product (both halves
+//              are accumulated into the same fp32 accumulator)
+//   kActSplit3 bf16 [3 rc][K]: a third term lo2 = bf16(v - hi - lo) in row 2 rc + r, 24 mantissa
+//              bits in all (used where the product is rounded to bf16 afterwards: the K/V rows)
+enum ActLayout : int32_t { kActF32 = 0, kActSplit = 1, kActSplit3 = 2 };
 
-__device__ __forceinline__ void store_act(void* buf, int layout, int r, int64_t i, int64_t K, float v) {
+__device__ __forceinline__ void store_act(void* buf, int layout, int rc, int r, int64_t i, int64_t K, float v) {
     if (layout == kActF32) {
         reinterpret_cast<float*>(buf)[(int64_t)r * K + i] = v;
     } else {
         __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(buf);
         const __nv_bfloat16 hi = __float2bfloat16_rn(v);
         b[(int64_t)r * K + i] = hi;
-        b[(int64_t)(kMaxRows + r) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        const float rest = v - __bfloat162float(hi);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(rest);
+        b[(int64_t)(rc + r) * K + i] = lo;
+        if (layout == kActSplit3) b[(int64_t)(2 * rc + r) * K + i] = __float2bfloat16_rn(rest - __bfloat162float(lo));
     }
 }
 

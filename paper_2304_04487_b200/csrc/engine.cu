@@ -50,8 +50,8 @@ static void free_engine(llma_engine* e) {
     cudaFree(e->y); cudaFree(e->out_tok); cudaFree(e->dev_err); cudaFree(e->x); cudaFree(e->qkv);
     cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
     cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
-    cudaFree(e->attn_ws_o); cudaFree(e->attn_ws_ml); cudaFree(e->attn_cnt);
-    cudaFree(e->gemm_ws); cudaFree(e->gemm_cnt); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss);
+    cudaFree(e->attn_ws_o); cudaFree(e->attn_ws_ml); cudaFree(e->trace); cudaFree(e->target);
+    cudaFree(e->gemm_ws); cudaFree(e->gemm_ws_wide); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss);
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
     if (e->h_err) cudaFreeHost(e->h_err);
@@ -70,7 +70,10 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     const int HD = cfg->n_heads * cfg->head_dim;
     if (cfg->d_model % 64 || HD % 64 || cfg->d_ffn % 64) return LLMA_ERR_CONFIG;
     if (cfg->dtype != LLMA_DTYPE_F32 && cfg->dtype != LLMA_DTYPE_BF16) return LLMA_ERR_CONFIG;
-    if (cfg->max_batch < 1 || cfg->max_k < 0 || cfg->max_batch * (cfg->max_k + 1) > kMaxRows) return LLMA_ERR_CONFIG;
+    if (cfg->max_batch < 1 || cfg->max_batch > kSeqCap || cfg->max_k < 0 ||
+        (int64_t)cfg->max_batch * (cfg->max_k + 1) > kRowCap)
+        return LLMA_ERR_CONFIG;
+    if (cfg->kv_proj_terms != 0 && cfg->kv_proj_terms != 2 && cfg->kv_proj_terms != 3) return LLMA_ERR_CONFIG;
     if (cfg->max_seq < 2 || cfg->max_ref < 0 || !(cfg->rms_eps >= 0.f) || !(cfg->rope_theta > 0.f)) return LLMA_ERR_CONFIG;
     if (cfg->gemm_impl < LLMA_GEMM_AUTO || cfg->gemm_impl > LLMA_GEMM_TCGEN05) return LLMA_ERR_CONFIG;
     if (!w->tok_emb || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
@@ -97,6 +100,14 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     d.d_ffn = cfg->d_ffn; d.vocab = cfg->vocab; d.hd_total = HD; d.max_batch = cfg->max_batch;
     d.max_seq = cfg->max_seq; d.max_ref = cfg->max_ref > 0 ? cfg->max_ref : 1; d.kp1 = cfg->max_k + 1;
     d.rms_eps = cfg->rms_eps; d.eos_id = cfg->eos_id;
+    // Row capacities.  Decoding steps hold at most max_batch * (max_k + 1) rows; prompt passes push up to
+    // prefill_rows consecutive positions of one sequence through the same kernels (128 on the tensor-core
+    // path, where the projections are compute-bound from about a hundred rows on).
+    e->decode_rows = (d.max_batch * d.kp1 + 15) / 16 * 16;
+    e->prefill_rows = std::max(e->decode_rows, e->gemm_impl == LLMA_GEMM_TCGEN05 ? 128 : 32);
+    e->row_cap = e->prefill_rows;
+    d.row_cap = e->row_cap;
+    e->qkv_terms = cfg->kv_proj_terms == 0 ? 3 : cfg->kv_proj_terms;
     e->tok_emb = w->tok_emb; e->lm_head = w->lm_head; e->final_norm = w->final_norm;
     for (int l = 0; l < L; ++l) {
         e->attn_norm.push_back(w->attn_norm[l]); e->ffn_norm.push_back(w->ffn_norm[l]);
@@ -123,16 +134,21 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     CREATE_TRY(dalloc(&e->doc_start, B * d.max_ref));
     CREATE_TRY(dalloc(&e->doc_end, B * d.max_ref));
     CREATE_TRY(dalloc(&e->y, B * e->y_cap));
-    CREATE_TRY(dalloc(&e->out_tok, (size_t)kMaxRows));
+    const size_t RC = (size_t)e->row_cap;
+    CREATE_TRY(dalloc(&e->out_tok, RC));
+    e->trace_cap = e->y_cap;
+    CREATE_TRY(dalloc(&e->trace, B * e->trace_cap * 2));
+    CREATE_TRY(dalloc(&e->target, B * e->y_cap));
     CREATE_TRY(dalloc(&e->dev_err, 1));
-    CREATE_TRY(dalloc(&e->x, (size_t)kMaxRows * d.d_model));
-    CREATE_TRY(dalloc(&e->qkv, (size_t)kMaxRows * 3 * HD));
-    CREATE_TRY(dalloc(&e->gate_up, (size_t)kMaxRows * 2 * d.d_ffn));
-    CREATE_TRY(dalloc(&e->logits, (size_t)kMaxRows * d.vocab));
-    // activation operands: fp32 [32][K] (CUDA-core GEMM) or split bf16 [64][K] (tensor cores): 4 bytes each
-    CREATE_TRY(dalloc((char**)&e->x_hat, (size_t)kMaxRows * d.d_model * 4));
-    CREATE_TRY(dalloc((char**)&e->attn, (size_t)kMaxRows * HD * 4));
-    CREATE_TRY(dalloc((char**)&e->h, (size_t)kMaxRows * d.d_ffn * 4));
+    CREATE_TRY(dalloc(&e->x, RC * d.d_model));
+    CREATE_TRY(dalloc(&e->qkv, RC * 3 * HD));
+    if (e->gemm_impl != LLMA_GEMM_TCGEN05) CREATE_TRY(dalloc(&e->gate_up, RC * 2 * d.d_ffn));
+    if (e->gemm_impl != LLMA_GEMM_TCGEN05 || cfg->keep_logits) CREATE_TRY(dalloc(&e->logits, RC * d.vocab));
+    // activation operands: fp32 [rc][K] (CUDA-core GEMM) or split bf16 [2 rc][K] (tensor cores): 4 bytes per
+    // element; x_hat carries a third bf16 term when the QKV projection multiplies three
+    CREATE_TRY(dalloc((char**)&e->x_hat, RC * d.d_model * 6));
+    CREATE_TRY(dalloc((char**)&e->attn, RC * HD * 4));
+    CREATE_TRY(dalloc((char**)&e->h, RC * d.d_ffn * 4));
     const size_t kv_elems = (size_t)L * B * d.n_heads * d.max_seq * d.head_dim;
     CREATE_TRY(dalloc((char**)&e->kcache, kv_elems * es));
     CREATE_TRY(dalloc((char**)&e->vcache, kv_elems * es));
@@ -160,14 +176,16 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         if (prop.major != 10) { free_engine(e); return LLMA_ERR_CONFIG; }  // tcgen05 needs sm_100
         e->num_sms = prop.multiProcessorCount;
         const int vt = (d.vocab + 127) / 128;
-        const int max_tiles = std::max(std::max(vt, 3 * HD / 128), std::max((d.d_ffn + 63) / 64, (d.d_model + 127) / 128));
-        CREATE_TRY(dalloc(&e->gemm_ws, (size_t)e->num_sms * 2 * 128 * 32));
         // hand-over slots start out empty: every word the all-ones pattern (see gemm_ws_kernel)
-        if (cudaMemset(e->gemm_ws, 0xFF, (size_t)e->num_sms * 2 * 128 * 32 * sizeof(float)) != cudaSuccess) { free_engine(e); return LLMA_ERR_CUDA; }
-        CREATE_TRY(dalloc(&e->gemm_cnt, (size_t)max_tiles));
-        CREATE_TRY(dalloc(&e->part_max, (size_t)vt * 32));
-        CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * 32));
-        CREATE_TRY(dalloc(&e->norm_ss, (size_t)((d.d_model + 127) / 128) * 32));
+        e->gemm_ws_bytes = (size_t)e->num_sms * 2 * 128 * 32 * sizeof(float);
+        CREATE_TRY(dalloc((char**)&e->gemm_ws, e->gemm_ws_bytes, false));
+        CREATE_TRY(cudaMemset(e->gemm_ws, 0xFF, e->gemm_ws_bytes));
+        e->gemm_ws_wide_bytes = (size_t)e->num_sms * 2 * 128 * RC * sizeof(float);
+        CREATE_TRY(dalloc((char**)&e->gemm_ws_wide, e->gemm_ws_wide_bytes, false));
+        CREATE_TRY(cudaMemset(e->gemm_ws_wide, 0xFF, e->gemm_ws_wide_bytes));
+        CREATE_TRY(dalloc(&e->part_max, (size_t)vt * RC));
+        CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * RC));
+        CREATE_TRY(dalloc(&e->norm_ss, (size_t)((d.d_model + 127) / 128) * RC));
         e->maps.resize(L);
         int bad = 0;
         for (int l = 0; l < L; ++l) {
@@ -182,19 +200,25 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         }
         bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
         // the MMA shape of decoding steps is fixed per engine (by its row capacity), never per step
-        e->decode_nr = d.max_batch * d.kp1 <= 16 ? 16 : 32;
+        e->decode_wide = e->decode_rows > 32;
+        e->decode_nr = e->decode_wide ? e->decode_rows : (e->decode_rows <= 16 ? 16 : 32);
+        // activation operands of the wide kernel: one box of nr rows per (buffer, use)
+        auto act_maps = [&](llma_engine::ActMaps& m, int nr) {
+            int bad2 = 0;
+            bad2 |= make_tensor_map_bf16(&m.x_hat, e->x_hat, 3 * RC, d.d_model, nr);
+            bad2 |= make_tensor_map_bf16(&m.attn, e->attn, 2 * RC, HD, nr);
+            bad2 |= make_tensor_map_bf16(&m.h, e->h, 2 * RC, d.d_ffn, nr);
+            return bad2;
+        };
+        bad |= act_maps(e->act_prefill, e->prefill_rows);
+        if (e->decode_wide) bad |= act_maps(e->act_decode, e->decode_rows);
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
         CREATE_TRY(init_gemm_tcgen05());
+        CREATE_TRY(init_gemm_wide());
         e->attn_chunks = (d.max_seq + kAttnChunk - 1) / kAttnChunk;
-        // the chunk merge keeps 2 floats per (chunk, row) in the shared memory of the K/V tiles
-        if ((size_t)e->attn_chunks * kMaxRows * 8 > (size_t)2 * (d.head_dim / 64) * kAttnChunk * 128) {
-            free_engine(e);
-            return LLMA_ERR_CONFIG;
-        }
-        const size_t parts = (size_t)B * d.n_heads * e->attn_chunks * kMaxRows;
+        const size_t parts = (size_t)d.n_heads * e->attn_chunks * RC;
         CREATE_TRY(dalloc(&e->attn_ws_o, parts * d.head_dim));
         CREATE_TRY(dalloc(&e->attn_ws_ml, parts * 2));
-        CREATE_TRY(dalloc(&e->attn_cnt, B * d.n_heads));
         const uint64_t kv_rows = (uint64_t)L * B * d.n_heads * d.max_seq;
         if (make_tensor_map_bf16(&e->map_kcache, e->kcache, kv_rows, d.head_dim, kAttnChunk) ||
             make_tensor_map_bf16(&e->map_vcache, e->vcache, kv_rows, d.head_dim, kAttnChunk)) {

@@ -34,24 +34,39 @@ struct llma_engine {
     float *rope_cos = nullptr, *rope_sin = nullptr;
     void *kcache = nullptr, *vcache = nullptr;
 
+    // row capacities (multiples of 16): activation buffers hold row_cap rows; a decoding step uses at most
+    // decode_rows = max_batch * (max_k + 1) of them, a prompt pass prefill_rows
+    int row_cap = 0, decode_rows = 0, prefill_rows = 0;
+    int qkv_terms = 2;              // bf16 terms of the QKV projection's activation operand (2 or 3)
+
     // tensor-core GEMM path (bf16): TMA descriptors of weights and activation buffers, work buffers
     struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };
     std::vector<LayerMaps> maps;
     CUtensorMap map_lm_head;
-    int decode_nr = 32;             // rows per half used by decoding steps (16 or 32); prefill always uses 32
-    int cur_nr = 32;                // what the launches being enqueued use
+    struct ActMaps { CUtensorMap x_hat, attn, h; };  // activation operands of gemm_wide_kernel, box of nr rows
+    ActMaps act_decode, act_prefill;
+    bool decode_wide = false;       // decoding steps of more than 32 rows use gemm_wide_kernel
+    int decode_nr = 32;             // rows the decoding GEMMs are shaped for (16 / 32 narrow, decode_rows wide)
+    // what the launches being enqueued use (decoding step or prompt pass)
+    bool cur_wide = false;
+    int cur_nr = 32, cur_rows = 32;
+    const ActMaps* cur_maps = nullptr;
     int num_sms = 0;
-    float* gemm_ws = nullptr;       // split-k partial tiles [num_sms][2][128][32]
-    int32_t* gemm_cnt = nullptr;    // (unused by the current kernels)
-    float* norm_ss = nullptr;       // per-tile sums of squares of the residual rows [d/128][32]
-    float* part_max = nullptr;      // LM-head per-tile maxima [tiles][32]
+    float* gemm_ws = nullptr;       // partial tiles of gemm_ws_kernel [num_sms][2][8][128] float4
+    float* gemm_ws_wide = nullptr;  // partial tiles of gemm_wide_kernel [num_sms][2][wide_nr / 4][128] float4
+    size_t gemm_ws_bytes = 0, gemm_ws_wide_bytes = 0;
+    float* norm_ss = nullptr;       // per-tile sums of squares of the residual rows [d/128][row_cap]
+    float* part_max = nullptr;      // LM-head per-tile maxima [tiles][row_cap]
     int32_t* part_idx = nullptr;
 
     // tensor-core attention: TMA descriptors of the K/V cache, chunk partials
     CUtensorMap map_kcache, map_vcache;
     int attn_chunks = 0;
     float *attn_ws_o = nullptr, *attn_ws_ml = nullptr;
-    int32_t* attn_cnt = nullptr;
+
+    // replay of a given step sequence (llma_generate_forced)
+    int32_t *trace = nullptr, *target = nullptr;
+    int32_t trace_cap = 0;
 
     // pinned host staging
     llma::SeqState* h_state = nullptr;

@@ -1,4 +1,5 @@
 // Small state-management and inspection entry points of the C ABI.
+#include <algorithm>
 #include <cstring>
 #include <vector>
 
@@ -61,9 +62,16 @@ extern "C" int llma_last_step_info(llma_engine* e, llma_step_info* info) {
 extern "C" int llma_debug_logits(llma_engine* e, float* out) {
     if (!e || !out) return LLMA_ERR_NULL;
     if (!e->cfg.keep_logits || !e->last_step_valid) return LLMA_ERR_STATE;
-    const size_t rows = (size_t)e->dims.max_batch * e->dims.kp1;
     CU_TRY(cudaStreamSynchronize(e->stream));
-    CU_TRY(cudaMemcpy(out, e->logits, rows * e->dims.vocab * sizeof(float), cudaMemcpyDeviceToHost));
+    // the rows of a step are packed; hand them out in the documented per-sequence slots
+    CU_TRY(cudaMemcpy(e->h_rows, e->rows, sizeof(RowDesc), cudaMemcpyDeviceToHost));
+    const size_t V = (size_t)e->dims.vocab;
+    for (int s = 0; s < e->dims.max_batch; ++s) {
+        const int first = e->h_rows->seq_first[s], cnt = std::min(e->h_rows->seq_cnt[s], e->dims.kp1);
+        if (cnt <= 0 || first < 0 || first + cnt > e->row_cap) continue;
+        CU_TRY(cudaMemcpy(out + (size_t)s * e->dims.kp1 * V, e->logits + (size_t)first * V, (size_t)cnt * V * sizeof(float),
+                          cudaMemcpyDeviceToHost));
+    }
     return LLMA_OK;
 }
 
@@ -103,6 +111,11 @@ extern "C" int llma_kv_len(llma_engine* e, int32_t seq) {
     return e->h_state[seq].kv_len;
 }
 
+extern "C" int llma_row_capacity(llma_engine* e) {
+    if (!e) return LLMA_ERR_NULL;
+    return e->row_cap;
+}
+
 extern "C" int llma_gemm_impl(llma_engine* e) {
     if (!e) return LLMA_ERR_NULL;
     return e->gemm_impl;
@@ -113,7 +126,7 @@ extern "C" int llma_debug_buffer(llma_engine* e, int32_t which, float* out, int6
     const ModelDims& d = e->dims;
     const int64_t cols = which == 0 ? d.d_model : which == 1 ? 3 * (int64_t)d.hd_total : which == 2 ? d.hd_total
                        : which == 3 ? d.d_ffn : -1;
-    if (cols < 0 || count != cols * kMaxRows) return LLMA_ERR_ARG;
+    if (cols < 0 || count != cols * e->row_cap) return LLMA_ERR_ARG;
     CU_TRY(cudaStreamSynchronize(e->stream));
     if (which <= 1) {
         CU_TRY(cudaMemcpy(out, which == 0 ? e->x : e->qkv, (size_t)count * sizeof(float), cudaMemcpyDeviceToHost));
@@ -124,7 +137,7 @@ extern "C" int llma_debug_buffer(llma_engine* e, int32_t which, float* out, int6
         CU_TRY(cudaMemcpy(out, src, (size_t)count * sizeof(float), cudaMemcpyDeviceToHost));
         return LLMA_OK;
     }
-    std::vector<uint16_t> raw((size_t)2 * count);  // split bf16 [64][K]: hi rows then lo rows
+    std::vector<uint16_t> raw((size_t)2 * count);  // split bf16 [2 rc][K]: hi rows then lo rows
     CU_TRY(cudaMemcpy(raw.data(), src, raw.size() * 2, cudaMemcpyDeviceToHost));
     for (int64_t i = 0; i < count; ++i) {
         uint32_t h = (uint32_t)raw[i] << 16, l = (uint32_t)raw[count + i] << 16;

@@ -29,16 +29,20 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
     GemmArgs a;
     std::memset(&a, 0, sizeof(a));
     a.mode = mode; a.n_out = n_out; a.n_tiles = n_tiles; a.chunks = k_in / 64; a.tiles_per_map = tiles_per_map;
-    a.rows = e->rows; a.ws = e->gemm_ws; a.cnt = e->gemm_cnt; a.dev_err = e->dev_err;
+    a.rows = e->rows; a.dev_err = e->dev_err;
+    a.rc = e->row_cap; a.nr = e->cur_nr; a.terms = 2;
+    a.ws = e->cur_wide ? e->gemm_ws_wide : e->gemm_ws;
+    a.xs_layout = kActSplit;
     a.dims = e->dims;
     return a;
 }
 
 static void run_gemm(llma_engine* e, GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
-                     const void* act) {
+                     const void* act, const CUtensorMap* act_map) {
     a.act = act;
     const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
-    launch_gemm_tcgen05(e->stream, grid, e->cur_nr, true, a, a0, a1, a2);
+    if (e->cur_wide) launch_gemm_wide(e->stream, grid, true, a, a0, a1, a2, *act_map);
+    else launch_gemm_tcgen05(e->stream, grid, true, a, a0, a1, a2);
 }
 
 // Tensor-core path (bf16): 5 kernels per layer.  Every projection is fused with what follows
@@ -50,38 +54,45 @@ static void with_norm(llma_engine* e, GemmArgs& a) {
     a.norm_dim = e->dims.d_model; a.norm_eps = e->dims.rms_eps;
 }
 
+// layout of x_hat when it feeds a QKV projection
+static int qkv_act_layout(const llma_engine* e) { return e->qkv_terms == 3 ? kActSplit3 : kActSplit; }
+
 static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const ModelDims& d = e->dims;
     cudaStream_t st = e->stream;
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
+    const llma_engine::ActMaps* am = e->cur_maps;
     for (int l = 0; l < d.n_layers; ++l) {
         const llma_engine::LayerMaps& m = e->maps[l];
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
         with_norm(e, q);
+        q.terms = e->qkv_terms;
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
-        run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat);
+        run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat, am ? &am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_QKV);
         AttnArgs at;
         at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
-        at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml; at.cnt = e->attn_cnt;
+        at.n_rows = e->cur_rows;
+        at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml;
         at.dev_err = e->dev_err;
         at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0;  // prompt passes: the device-side length is stale
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
-        run_gemm(e, o, m.wo, m.wo, m.wo, e->attn);
+        run_gemm(e, o, m.wo, m.wo, m.wo, e->attn, am ? &am->attn : nullptr);
         mark(e, LLMA_K_GEMM_O);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         with_norm(e, gu);
         gu.out_act = e->h;
-        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat);
+        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat, am ? &am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
-        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h);
+        if (l + 1 < d.n_layers) dn.xs_layout = qkv_act_layout(e);  // feeds the next layer's QKV projection
+        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h, am ? &am->h : nullptr);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 6;
     }
@@ -91,11 +102,9 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         with_norm(e, lm);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
-        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->x_hat);
+        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->x_hat, am ? &am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_LMHEAD);
-        launch_argmax_final(st, true, e->rows, e->part_max, e->part_idx, vt, e->out_tok);
-        mark(e, LLMA_K_ARGMAX);
-        e->launch_counter += 2;
+        e->launch_counter += 1;
     }
 }
 
@@ -106,8 +115,9 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
     cudaStream_t st = e->stream;
     const bool b = e->bf16;
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
+    const int nr = e->cur_rows, rc = e->row_cap;
     for (int l = 0; l < d.n_layers; ++l) {
-        launch_rmsnorm(st, kActF32, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, nr, rc, e->rows, e->x, e->attn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->wq[l], (const float*)e->x_hat, e->qkv, HD, D, 3 * HD, false);
         mark(e, LLMA_K_GEMM_QKV);
@@ -115,30 +125,30 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
         mark(e, LLMA_K_GEMM_QKV);
         launch_gemm_simt(st, b, e->rows, e->wv[l], (const float*)e->x_hat, e->qkv + 2 * HD, HD, D, 3 * HD, false);
         mark(e, LLMA_K_GEMM_QKV);
-        launch_qkv_post(st, b, d, l, e->rows, e->qkv, e->rope_cos, e->rope_sin, e->kcache, e->vcache);
+        launch_qkv_post(st, b, d, l, nr, e->rows, e->qkv, e->rope_cos, e->rope_sin, e->kcache, e->vcache);
         mark(e, LLMA_K_EPILOGUE);
-        launch_attention_simt(st, b, d, l, e->rows, e->qkv, e->kcache, e->vcache, e->attn, kActF32);
+        launch_attention_simt(st, b, d, l, nr, e->rows, e->qkv, e->kcache, e->vcache, e->attn, kActF32);
         mark(e, LLMA_K_ATTN);
         launch_gemm_simt(st, b, e->rows, e->wo[l], (const float*)e->attn, e->x, D, HD, D, true);
         mark(e, LLMA_K_GEMM_O);
-        launch_rmsnorm(st, kActF32, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, nr, rc, e->rows, e->x, e->ffn_norm[l], e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->w_gate[l], (const float*)e->x_hat, e->gate_up, F, D, 2 * F, false);
         mark(e, LLMA_K_GEMM_GATEUP);
         launch_gemm_simt(st, b, e->rows, e->w_up[l], (const float*)e->x_hat, e->gate_up + F, F, D, 2 * F, false);
         mark(e, LLMA_K_GEMM_GATEUP);
-        launch_silu_mul(st, e->rows, e->gate_up, (float*)e->h, F);
+        launch_silu_mul(st, nr, e->rows, e->gate_up, (float*)e->h, F);
         mark(e, LLMA_K_EPILOGUE);
         launch_gemm_simt(st, b, e->rows, e->w_down[l], (const float*)e->h, e->x, D, F, D, true);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 12;
     }
     if (lm_head) {
-        launch_rmsnorm(st, kActF32, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
+        launch_rmsnorm(st, kActF32, nr, rc, e->rows, e->x, e->final_norm, e->x_hat, D, d.rms_eps);
         mark(e, LLMA_K_NORM);
         launch_gemm_simt(st, b, e->rows, e->lm_head, (const float*)e->x_hat, e->logits, d.vocab, D, d.vocab, false);
         mark(e, LLMA_K_GEMM_LMHEAD);
-        launch_argmax(st, e->rows, e->logits, d.vocab, e->out_tok);
+        launch_argmax(st, nr, e->rows, e->logits, d.vocab, e->out_tok);
         mark(e, LLMA_K_ARGMAX);
         e->launch_counter += 3;
     }
@@ -146,25 +156,50 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
 
 static void enqueue_embed(llma_engine* e) {
     if (e->gemm_impl == LLMA_GEMM_TCGEN05)
-        launch_embed_norm(e->stream, e->dims, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat, e->norm_ss, e->dev_err);
+        launch_embed_norm(e->stream, e->dims, e->cur_rows, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat,
+                          qkv_act_layout(e), e->norm_ss, e->dev_err);
     else
-        launch_embed(e->stream, e->dims, e->bf16, e->rows, e->tok_emb, e->x, e->dev_err);
+        launch_embed(e->stream, e->dims, e->bf16, e->cur_rows, e->rows, e->tok_emb, e->x, e->dev_err);
 }
 
-// plan (trigger search + copy) -> embedding gather -> forward -> accept + K/V commit
-static void enqueue_step(llma_engine* e, int n, int k) {
-    const ModelDims& d = e->dims;
-    e->cur_nr = e->decode_nr;
-    launch_plan(e->stream, d, e->seq_state, e->rows, e->ref, e->doc_start, e->doc_end, e->y, e->y_cap, n, k,
-                e->dev_err);
-    mark(e, LLMA_K_PLAN);
+// what the launches that follow are shaped for: a decoding step or a prompt pass
+static void shape_for_decode(llma_engine* e) {
+    e->cur_wide = e->decode_wide; e->cur_nr = e->decode_nr; e->cur_rows = e->decode_rows;
+    e->cur_maps = e->decode_wide ? &e->act_decode : nullptr;
+}
+static void shape_for_prefill(llma_engine* e) {
+    e->cur_wide = e->gemm_impl == LLMA_GEMM_TCGEN05; e->cur_nr = e->prefill_rows; e->cur_rows = e->prefill_rows;
+    e->cur_maps = e->cur_wide ? &e->act_prefill : nullptr;
+}
+
+// the integer kernel between forward passes: acceptance + K/V commit of the pass that has finished,
+// trigger search + copy + row packing for the one that follows
+static void enqueue_tail(llma_engine* e, int n, int k, bool accept, bool plan) {
+    TailArgs t;
+    std::memset(&t, 0, sizeof(t));
+    t.dims = e->dims; t.st = e->seq_state; t.rows = e->rows; t.ref = e->ref; t.doc_start = e->doc_start;
+    t.doc_end = e->doc_end; t.y = e->y; t.y_cap = e->y_cap; t.n = n; t.k = k;
+    t.do_accept = accept ? 1 : 0; t.do_plan = plan ? 1 : 0;
+    if (e->gemm_impl == LLMA_GEMM_TCGEN05) {
+        t.part_max = e->part_max; t.part_idx = e->part_idx; t.n_tiles = (e->dims.vocab + 127) / 128;
+    }
+    t.out_tok = e->out_tok;
+    t.trace = e->trace; t.target = e->target; t.trace_cap = e->trace_cap;
+    t.dev_err = e->dev_err;
+    launch_step_tail(e->stream, t);
+    mark(e, accept ? LLMA_K_ACCEPT : LLMA_K_PLAN);
+    e->launch_counter += 1;
+}
+
+// One decoding step after its plan: embedding gather -> forward -> accept + K/V commit, and (inside
+// llma_generate's graph) the plan of the next step in the same launch.
+static void enqueue_step_body(llma_engine* e, int n, int k, bool plan_next) {
+    shape_for_decode(e);
     enqueue_embed(e);
     mark(e, LLMA_K_EMBED);
-    e->launch_counter += 3;
-    enqueue_forward(e, true);
-    launch_accept(e->stream, d, e->seq_state, e->ref, e->out_tok, e->y, e->y_cap);
-    mark(e, LLMA_K_ACCEPT);
     e->launch_counter += 1;
+    enqueue_forward(e, true);
+    enqueue_tail(e, n, k, true, plan_next);
 }
 
 static int check_device_error(llma_engine* e) {
@@ -175,8 +210,10 @@ static int check_device_error(llma_engine* e) {
     CU_TRY(cudaMemsetAsync(e->dev_err, 0, sizeof(int32_t), e->stream));
     // a kernel that gave up may have left partial tiles in the hand-over slots: empty them again, so that
     // a caller who carries on after the error does not sum stale partials into later projections
-    if (code == kDevErrTimeout && e->gemm_ws)
-        CU_TRY(cudaMemsetAsync(e->gemm_ws, 0xFF, (size_t)e->num_sms * 2 * 128 * 32 * sizeof(float), e->stream));
+    if (code == kDevErrTimeout && e->gemm_ws) {
+        CU_TRY(cudaMemsetAsync(e->gemm_ws, 0xFF, e->gemm_ws_bytes, e->stream));
+        CU_TRY(cudaMemsetAsync(e->gemm_ws_wide, 0xFF, e->gemm_ws_wide_bytes, e->stream));
+    }
     CU_TRY(cudaStreamSynchronize(e->stream));
     if (code == kDevErrTimeout) return LLMA_ERR_DEVICE_TIMEOUT;
     if (code == kDevErrCapacity) return LLMA_ERR_CAPACITY;
@@ -206,22 +243,23 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
         if (prompt[i] < 0 || prompt[i] >= d.vocab) return LLMA_ERR_TOKEN_RANGE;
     int rc = read_state(e);
     if (rc) return rc;
-    // push prompt[0 .. P-2] through the decoder, kMaxRows consecutive positions per pass
+    // push prompt[0 .. P-2] through the decoder, prefill_rows consecutive positions per pass
     const int n_cache = n_prompt - 1;
-    for (int p0 = 0; p0 < n_cache; p0 += kMaxRows) {
-        const int cnt = std::min(kMaxRows, n_cache - p0);
+    const int PR = e->prefill_rows;
+    shape_for_prefill(e);
+    for (int p0 = 0; p0 < n_cache; p0 += PR) {
+        const int cnt = std::min(PR, n_cache - p0);
         RowDesc* R = e->h_rows;
-        for (int r = 0; r < kMaxRows; ++r) {
+        for (int r = 0; r < kRowCap; ++r) {
             R->tok[r] = r < cnt ? prompt[p0 + r] : 0;
             R->pos[r] = r < cnt ? p0 + r : -1;
             R->seq[r] = seq;
         }
-        for (int s2 = 0; s2 < kMaxRows; ++s2) { R->seq_first[s2] = 0; R->seq_cnt[s2] = 0; R->seq_maxpos[s2] = -1; }
+        for (int s2 = 0; s2 < kSeqCap; ++s2) { R->seq_first[s2] = 0; R->seq_cnt[s2] = 0; R->seq_maxpos[s2] = -1; }
         R->seq_first[seq] = 0; R->seq_cnt[seq] = cnt; R->seq_maxpos[seq] = p0 + cnt - 1;
         R->rows_used = cnt;
         R->max_pos = p0 + cnt - 1;
         CU_TRY(cudaMemcpyAsync(e->rows, R, sizeof(RowDesc), cudaMemcpyHostToDevice, e->stream));
-        e->cur_nr = 32;  // prompt chunks fill all 32 rows
         enqueue_embed(e);
         enqueue_forward(e, false);
         CU_TRY(cudaGetLastError());
@@ -301,7 +339,8 @@ extern "C" int llma_step(llma_engine* e, int32_t n, int32_t k, int32_t* out_toke
         rc = write_state(e, s);
         if (rc) return rc;
     }
-    enqueue_step(e, n, k);
+    enqueue_tail(e, n, k, false, true);
+    enqueue_step_body(e, n, k, false);
     CU_TRY(cudaGetLastError());
     rc = check_device_error(e);
     if (rc) return rc;
@@ -325,7 +364,7 @@ static int get_step_graph(llma_engine* e, int n, int k, cudaGraphExec_t* out) {
     cudaGraph_t g = nullptr;
     const int64_t before = e->launch_counter;
     CU_TRY(cudaStreamBeginCapture(e->stream, cudaStreamCaptureModeThreadLocal));
-    enqueue_step(e, n, k);
+    enqueue_step_body(e, n, k, true);
     cudaError_t ce = cudaStreamEndCapture(e->stream, &g);
     e->launches_per_step = e->launch_counter - before;
     e->launch_counter = before;
@@ -373,6 +412,13 @@ extern "C" int llma_generate(llma_engine* e, int32_t max_new, int32_t n, int32_t
     // can never be too many.  Launch that many back to back, look at the counters once, repeat.
     int64_t launches = 0;
     CU_TRY(cudaEventRecord(e->ev0, e->stream));
+    // the first step's plan; every graph launch then ends with the plan of the step after it
+    {
+        const int64_t before = e->launch_counter;
+        enqueue_tail(e, n, k, false, true);
+        launches += e->launch_counter - before;
+        e->launch_counter = before;
+    }
     for (;;) {
         int left = 0;
         for (int s = 0; s < d.max_batch; ++s) {
@@ -413,6 +459,75 @@ extern "C" int llma_generate(llma_engine* e, int32_t max_new, int32_t n, int32_t
     return LLMA_OK;
 }
 
+// Replay of a given sequence of step shapes (the paper's target-guided measurement, Section 3.2 and
+// Algorithm 2): the forward passes are the real ones, the trigger and acceptance decisions come from the trace.
+extern "C" int llma_generate_forced(llma_engine* e, int32_t seq, const int32_t* trace, int32_t n_steps,
+                                    const int32_t* target, int32_t n_target, llma_stats* stats) {
+    if (!e || !trace || !target) return LLMA_ERR_NULL;
+    const ModelDims& d = e->dims;
+    if (seq < 0 || seq >= d.max_batch) return LLMA_ERR_CAPACITY;
+    if (n_steps < 1 || n_target < 1 || n_steps > e->trace_cap) return LLMA_ERR_ARG;
+    int64_t total = 0;
+    for (int i = 0; i < n_steps; ++i) {
+        const int r = trace[2 * i], m = trace[2 * i + 1];
+        if (r < 1 || r > d.kp1 || m < 1 || m > r) return LLMA_ERR_ARG;
+        total += m;
+    }
+    if (total != n_target) return LLMA_ERR_ARG;
+    for (int i = 0; i < n_target; ++i)
+        if (target[i] < 0 || target[i] >= d.vocab) return LLMA_ERR_TOKEN_RANGE;
+    int rc = read_state(e);
+    if (rc) return rc;
+    for (int s = 0; s < d.max_batch; ++s)
+        if (s != seq && e->h_state[s].active && !e->h_state[s].done) return LLMA_ERR_STATE;
+    const SeqState s0 = e->h_state[seq];
+    if (!s0.active) return LLMA_ERR_STATE;
+    if (s0.kv_len + n_target > d.max_seq || s0.y_len + n_target > e->y_cap) return LLMA_ERR_CAPACITY;
+    CU_TRY(cudaMemcpyAsync(e->trace + (size_t)seq * e->trace_cap * 2, trace, (size_t)n_steps * 2 * sizeof(int32_t),
+                           cudaMemcpyHostToDevice, e->stream));
+    CU_TRY(cudaMemcpyAsync(e->target + (size_t)seq * e->y_cap + s0.y_len, target, (size_t)n_target * sizeof(int32_t),
+                           cudaMemcpyHostToDevice, e->stream));
+    SeqState& S = e->h_state[seq];
+    S.target_len = S.y_len + n_target; S.done = 0; S.forced_rows = 1; S.forced_emit = 1; S.trace_step = 0;
+    rc = write_state(e, seq);  // synchronises: the host arrays may go after this
+    if (rc) return rc;
+    cudaGraphExec_t graph = nullptr;
+    rc = get_step_graph(e, 1, 0, &graph);
+    if (rc) return rc;
+    CU_TRY(cudaEventRecord(e->ev0, e->stream));
+    const int64_t before = e->launch_counter;
+    enqueue_tail(e, 1, 0, false, true);
+    const int64_t tail_launches = e->launch_counter - before;
+    e->launch_counter = before;
+    for (int i = 0; i < n_steps; ++i) CU_TRY(cudaGraphLaunch(graph, e->stream));
+    CU_TRY(cudaEventRecord(e->ev1, e->stream));
+    rc = check_device_error(e);
+    if (rc) return rc;
+    rc = read_state(e);
+    if (rc) return rc;
+    SeqState& T = e->h_state[seq];
+    llma_stats st;
+    std::memset(&st, 0, sizeof(st));
+    st.steps = T.steps - s0.steps; st.trigger_steps = T.trigger_steps - s0.trigger_steps;
+    st.copied_accepted = T.copied_accepted - s0.copied_accepted; st.tokens = T.y_len - s0.y_len;
+    st.launches = tail_launches + (int64_t)n_steps * e->launches_per_step;
+    CU_TRY(cudaEventElapsedTime(&st.device_ms, e->ev0, e->ev1));
+    T.forced_rows = 0; T.forced_emit = 0; T.trace_step = 0;
+    rc = write_state(e, seq);
+    if (rc) return rc;
+    if (stats) *stats = st;
+    e->last_step_valid = false;
+    return st.tokens == n_target ? LLMA_OK : LLMA_ERR_STATE;
+}
+
+extern "C" int llma_debug_set_device_error(llma_engine* e, int32_t code) {
+    if (!e) return LLMA_ERR_NULL;
+    if (code < kDevErrNone || code > kDevErrToken) return LLMA_ERR_ARG;
+    CU_TRY(cudaMemcpyAsync(e->dev_err, &code, sizeof(int32_t), cudaMemcpyHostToDevice, e->stream));
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    return LLMA_OK;
+}
+
 extern "C" int llma_profile_steps(llma_engine* e, int32_t n, int32_t k, int32_t steps, llma_profile* out) {
     if (!e || !out) return LLMA_ERR_NULL;
     int rc = check_nk(e, n, k);
@@ -439,7 +554,8 @@ extern "C" int llma_profile_steps(llma_engine* e, int32_t n, int32_t k, int32_t 
         e->prof_on = true;
         e->prof_n = 0;
         mark(e, -1);
-        enqueue_step(e, n, k);
+        enqueue_tail(e, n, k, false, true);
+        enqueue_step_body(e, n, k, false);
         e->prof_on = false;
         CU_TRY(cudaGetLastError());
         rc = check_device_error(e);

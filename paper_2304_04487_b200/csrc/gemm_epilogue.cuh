@@ -1,7 +1,9 @@
-// Epilogues of the weight-streaming GEMM: what happens to a finished 128 x 32 fp32 tile.
-// Called by the 128 epilogue threads after the tile has been staged in shared memory:
+// Epilogues of the weight-streaming GEMM: what happens to a finished 128 x 32 fp32 block.
+// Called by the 128 epilogue threads after the block has been staged in shared memory:
 // stage[f][j] is the result for output feature f of the tile (thread `row` staged its own
-// feature) and activation row j.  red_f / red_i are [4][32] scratch for per-warp reductions.
+// feature) and activation row jb + j, j < nj <= 32.  Engines of at most 32 rows have one
+// block per tile (jb = 0); the wide kernel walks a tile in blocks of 32 rows.
+// red_f / red_i are [4][32] scratch for per-warp reductions.
 //
 // The loops over activation rows are deliberately NOT unrolled over all 32 rows: this code
 // runs once per tile, so its cost is dominated by instruction fetch, and compact loops
@@ -26,9 +28,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 // x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
 // When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
 // per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
-// With kHavePre, xpre holds x[0..11, col] and the gain, read earlier by the caller.
+// With kHavePre (jb = 0 only), xpre holds x[0..11, col] and the gain, read earlier by the caller.
 template <bool kHavePre>
-__device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int rows_used,
+__device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                float (*stage)[33], float* red_f, const float (&xpre)[kXPre]) {
     const int col = tile * 128 + row;
     const bool valid = col < g.n_out;
@@ -39,49 +41,51 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
     if (kHavePre) {
 #pragma unroll
         for (int u = 0; u < kXPre - 1; ++u)
-            if (u < rows_used) stage[row][u] += xpre[u];
+            if (u < nj) stage[row][u] += xpre[u];
     }
-    for (int j0 = kHavePre ? kXPre - 1 : 0; j0 < rows_used; j0 += 8) {
+    for (int j0 = kHavePre ? kXPre - 1 : 0; j0 < nj; j0 += 8) {
         float xv[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            xv[u] = (valid && j0 + u < rows_used) ? __ldcg(&g.out_f32[(int64_t)(j0 + u) * g.ld + col]) : 0.f;
+            xv[u] = (valid && j0 + u < nj) ? __ldcg(&g.out_f32[(int64_t)(jb + j0 + u) * g.ld + col]) : 0.f;
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            if (j0 + u < rows_used) stage[row][j0 + u] += xv[u];
+            if (j0 + u < nj) stage[row][j0 + u] += xv[u];
     }
 #pragma unroll 1
-    for (int j = 0; j < rows_used; ++j) {
+    for (int j = 0; j < nj; ++j) {
         const float xn = valid ? stage[row][j] : 0.f;
-        if (valid) g.out_f32[(int64_t)j * g.ld + col] = xn;
+        if (valid) g.out_f32[(int64_t)(jb + j) * g.ld + col] = xn;
         if (fold) {
-            if (valid) store_act(g.xs_out, kActSplit, j, col, g.n_out, xn * gain);
+            if (valid) store_act(g.xs_out, g.xs_layout, g.rc, jb + j, col, g.n_out, xn * gain);
             const float sq = warp_sum(xn * xn);
             if (lane == 0) red_f[warp * 32 + j] = sq;
         }
     }
     if (!fold) return;
     epi_sync();
-    if (row < rows_used)
-        g.ss_out[(int64_t)tile * 32 + row] = ((red_f[row] + red_f[32 + row]) + red_f[64 + row]) + red_f[96 + row];
+    if (row < nj)
+        g.ss_out[(int64_t)tile * g.rc + jb + row] = ((red_f[row] + red_f[32 + row]) + red_f[64 + row]) + red_f[96 + row];
     epi_sync();
 }
 
 // out[r, n] = acc
-__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int row, int rows_used,
+__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                float (*stage)[33]) {
     const int col = tile * 128 + row;
     if (col >= g.n_out) return;
 #pragma unroll 1
-    for (int j = 0; j < rows_used; ++j) g.out_f32[(int64_t)j * g.ld + col] = stage[row][j];
+    for (int j = 0; j < nj; ++j) g.out_f32[(int64_t)(jb + j) * g.ld + col] = stage[row][j];
 }
 
 // QKV: rotary embedding on q and k (pair (i, i + hd/2)), q to the fp32 qkv buffer, k and v
 // rows into the bf16 cache at (sequence, position) of every used row.
-__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, int rows_used,
-                                             float (*stage)[33], const int* rowinfo, const float2* rope_s) {
-    // rowinfo[j] = position of activation row j (-1: unused), rowinfo[32 + j] = its sequence slot;
-    // rope_s[j * hd/2 + i] = (cos, sin) of row j's position for rotary pair i
+//   row_pos[r] / row_seq[r]: position (-1: unused) and sequence slot of activation row r;
+//   rope_s: (cos, sin) of rows jb .. jb+31 staged in shared memory, [j][hd/2], or nullptr to read
+//   the tables in global memory.
+__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int row, int jb, int nj,
+                                             float (*stage)[33], const int* row_pos, const int* row_seq,
+                                             const float2* rope_s) {
     const ModelDims& d = g.dims;
     const int mat = tile / g.tiles_per_map;
     const int col = (tile % g.tiles_per_map) * 128 + row;
@@ -92,20 +96,22 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
     const int fi = idx % half;
     if (col < g.n_out) {
 #pragma unroll 1
-        for (int j = 0; j < rows_used; ++j) {
-            const int pos = rowinfo[j];
+        for (int j = 0; j < nj; ++j) {
+            const int pos = row_pos[jb + j];
             if (pos < 0) continue;
             float val = stage[row][j];
             if (mat < 2) {
-                const float2 cs = rope_s[j * half + fi];
+                const float2 cs = rope_s ? rope_s[j * half + fi]
+                                         : make_float2(__ldg(&g.rope_cos[(int64_t)pos * half + fi]),
+                                                       __ldg(&g.rope_sin[(int64_t)pos * half + fi]));
                 const float other = stage[prow][j];
                 val = lower ? (val * cs.x - other * cs.y) : (other * cs.y + val * cs.x);
             }
             if (mat == 0) {
-                g.out_f32[(int64_t)j * g.ld + col] = val;
+                g.out_f32[(int64_t)(jb + j) * g.ld + col] = val;
             } else {
                 __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
-                cache[kv_row_index(d, g.layer, rowinfo[32 + j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
+                cache[kv_row_index(d, g.layer, row_seq[jb + j], head, pos) * hd + idx] = __float2bfloat16_rn(val);
             }
         }
     }
@@ -113,29 +119,29 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
 }
 
 // SwiGLU: tile rows 0..63 are gate features, 64..127 the matching up features.
-__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, int rows_used,
+__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33]) {
     const int fi = row & 63, f = tile * 64 + fi;
     if (f < g.n_out) {
 #pragma unroll 1
-        for (int j = row >> 6; j < rows_used; j += 2) {
+        for (int j = row >> 6; j < nj; j += 2) {
             const float gate = stage[fi][j], up = stage[64 + fi][j];
-            store_act(g.out_act, kActSplit, j, f, g.n_out, gate / (1.f + expf(-gate)) * up);
+            store_act(g.out_act, kActSplit, g.rc, jb + j, f, g.n_out, gate / (1.f + expf(-gate)) * up);
         }
     }
     epi_sync();
 }
 
 // LM head: optional logits store, then the tile's (max, lowest argmax) for every used row.
-__device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, int rows_used,
+__device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33], float* red_f, int* red_i) {
     const int v = tile * 128 + row;
     const bool valid = v < g.n_out;
     const int warp = row >> 5, lane = row & 31;
 #pragma unroll 1
-    for (int j = 0; j < rows_used; ++j) {
+    for (int j = 0; j < nj; ++j) {
         const float a = stage[row][j];
-        if (g.out_f32 && valid) g.out_f32[(int64_t)j * g.ld + v] = a;
+        if (g.out_f32 && valid) g.out_f32[(int64_t)(jb + j) * g.ld + v] = a;
         float bv = valid ? a : -INFINITY;
         int bi = valid ? v : 0x7fffffff;
         for (int o = 16; o > 0; o >>= 1) {
@@ -146,16 +152,26 @@ __device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int
         if (lane == 0) { red_f[warp * 32 + j] = bv; red_i[warp * 32 + j] = bi; }
     }
     epi_sync();
-    if (row < rows_used) {
+    if (row < nj) {
         float bv = red_f[row]; int bi = red_i[row];
         for (int w = 1; w < 4; ++w) {
             const float ov = red_f[w * 32 + row]; const int oi = red_i[w * 32 + row];
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
-        g.part_max[(int64_t)tile * 32 + row] = bv;
-        g.part_idx[(int64_t)tile * 32 + row] = bi;
+        g.part_max[(int64_t)tile * g.rc + jb + row] = bv;
+        g.part_idx[(int64_t)tile * g.rc + jb + row] = bi;
     }
     epi_sync();
 }
+
+// Partial tiles in the workspace: [cta][slot][q][feature] float4, q = group of four activation rows
+// (qn groups per slot).  The 32 features of a warp are 512 consecutive bytes, so one store or polling
+// load of a warp touches four lines.
+__device__ __forceinline__ float4* ws_slot(float* ws, int qn, int cta, int slot, int feature) {
+    return reinterpret_cast<float4*>(ws) + ((int64_t)cta * 2 + slot) * ((int64_t)qn * 128) + feature;
+}
+
+// Range of flat (tile, chunk) work items owned by CTA b of G.
+__device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
 
 }  // namespace llma

@@ -10,7 +10,7 @@ using namespace llma;
 
 namespace llma {
 int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, int32_t k_in, float* ws,
-                       int32_t* cnt, int32_t* dev_err, int grid, cudaStream_t st);
+                       int32_t* dev_err, int grid, cudaStream_t st);
 }
 
 namespace {
@@ -20,7 +20,7 @@ constexpr int kMaxTiles = 2048;      // n_out <= 262144
 constexpr int kMaxK = 16384;         // k_in limit of the operand staging
 constexpr size_t kWsBytes = (size_t)kMaxGrid * 2 * 128 * 32 * sizeof(float);      // 5,242,880
 constexpr size_t kCntBytes = ((size_t)(kMaxTiles + 1) * sizeof(int32_t) + 255) / 256 * 256;
-constexpr size_t kOperandBytes = (size_t)kGemmN * kMaxK * sizeof(__nv_bfloat16);  // 2,097,152
+constexpr size_t kOperandBytes = (size_t)64 * kMaxK * sizeof(__nv_bfloat16);     // 2,097,152
 constexpr size_t kScratchBytes = kWsBytes + kCntBytes + kOperandBytes;            // about 7.0 MiB
 
 // Every GPU that loads this library holds this array until the process exits.  In host
@@ -68,7 +68,7 @@ extern "C" int llma_gemm_rows32_bf16_noalloc(const void* W, const void* a, float
     cudaStream_t st = (cudaStream_t)cuda_stream;
     int grid = gemm_grid_for((int64_t)n_tiles * (k_in / 64), sms);
     if (grid > kMaxGrid) grid = kMaxGrid;
-    const size_t a_bytes = (size_t)kMaxRows * k_in * sizeof(__nv_bfloat16);
+    const size_t a_bytes = (size_t)32 * k_in * sizeof(__nv_bfloat16);
     // the array keeps the previous call's contents: the error word must start at
     // zero, and the low half of the operand must be zero (this entry point takes plain bf16 rows)
     CU_TRY(cudaMemsetAsync(cnt, 0, ((size_t)n_tiles + 1) * sizeof(int32_t), st));
@@ -76,7 +76,7 @@ extern "C" int llma_gemm_rows32_bf16_noalloc(const void* W, const void* a, float
     CU_TRY(cudaMemsetAsync(ws, 0xFF, (size_t)grid * 2 * 128 * 32 * sizeof(float), st));
     CU_TRY(cudaMemcpyAsync(operand, a, a_bytes, cudaMemcpyDeviceToDevice, st));
     CU_TRY(cudaMemsetAsync(reinterpret_cast<char*>(operand) + a_bytes, 0, a_bytes, st));
-    int rc = gemm_rows32_launch(W, operand, out, n_out, k_in, ws, cnt, cnt + n_tiles, grid, st);
+    int rc = gemm_rows32_launch(W, operand, out, n_out, k_in, ws, cnt + n_tiles, grid, st);
     if (rc) return rc;
     int32_t err = 0;
     CU_TRY(cudaMemcpyAsync(&err, cnt + n_tiles, sizeof(int32_t), cudaMemcpyDeviceToHost, st));

@@ -1,7 +1,7 @@
 // Weight-streaming GEMM on tcgen05 tensor cores: TMA -> shared-memory ring -> UMMA with the
 // accumulator in tensor memory -> fused epilogue.  See gemm_tcgen05.cuh for the contract.
 //
-// Roles inside one CTA of 192 threads:
+// Roles inside one CTA of 320 threads:
 //   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue
 //   warp  4    producer: one thread issues the TMA loads of the weight tiles
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
@@ -26,22 +26,15 @@ namespace llma {
 
 using namespace ptx;
 
-// Partial tiles in the workspace: [cta][slot][q][feature] float4, q = group of four activation rows.  The 32
-// features of a warp are 512 consecutive bytes, so one store or polling load of a warp touches four lines.
-__device__ __forceinline__ float4* ws_slot(float* ws, int cta, int slot, int feature) {
-    return reinterpret_cast<float4*>(ws) + ((int64_t)cta * 2 + slot) * (8 * 128) + feature;
-}
-
-// Range of flat (tile, chunk) work items owned by CTA b of G.
-__device__ __forceinline__ int64_t cta_begin(int64_t work, int b, int G) { return work * b / G; }
-
-// NR = activation rows per half (hi / lo): 16 or 32.  MMA N = 2 * NR.  MODE = GemmMode: one kernel per
-// fused epilogue, so that each carries only the code it runs (the end of a launch is instruction-fetch-bound).
-template <int NR, int MODE>
+// NR = activation rows: 16 or 32 = MMA N.  NT = bf16 terms of the activation operand (2 or 3): each weight
+// tile is multiplied by every term, all into the same accumulator.  MODE = GemmMode: one kernel per fused
+// epilogue, so that each carries only the code it runs (the end of a launch is instruction-fetch-bound).
+template <int NR, int NT, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2) {
-    using Cfg = GemmCfg<NR>;
+    using Cfg = GemmCfg<NR, NT>;
+    constexpr uint32_t kTmemCols = 2 * NR;  // two accumulators of NR columns (32 is the smallest allocation)
     constexpr int S = Cfg::kStages;
     constexpr uint32_t kBBytes = Cfg::kBBytes;
 
@@ -79,7 +72,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         fence_mbar_init();
     }
     if (warp == 5) {
-        tmem_alloc(smem_u32((const void*)&sh[0]), 4 * NR);
+        tmem_alloc(smem_u32((const void*)&sh[0]), kTmemCols);
         tmem_relinquish();
     }
     if (warp == 4 && lane == 0) {
@@ -127,7 +120,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else if (warp == 5) {
         // ------------------------------- MMA issuer ---------------------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_m128(2 * NR);
+            constexpr uint32_t idesc = idesc_bf16_m128(NR);
             int64_t it = 0;
             int seg = 0;
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
@@ -137,7 +130,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const uint32_t use = (uint32_t)(seg >> 1);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (2 * NR);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * NR;
                 for (int c = c0; c < c1; ++c, ++it) {
                     const int s = (int)(it % S);
                     const uint32_t ph = (uint32_t)((it / S) & 1);
@@ -146,8 +139,12 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
                     const uint64_t db = smem_desc_sw128(sB + s * kBBytes);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-                        umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk) {  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+#pragma unroll
+                        for (int t = 0; t < NT; ++t)  // term t of the activations: NR rows of 128 bytes further on
+                            umma_bf16(d_tmem, da + 2 * kk, db + (uint64_t)(t * NR * 8) + 2 * kk, idesc,
+                                      (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
+                    }
                     umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
                 }
                 if (sh[1]) break;
@@ -158,17 +155,17 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else if (warp >= 6) {
         // ------------------------------- activation loaders ----------------------------------------
         // Tile layout in shared memory (what the MMA's K-major, 128-byte
-        // swizzled descriptor reads): row r = 0..2NR-1 (hi rows, then lo rows) at r * 128 bytes, its
+        // swizzled descriptor reads): row r = 0..NT*NR-1 (NR rows per term) at r * 128 bytes, its
         // 16-byte unit j stored at position j ^ (r & 7).  Rows past those in use are left as they are:
         // their columns of the accumulator are never read.
         constexpr int NW = 4;  // loader warps: warp 6 + i takes items i, i + NW, ...
         const int sw = warp - 6;
         grid_dependency_wait();  // activations are written by the kernel before this one
-        const int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : NR;
+        const int rows_used = g.rows ? min(__ldcg(&g.rows->rows_used), NR) : NR;
         const int64_t n_items = w_end - w_beg;
         const int64_t ld_bytes = (int64_t)C * 128;  // one activation row: k_in bf16
         const char* act = reinterpret_cast<const char*>(g.act);
-        constexpr int kUnits = 2 * NR * 8 / 32;     // 16-byte units per lane
+        constexpr int kUnits = NT * NR * 8 / 32;    // 16-byte units per lane
         // rows of the next tile are requested before waiting for its stage to come free, so the
         // latency of the loads hides behind the MMAs of the tiles in between
         uint4 v[kUnits];
@@ -177,8 +174,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
             for (int u = 0; u < kUnits; ++u) {
                 const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
-                const int rr = r < NR ? r : r - NR;                   // row inside its half
-                const int src_row = r < NR ? r : kMaxRows + rr;       // lo rows start at kMaxRows
+                const int t = r / NR, rr = r - t * NR;                // term, row inside it
+                const int src_row = t * g.rc + rr;                    // term t starts at row t * rc
                 v[u] = make_uint4(0u, 0u, 0u, 0u);
                 if (rr < row_limit)
                     v[u] = __ldcg(reinterpret_cast<const uint4*>(act + src_row * ld_bytes + (int64_t)c * 128 + j * 16));
@@ -197,7 +194,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
             for (int u = 0; u < kUnits; ++u) {
                 const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
-                const int rr = r < NR ? r : r - NR;
+                const int rr = r % NR;
                 if (rr < rows_used) st_shared_v4(sB + st * kBBytes + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
             }
             fence_proxy_async_shared();  // make the stores visible to the tensor core's reads
@@ -208,19 +205,19 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
-        const int rows_used = g.rows ? g.rows->rows_used : NR;
+        const int rows_used = g.rows ? min(g.rows->rows_used, NR) : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
-        if (g.ss_in && row < 32) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
+        if (g.ss_in && row < NR) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
             float ssum = 0.f;
             int t = 0;
             for (; t + 8 <= g.ss_tiles; t += 8) {  // eight loads in flight
                 float v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = __ldcg(&g.ss_in[(int64_t)(t + u) * 32 + row]);
+                for (int u = 0; u < 8; ++u) v[u] = __ldcg(&g.ss_in[(int64_t)(t + u) * g.rc + row]);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) ssum += v[u];
             }
-            for (; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * 32 + row]);
+            for (; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * g.rc + row]);
             rscale[row] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
         }
         if (MODE == kGemmQKV) {  // the rows' positions and sequence slots, read once per CTA
@@ -253,7 +250,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
         };
         // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
-        auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[kXPre]) {
+        auto finish_tile = [&](int tile, float (&acc)[NR], const float (&xpre)[kXPre]) {
             if (g.ss_in) {
 #pragma unroll
                 for (int j = 0; j < NR; ++j) stage[row][j] = acc[j] * rscale[j];
@@ -262,11 +259,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 for (int j = 0; j < NR; ++j) stage[row][j] = acc[j];
             }
             epi_sync();
-            if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, rows_used, stage, red_i, rope_s);
-            else if constexpr (MODE == kGemmResid) epilogue_resid<kPrefetchX>(g, tile, row, rows_used, stage, red_f, xpre);
-            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, rows_used, stage);
-            else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, rows_used, stage);
-            else epilogue_lmhead(g, tile, row, rows_used, stage, red_f, red_i);
+            if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, 0, rows_used, stage, red_i, red_i + 32, rope_s);
+            else if constexpr (MODE == kGemmResid) epilogue_resid<kPrefetchX>(g, tile, row, 0, rows_used, stage, red_f, xpre);
+            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, 0, rows_used, stage);
+            else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, 0, rows_used, stage);
+            else epilogue_lmhead(g, tile, row, 0, rows_used, stage, red_f, red_i);
         };
         // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks
         // its own partial (slot 0 of its workspace) and completes the tile after its last segment.  Every
@@ -297,20 +294,11 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             epi_sync();
             if (!ok) { aborted = true; break; }
             tc_fence_after();
-            float acc[32];
+            float acc[NR];
             {
-                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (2 * NR);
-                if (NR == 32) {
-                    float lo[32];
-                    tmem_ld_32cols(t0, acc);
-                    tmem_ld_32cols(t0 + 32, lo);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
-                } else {
-                    tmem_ld_32cols(t0, acc);  // columns 0..15 hi, 16..31 lo
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) { acc[j] += acc[16 + j]; acc[16 + j] = 0.f; }
-                }
+                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * NR;
+                if constexpr (NR == 32) tmem_ld_32cols(t0, acc);
+                else tmem_ld_16cols(t0, acc);
             }
             tc_fence_before();
             __syncwarp();
@@ -319,7 +307,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
             if (w_beg > t_lo || w_end < t_hi) {  // the tile is shared with a neighbour
                 const bool owner = w_end >= t_hi;
-                float4* dst = ws_slot(g.ws, b, owner ? 0 : 1, row);
+                float4* dst = ws_slot(g.ws, NR / 4, b, owner ? 0 : 1, row);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q)  // only the columns of rows in use travel
                     if (4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
@@ -336,13 +324,13 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         if (own_tile >= 0 && !aborted) {
             float xpre[kXPre];
             prefetch_x(own_tile, xpre);
-            float acc[32];
+            float acc[NR];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+            for (int j = 0; j < NR; ++j) acc[j] = 0.f;
             // this CTA's own partial (parked in slot 0 by these same threads) is requested now and added last
             float4 own[NR / 4];
             {
-                const float4* src = ws_slot(g.ws, b, 0, row);
+                const float4* src = ws_slot(g.ws, NR / 4, b, 0, row);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q)
                     if (4 * q < rows_used) own[q] = src[q * 128];
@@ -357,7 +345,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
                     for (int u = 0; u < kBatch; ++u) {
                         if (bb + u < b) {
-                            const float4* src = ws_slot(g.ws, bb + u, 1, row);
+                            const float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q)
                                 if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q * 128);
@@ -383,7 +371,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     if (bb + u < b) {
-                        float4* src = ws_slot(g.ws, bb + u, 1, row);
+                        float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
 #pragma unroll
                         for (int q = 0; q < NR / 4; ++q) {
                             if (4 * q < rows_used) {
@@ -409,36 +397,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 4 * NR);
-    }
-}
-
-// ---- argmax over the per-tile partials --------------------------------------------------------
-__global__ void __launch_bounds__(128) argmax_final_kernel(const RowDesc* __restrict__ rows,
-                                                           const float* __restrict__ part_max,
-                                                           const int32_t* __restrict__ part_idx, int n_tiles,
-                                                           int32_t* __restrict__ out_tok) {
-    grid_launch_dependents();
-    grid_dependency_wait();
-    const int r = blockIdx.x;
-    if (rows->pos[r] < 0) { if (threadIdx.x == 0) out_tok[r] = -1; return; }
-    float bv = -INFINITY; int bi = 0x7fffffff;
-    for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
-        const float v = part_max[(int64_t)t * 32 + r]; const int i = part_idx[(int64_t)t * 32 + r];
-        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-    }
-    __shared__ float sv[4]; __shared__ int si[4];
-    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = bv; si[threadIdx.x >> 5] = bi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < 4; ++w)
-            if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
-        out_tok[r] = bi;
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -471,19 +430,20 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int NR, int MODE>
+template <int NR, int NT, int MODE>
 static cudaError_t opt_in() {
-    return cudaFuncSetAttribute(gemm_ws_kernel<NR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)GemmCfg<NR>::kSmemBytes);
+    return cudaFuncSetAttribute(gemm_ws_kernel<NR, NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)GemmCfg<NR, NT>::kSmemBytes);
 }
 template <int NR>
 static cudaError_t opt_in_all() {
     cudaError_t e;
-    if ((e = opt_in<NR, kGemmQKV>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, kGemmResid>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, kGemmSwiGLU>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, kGemmLmHead>()) != cudaSuccess) return e;
-    return opt_in<NR, kGemmStore>();
+    if ((e = opt_in<NR, 2, kGemmQKV>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, 3, kGemmQKV>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, 2, kGemmResid>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, 2, kGemmSwiGLU>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, 2, kGemmLmHead>()) != cudaSuccess) return e;
+    return opt_in<NR, 2, kGemmStore>();
 }
 
 cudaError_t init_gemm_tcgen05() {
@@ -492,37 +452,40 @@ cudaError_t init_gemm_tcgen05() {
     return opt_in_all<32>();
 }
 
+// three terms exist for the QKV projection only (its K/V rows are rounded to bf16 afterwards)
 template <int NR>
 static void launch_mode(cudaLaunchConfig_t* cfg, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
                         const CUtensorMap& a2) {
     switch (args.mode) {
-        case kGemmQKV: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmQKV>, args, a0, a1, a2); break;
-        case kGemmResid: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmResid>, args, a0, a1, a2); break;
-        case kGemmSwiGLU: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmSwiGLU>, args, a0, a1, a2); break;
-        case kGemmLmHead: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmLmHead>, args, a0, a1, a2); break;
-        default: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmStore>, args, a0, a1, a2); break;
+        case kGemmQKV:
+            if (args.terms == 3) {
+                cfg->dynamicSmemBytes = GemmCfg<NR, 3>::kSmemBytes;
+                cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 3, kGemmQKV>, args, a0, a1, a2);
+            } else {
+                cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmQKV>, args, a0, a1, a2);
+            }
+            break;
+        case kGemmResid: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmResid>, args, a0, a1, a2); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmSwiGLU>, args, a0, a1, a2); break;
+        case kGemmLmHead: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmLmHead>, args, a0, a1, a2); break;
+        default: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmStore>, args, a0, a1, a2); break;
     }
 }
 
-void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = nr == 16 ? GemmCfg<16>::kSmemBytes : GemmCfg<32>::kSmemBytes;
+    cfg.dynamicSmemBytes = args.nr == 16 ? GemmCfg<16, 2>::kSmemBytes : GemmCfg<32, 2>::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (nr == 16) launch_mode<16>(&cfg, args, a0, a1, a2);
+    if (args.nr == 16) launch_mode<16>(&cfg, args, a0, a1, a2);
     else launch_mode<32>(&cfg, args, a0, a1, a2);
-}
-
-void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
-                         int32_t n_tiles, int32_t* out_tok) {
-    launch_pdl(st, pdl, dim3(kMaxRows), dim3(128), 0, argmax_final_kernel, rows, part_max, part_idx, (int)n_tiles, out_tok);
 }
 
 }  // namespace llma

@@ -1,16 +1,22 @@
 // Weight-streaming GEMM for the decoder's projections (library-private interface).
 //
-//   out[r, n] = sum_k W[n, k] * a[r, k],  r < 32 activation rows, W bf16 [n_out, k_in].
+//   out[r, n] = sum_k W[n, k] * a[r, k],  r < rows (up to 256 activation rows), W bf16 [n_out, k_in].
 //
-// The activations arrive split into two bf16 halves (ActLayout kActSplit: 64 rows, hi then lo);
-// the MMA's N dimension is those 64 rows and the epilogue adds the hi and lo columns, so the
-// product keeps 16 mantissa bits of the activations at no cost in weight traffic.
+// The activations arrive split into bf16 terms (ActLayout kActSplit / kActSplit3: hi rows, lo rows,
+// optionally a third term); every term is multiplied by the same weight tile and accumulated into
+// the same fp32 accumulator, so the product keeps 16 (24) mantissa bits of the activations at no
+// cost in weight traffic.
 //
 // The weight matrix is the MMA's M operand (128 output features per tile) and the
 // activation rows are its N operand, so every weight byte crosses HBM exactly once per
 // step however many rows are verified.  Work is the flat list of (tile, 64-wide k-chunk)
 // pairs, cut into equal contiguous ranges, one per CTA; partial tiles are summed in a fixed
 // order that depends on the matrix shape and grid only -- never on the rows in use.
+//
+// Two kernels share the fused epilogues: gemm_ws_kernel<NR> for engines of at most 32 rows (NR = 16
+// or 32 fixed per engine; activation tiles copied by loader warps) and gemm_wide_kernel for up to
+// 256 rows (activation tiles by TMA, MMA N = the rows in use rounded up to 16, epilogue in blocks of
+// 32 rows).
 #pragma once
 #include <cuda.h>
 
@@ -23,7 +29,7 @@ enum GemmMode : int32_t {
     kGemmResid = 1,   // x[r, n] += acc
     kGemmSwiGLU = 2,  // A maps = {w_gate, w_up}, 64 + 64 rows per tile; h = silu(g) * u (bf16)
     kGemmLmHead = 3,  // per-tile (max, argmax) per row; optional logits store
-    kGemmStore = 4,   // out[r, n] = acc for all 32 rows (stand-alone product)
+    kGemmStore = 4,   // out[r, n] = acc for all rows (stand-alone product)
 };
 
 struct GemmArgs {
@@ -32,55 +38,68 @@ struct GemmArgs {
     int32_t n_tiles;        // tiles over all matrices
     int32_t chunks;         // k_in / 64
     int32_t tiles_per_map;  // tiles per A map
-    const RowDesc* rows;    // nullptr: all 32 rows are in use
-    const void* act;        // activation operand, ActLayout kActSplit [2 * kMaxRows][k_in] bf16
-    float* ws;              // partial tiles [grid][2][128][32] fp32; slot 1 of every CTA all-ones (empty) at launch
-    int32_t* cnt;           // unused by the kernel (kept for the layout of callers' scratch)
+    const RowDesc* rows;    // nullptr: all nr rows are in use
+    const void* act;        // activation operand, ActLayout kActSplit(3) [terms * rc][k_in] bf16
+    int32_t rc;             // row capacity of the activation buffers and per-row scratch arrays
+    int32_t nr;             // rows the launch is shaped for (wide kernel: multiple of 16, <= 256)
+    int32_t terms;          // bf16 terms of the activation operand that are multiplied (2 or 3)
+    float* ws;              // partial tiles [grid][2][nr / 4][128] float4; slot 1 of every CTA all-ones (empty) at launch
     int32_t* dev_err;
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
     int32_t ld;             // leading dimension of out_f32
-    void* out_act;          // SwiGLU: h in ActLayout kActSplit [64][d_ffn]
+    void* out_act;          // SwiGLU: h in ActLayout kActSplit [2 rc][d_ffn]
     // RMSNorm folded into the projections: the producer of the residual stream x writes
     // xs = split(x * gain) and, per 128-column tile, the rows' sums of squares; the consumer
     // multiplies its accumulators by rsqrt(sum / norm_dim + eps), which equals projecting the
     // normalised row because the scale is one number per row.
-    const float* ss_in;     // consumer: [ss_tiles][32] partial sums of squares, or nullptr
+    const float* ss_in;     // consumer: [ss_tiles][rc] partial sums of squares, or nullptr
     int32_t ss_tiles;
     int32_t norm_dim;
     float norm_eps;
     const float* gain_next; // Resid producer: gain of the next norm [n_out], with xs_out / ss_out
-    void* xs_out;           // ActLayout kActSplit [64][n_out], or nullptr
-    float* ss_out;          // [n_tiles][32]
+    void* xs_out;           // ActLayout xs_layout [terms * rc][n_out], or nullptr
+    int32_t xs_layout;      // kActSplit or kActSplit3
+    float* ss_out;          // [n_tiles][rc]
     // QKV
     ModelDims dims;
     int32_t layer;
     const float *rope_cos, *rope_sin;
     __nv_bfloat16 *kcache, *vcache;
     // LmHead
-    float* part_max;        // [n_tiles][32]
+    float* part_max;        // [n_tiles][rc]
     int32_t* part_idx;
 };
 
-constexpr int kGemmN = 2 * kMaxRows;  // rows of a split activation buffer: hi rows then lo rows
 constexpr int kGemmThreads = 320;  // 4 epilogue warps, TMA producer, MMA issuer, 4 activation-loader warps
+constexpr int kGemmWideThreads = 224;  // 4 epilogue warps, weight producer, MMA issuer, activation producer
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 
-// The kernel exists for NR = 16 or 32 activation rows per half (MMA N = 2 NR).  Ring depths are the
-// ones measured fastest inside a decoding step (8 stages at NR 16, 6 at NR 32; deeper rings only
+// gemm_ws_kernel exists for NR = 16 or 32 activation rows and NT = 2 or 3 terms (MMA N = NR, issued once
+// per term).  Ring depths are the ones measured fastest inside a decoding step (deeper rings only
 // lengthen the queues that the epilogue's traffic also waits in).  The activation tile of a stage
-// is NOT fetched by TMA: a second, small TMA copy per stage slowed the weight stream by a
+// is NOT fetched by TMA here: a second, small TMA copy per stage slowed the weight stream by a
 // quarter wherever it came from (shared buffer, per-CTA replica, one hot 4 KB block), whereas
 // plain loads by otherwise idle warps cost almost nothing.  Four loader warps take turns copying
 // the rows from global memory into the 128-byte-swizzled layout the MMA expects.
 // The request is padded to more than half an SM's shared memory so that the CTAs of two
 // consecutive projections never share an SM (measured 10 % slower when they do).
-template <int NR> struct GemmCfg {
-    static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
-    static constexpr int kStages = NR == 16 ? 8 : 6;
-    static constexpr size_t kRopeBytes = kMaxRows * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
+template <int NR, int NT> struct GemmCfg {
+    static constexpr uint32_t kBBytes = NT * NR * 64 * 2;
+    static constexpr int kStages = NR == 16 ? 8 : (NT == 2 ? 7 : 6);
+    static constexpr size_t kRopeBytes = 32 * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
     static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
+
+// Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight tiles (16 KB each) and a ring of
+// activation tiles (nr rows of 128 bytes each: one term of one 64-wide k-chunk), as many as fit.
+struct GemmWideCfg {
+    uint32_t b_slot;    // bytes of one activation tile
+    int sa, sb;         // ring depths (each at most 8)
+    uint32_t tmem_cols; // power of two >= 2 nr (two accumulators)
+    size_t smem_bytes;
+};
+GemmWideCfg gemm_wide_cfg(int nr);
 
 // grid size used for a problem with `work` = n_tiles * chunks (a function of the shape only)
 int gemm_grid_for(int64_t work, int num_sms);
@@ -92,13 +111,15 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-// nr = 16 or 32 activation rows per half; pdl = launch with programmatic stream serialization (the
-// kernel before it must be one of this library's)
-void launch_gemm_tcgen05(cudaStream_t st, int grid, int nr, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+// args.nr = 16 or 32 rows, args.terms = 2 or 3; pdl = launch with programmatic stream serialization
+// (the kernel before it must be one of this library's)
+void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2);
 
-// out_tok[r] = index of the largest logit over all tiles (lowest index on ties)
-void launch_argmax_final(cudaStream_t st, bool pdl, const RowDesc* rows, const float* part_max, const int32_t* part_idx,
-                         int32_t n_tiles, int32_t* out_tok);
+// args.nr = 16 .. 256 (multiple of 16); map_b covers the activation buffer [terms * rc][k_in] with a
+// {64, nr} box
+cudaError_t init_gemm_wide();
+void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& map_b);
 
 }  // namespace llma

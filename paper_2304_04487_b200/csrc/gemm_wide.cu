@@ -1,0 +1,389 @@
+// Weight-streaming GEMM for up to 256 activation rows (batched decoding steps, prompt passes).
+// Same contract, work split and fused epilogues as gemm_ws_kernel (see gemm_tcgen05.cuh); what differs:
+//   * the activation tiles are large enough for TMA to pay: a second producer thread streams them
+//     through a ring of their own (one slot = nr rows x 64 columns of ONE bf16 term), so the number of
+//     terms does not change the depth of the weight ring;
+//   * MMA N = the rows in use rounded up to 16 (a run-time field of the instruction descriptor);
+//   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
+//
+// Roles inside one CTA of 224 threads:
+//   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue, block by block
+//   warp  4    one thread issues the TMA loads of the weight tiles (they depend on no earlier kernel)
+//   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
+//   warp  6    one thread issues the TMA loads of the activation tiles (after the dependency wait)
+//
+// Every wait is bounded: when one runs out the kernel raises the device error word, stops
+// issuing work, lets its outstanding copies land, frees TMEM and returns.
+#include <cuda.h>
+
+#include "gemm_epilogue.cuh"
+#include "gemm_tcgen05.cuh"
+#include "ptx_sm100.cuh"
+
+namespace llma {
+
+using namespace ptx;
+
+constexpr size_t kWideStageBytes = 128 * 33 * 4;
+constexpr size_t kWideTailBytes = 5120;  // barriers, flags, per-row scales, reduction scratch, row positions and slots
+
+template <int MODE>
+__global__ void __launch_bounds__(kGemmWideThreads, 1)
+gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
+                 const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
+                 const int SA, const int SB, const uint32_t tmem_cols) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const int nr = g.nr, NT = g.terms;
+    const uint32_t b_slot = (uint32_t)nr * 128u;
+    const uint32_t sA = base, sB = base + (uint32_t)SA * kGemmABytes;
+    uint8_t* after = gen_base + (size_t)SA * kGemmABytes + (size_t)SB * b_slot;
+    float (*stage)[33] = reinterpret_cast<float (*)[33]>(after);
+    uint8_t* tail = after + kWideStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full_a[8], empty_a[8], full_b[8], empty_b[8], acc_full[2], acc_empty[2]
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + 36 * 8);  // [0] TMEM base, [1] abort, [2] broadcast
+    float* rscale = reinterpret_cast<float*>(tail + 36 * 8 + 16);                 // [256] per-row norm scales
+    float* red_f = rscale + kRowCap;                                              // [4][32]
+    int* red_i = reinterpret_cast<int*>(red_f + 128);                             // [4][32]
+    int* s_pos = red_i + 128;                                                     // [256] (QKV mode)
+    int* s_seq = s_pos + kRowCap;                                                 // [256]
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_a = [&](int s) { return bar0 + 8u * s; };
+    auto empty_a = [&](int s) { return bar0 + 8u * (8 + s); };
+    auto full_b = [&](int s) { return bar0 + 8u * (16 + s); };
+    auto empty_b = [&](int s) { return bar0 + 8u * (24 + s); };
+    auto accf_bar = [&](int i) { return bar0 + 8u * (32 + i); };
+    auto acce_bar = [&](int i) { return bar0 + 8u * (34 + i); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x, b = blockIdx.x;
+    const int C = g.chunks;
+    const int64_t work = (int64_t)g.n_tiles * C;
+    const int64_t w_beg = cta_begin(work, b, G), w_end = cta_begin(work, b + 1, G);
+    const int64_t n_items = w_end - w_beg;
+
+    grid_launch_dependents();  // the next kernel may begin its own prologue now
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 8; ++s) {
+            mbar_init(full_a(s), 1); mbar_init(empty_a(s), 1); mbar_init(full_b(s), 1); mbar_init(empty_b(s), 1);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(accf_bar(i), 1); mbar_init(acce_bar(i), 4); }
+        sh[1] = 0; sh[2] = 0;
+        fence_mbar_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32((const void*)&sh[0]), tmem_cols);
+        tmem_relinquish();
+    }
+    if (warp == 4 && lane == 0) {
+        tma_prefetch_desc(&map_a0);
+        if (MODE == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
+        if (MODE == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
+    }
+    if (warp == 6 && lane == 0) tma_prefetch_desc(&map_b);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh[0];
+
+    if (warp == 4) {
+        // ------------------------------- weight producer -----------------------------------------
+        if (lane == 0) {
+            int64_t it = 0;
+            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w, ++it) {
+                const int s = (int)(it % SA);
+                const uint32_t ph = (uint32_t)((it / SA) & 1);
+                if (it >= SA && !mbar_wait(empty_a(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                mbar_arrive_expect_tx(full_a(s), kGemmABytes);
+                const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
+                const uint32_t dstA = sA + s * kGemmABytes;
+                if (MODE == kGemmSwiGLU) {
+                    tma_load_2d(dstA, &map_a0, full_a(s), c * 64, tile * 64);
+                    tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_a(s), c * 64, tile * 64);
+                } else {
+                    const int m = tile / g.tiles_per_map, r0 = (tile % g.tiles_per_map) * 128;
+                    const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
+                    tma_load_2d(dstA, mp, full_a(s), c * 64, r0);
+                }
+            }
+            if (sh[1]) {  // give up: let the copies already issued land before the CTA's memory goes away
+                const int64_t first = it > SA ? it - SA : 0;
+                for (int64_t j = first; j < it; ++j)
+                    (void)mbar_wait(full_a((int)(j % SA)), (uint32_t)((j / SA) & 1), 100000000ull);
+            }
+        }
+    } else if (warp == 6) {
+        // ------------------------------- activation producer ---------------------------------------
+        if (lane == 0) {
+            grid_dependency_wait();  // activations are written by the kernel before this one
+            int64_t it = 0;          // counts (item, term) pairs
+            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w) {
+                const int c = (int)(w % C);
+                for (int t = 0; t < NT; ++t, ++it) {
+                    const int s = (int)(it % SB);
+                    const uint32_t ph = (uint32_t)((it / SB) & 1);
+                    if (it >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    mbar_arrive_expect_tx(full_b(s), b_slot);
+                    tma_load_2d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, t * g.rc);
+                }
+                if (sh[1]) break;
+            }
+            if (sh[1]) {
+                const int64_t first = it > SB ? it - SB : 0;
+                for (int64_t j = first; j < it; ++j)
+                    (void)mbar_wait(full_b((int)(j % SB)), (uint32_t)((j / SB) & 1), 100000000ull);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------- MMA issuer ---------------------------------------------
+        if (lane == 0) {
+            grid_dependency_wait();  // the count of rows in use comes from the planning kernel
+            int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : nr;
+            rows_used = max(1, min(rows_used, nr));
+            const uint32_t idesc = idesc_bf16_m128((uint32_t)((rows_used + 15) & ~15));
+            int64_t ia = 0, ib = 0;
+            int seg = 0;
+            for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
+                const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
+                const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
+                const int buf = seg & 1;
+                const uint32_t use = (uint32_t)(seg >> 1);
+                if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)nr;
+                for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
+                    const int s = (int)(ia % SA);
+                    if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
+                    for (int t = 0; t < NT; ++t, ++ib) {
+                        const int sb = (int)(ib % SB);
+                        if (!mbar_wait(full_b(sb), (uint32_t)((ib / SB) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                        tc_fence_after();
+                        const uint64_t db = smem_desc_sw128(sB + (uint32_t)sb * b_slot);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
+                        umma_commit(empty_b(sb));  // slot is free once these MMAs have read it
+                    }
+                    if (sh[1]) break;
+                    umma_commit(empty_a(s));
+                }
+                if (sh[1]) break;
+                umma_commit(accf_bar(buf));  // accumulator complete
+                w += c1 - c0;
+            }
+        }
+    } else {
+        // ------------------------------- epilogue warps ------------------------------------------
+        grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
+        const int rows_used = g.rows ? min(g.rows->rows_used, nr) : nr;
+        const int nblk = (rows_used + 31) >> 5;
+        const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
+        if (g.ss_in) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
+            for (int r = row; r < rows_used; r += 128) {
+                float ssum = 0.f;
+                int t = 0;
+                for (; t + 8 <= g.ss_tiles; t += 8) {  // eight loads in flight
+                    float v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = __ldcg(&g.ss_in[(int64_t)(t + u) * g.rc + r]);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) ssum += v[u];
+                }
+                for (; t < g.ss_tiles; ++t) ssum += __ldcg(&g.ss_in[(int64_t)t * g.rc + r]);
+                rscale[r] = rsqrtf(ssum / (float)g.norm_dim + g.norm_eps);
+            }
+        }
+        if (MODE == kGemmQKV) {  // the rows' positions and sequence slots, read once per CTA
+            for (int r = row; r < rows_used; r += 128) {
+                s_pos[r] = __ldcg(&g.rows->pos[r]);
+                s_seq[r] = __ldcg(&g.rows->seq[r]);
+            }
+        }
+        epi_sync();
+        const float xnone[kXPre] = {};
+        // stage a 32-row block in shared memory (scaled by the folded RMSNorm), then the fused epilogue
+        auto finish_block = [&](int tile, int rb, float (&acc)[32]) {
+            const int jb = rb * 32, nj = min(32, rows_used - jb);
+            if (g.ss_in) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[min(jb + j, kRowCap - 1)];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
+            }
+            epi_sync();
+            if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, jb, nj, stage, s_pos, s_seq, nullptr);
+            else if constexpr (MODE == kGemmResid) epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
+            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, jb, nj, stage);
+            else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, jb, nj, stage);
+            else epilogue_lmhead(g, tile, row, jb, nj, stage, red_f, red_i);
+            epi_sync();  // the staging area is rewritten by the next block
+        };
+        // Tiles cut by a range boundary: see gemm_ws_kernel.  The hand-over slots hold nr / 4 row groups.
+        constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+        const int qn = nr >> 2;
+        int own_tile = -1, own_first = 0;
+        bool aborted = false;
+        int seg = 0;
+        for (int64_t w = w_beg; w < w_end; ++seg) {
+            const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
+            const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
+            w += c1 - c0;
+            const int buf = seg & 1;
+            const uint32_t use = (uint32_t)(seg >> 1);
+            if (threadIdx.x == 0) {
+                bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
+                if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
+                sh[2] = ok ? 1u : 0u;
+            }
+            epi_sync();
+            const bool ok = sh[2] != 0;
+            epi_sync();
+            if (!ok) { aborted = true; break; }
+            tc_fence_after();
+            const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
+            const bool shared_tile = w_beg > t_lo || w_end < t_hi;
+            const bool owner = w_end >= t_hi;
+            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)nr;
+            for (int rb = 0; rb < nblk; ++rb) {
+                float acc[32];
+                tmem_ld_32cols(t0 + (uint32_t)rb * 32u, acc);
+                if (shared_tile) {
+                    float4* dst = ws_slot(g.ws, qn, b, owner ? 0 : 1, row) + (int64_t)rb * 8 * 128;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)  // only the columns of rows in use travel
+                        if (rb * 32 + 4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                } else {
+                    finish_block(tile, rb, acc);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
+            if (shared_tile && owner) {
+                int b_first = (int)(t_lo * G / work);
+                while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
+                while (cta_begin(work, b_first, G) > t_lo) --b_first;
+                own_tile = tile; own_first = b_first;
+            }
+        }
+        if (own_tile >= 0 && !aborted) {
+            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
+            bool timed_out = false;
+            for (int rb = 0; rb < nblk; ++rb) {
+                const int jb = rb * 32;
+                float acc[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                for (int bb = own_first; bb < b; ++bb) {  // ascending k: a fixed summation order
+                    const float4* src = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
+                    float4 p[8];
+                    bool valid;
+                    do {
+                        valid = true;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            if (jb + 4 * q < rows_used) {
+                                valid = valid && __float_as_uint(p[q].x) != kEmpty;
+                                if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
+                                if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
+                                if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
+                            }
+                        }
+                        if (!valid && (timed_out || globaltimer_ns() > give_up)) {
+                            atomicExch(g.dev_err, kDevErrTimeout); timed_out = true; break;
+                        }
+                    } while (!valid);
+                    const float e = __uint_as_float(kEmpty);
+                    float4* wr = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (jb + 4 * q < rows_used) {
+                            wr[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
+                            acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
+                        }
+                    }
+                }
+                // this CTA's own partial comes last (it holds the highest k)
+                const float4* mine = ws_slot(g.ws, qn, b, 0, row) + (int64_t)rb * 8 * 128;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (jb + 4 * q < rows_used) {
+                        const float4 o = mine[q * 128];
+                        acc[4 * q] += o.x; acc[4 * q + 1] += o.y; acc[4 * q + 2] += o.z; acc[4 * q + 3] += o.w;
+                    }
+                }
+                finish_block(own_tile, rb, acc);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+GemmWideCfg gemm_wide_cfg(int nr) {
+    GemmWideCfg c;
+    c.b_slot = (uint32_t)nr * 128u;
+    const size_t budget = (size_t)227 * 1024 - 1024 - kWideStageBytes - kWideTailBytes;
+    // four weight tiles in flight first, then as many activation tiles as fit, then more weight tiles
+    c.sb = (int)((budget - 4 * kGemmABytes) / c.b_slot);
+    if (c.sb > 8) c.sb = 8;
+    c.sa = (int)((budget - (size_t)c.sb * c.b_slot) / kGemmABytes);
+    if (c.sa > 8) c.sa = 8;
+    uint32_t cols = 32;
+    while (cols < 2u * (uint32_t)nr) cols <<= 1;
+    c.tmem_cols = cols;
+    c.smem_bytes = 1024 + (size_t)c.sa * kGemmABytes + (size_t)c.sb * c.b_slot + kWideStageBytes + kWideTailBytes;
+    if (c.smem_bytes < 120 * 1024) c.smem_bytes = 120 * 1024;  // one CTA per SM, as for the narrow kernel
+    return c;
+}
+
+template <int MODE>
+static cudaError_t wide_opt_in() {
+    return cudaFuncSetAttribute(gemm_wide_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+cudaError_t init_gemm_wide() {
+    cudaError_t e;
+    if ((e = wide_opt_in<kGemmQKV>()) != cudaSuccess) return e;
+    if ((e = wide_opt_in<kGemmResid>()) != cudaSuccess) return e;
+    if ((e = wide_opt_in<kGemmSwiGLU>()) != cudaSuccess) return e;
+    if ((e = wide_opt_in<kGemmLmHead>()) != cudaSuccess) return e;
+    return wide_opt_in<kGemmStore>();
+}
+
+void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
+                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& map_b) {
+    const GemmWideCfg c = gemm_wide_cfg(args.nr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kGemmWideThreads);
+    cfg.dynamicSmemBytes = c.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const int sa = c.sa, sb = c.sb;
+    const uint32_t cols = c.tmem_cols;
+    switch (args.mode) {
+        case kGemmQKV: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmQKV>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+        case kGemmResid: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmResid>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmSwiGLU>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+        case kGemmLmHead: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmLmHead>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+        default: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmStore>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+    }
+}
+
+}  // namespace llma

@@ -12,13 +12,13 @@ namespace llma {
 // ---- RMSNorm -----------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const RowDesc* __restrict__ rows, const float* __restrict__ x,
                                                       const float* __restrict__ g, void* __restrict__ out, int layout,
-                                                      int d, float eps) {
+                                                      int rc, int d, float eps) {
     pdl_trigger();
     pdl_wait();
     const int r = blockIdx.x;
     const float* xr = x + (int64_t)r * d;
     if (rows->pos[r] < 0) {
-        for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, r, i, d, 0.f);
+        for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, rc, r, i, d, 0.f);
         return;
     }
     float ss = 0.f;
@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const RowDesc* __restrict_
     float tot = 0.f;
     for (int w = 0; w < 8; ++w) tot += red[w];  // fixed order
     const float inv = rsqrtf(tot / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, r, i, d, xr[i] * inv * g[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) store_act(out, layout, rc, r, i, d, xr[i] * inv * g[i]);
 }
 
 // ---- small-M GEMM: one warp per output feature --------------------------------------------
@@ -148,9 +148,9 @@ __global__ void __launch_bounds__(256) argmax_kernel(const RowDesc* __restrict__
 }
 
 // ---- launchers -------------------------------------------------------------------------------
-void launch_rmsnorm(cudaStream_t st, int act_layout, const RowDesc* rows, const float* x, const float* g, void* x_hat,
-                    int32_t d, float eps) {
-    launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, rmsnorm_kernel, rows, x, g, x_hat, act_layout, d, eps);
+void launch_rmsnorm(cudaStream_t st, int act_layout, int n_rows, int rc, const RowDesc* rows, const float* x,
+                    const float* g, void* x_hat, int32_t d, float eps) {
+    launch_pdl(st, true, dim3(n_rows), dim3(256), 0, rmsnorm_kernel, rows, x, g, x_hat, act_layout, rc, d, eps);
 }
 
 void launch_gemm_simt(cudaStream_t st, bool bf16, const RowDesc* rows, const void* W, const float* a, float* out,
@@ -162,13 +162,13 @@ void launch_gemm_simt(cudaStream_t st, bool bf16, const RowDesc* rows, const voi
         launch_pdl(st, true, dim3(blocks), dim3(256), 0, gemm_simt_kernel<float, 8>, rows, (const float*)W, a, out, n_out, k_in, ld_out, accumulate ? 1 : 0);
 }
 
-void launch_silu_mul(cudaStream_t st, const RowDesc* rows, const float* gate_up, float* h, int32_t d_ffn) {
-    dim3 grid((d_ffn + 255) / 256, kMaxRows);
+void launch_silu_mul(cudaStream_t st, int n_rows, const RowDesc* rows, const float* gate_up, float* h, int32_t d_ffn) {
+    dim3 grid((d_ffn + 255) / 256, n_rows);
     launch_pdl(st, true, grid, dim3(256), 0, silu_mul_kernel, rows, gate_up, h, d_ffn);
 }
 
-void launch_argmax(cudaStream_t st, const RowDesc* rows, const float* logits, int32_t vocab, int32_t* out_tok) {
-    launch_pdl(st, true, dim3(kMaxRows), dim3(256), 0, argmax_kernel, rows, logits, vocab, out_tok);
+void launch_argmax(cudaStream_t st, int n_rows, const RowDesc* rows, const float* logits, int32_t vocab, int32_t* out_tok) {
+    launch_pdl(st, true, dim3(n_rows), dim3(256), 0, argmax_kernel, rows, logits, vocab, out_tok);
 }
 
 }  // namespace llma

@@ -52,59 +52,79 @@ def logits_close(got: np.ndarray, want: np.ndarray, mode: str, n_layers: int = 1
 
 def step_parity(eng, oracle_model, prompt: Sequence[int], ref: Sequence[int], offs: Optional[Sequence[int]],
                 n: int, k: int, n_new: int, mode: str, seq: int = 0, tie_margin: float = 1e-3) -> ParityReport:
-    """Drive ``eng.llma_step`` and the oracle side by side for ``n_new`` tokens."""
-    rep = ParityReport()
-    ref = [int(t) for t in ref]
-    kp1 = eng.max_k + 1
-    eng.llma_prefill(seq, prompt)
-    eng.llma_set_reference(seq, ref, offs)
-    L, pending = D.prefill(oracle_model, prompt)
-    assert eng.llma_kv_len(seq) == L
-    y: List[int] = []
-    while len(y) < n_new:
-        matched, pos, _ = D.match_ngrams(y, ref, offs, n)
-        k_eff = D.copy_length(pos, len(ref), offs, k, eng.max_seq - L) if matched else 0
-        inputs = [pending] + (ref[pos:pos + k_eff] if k_eff > 0 else [])
-        want_rows = np.stack([oracle_model.forward(tok, L + j) for j, tok in enumerate(inputs)])
-        outs = want_rows.argmax(1).tolist()
-        a = 0
-        while a < k_eff and outs[a] == ref[pos + a]:
-            a += 1
-        want_tokens = outs[:a + 1]
+    """Drive ``eng.llma_step`` and the oracle side by side for ``n_new`` tokens of one sequence."""
+    assert seq == 0
+    return step_parity_batch(eng, [oracle_model], [prompt], [ref], [offs], n, k, n_new, mode, tie_margin)[0]
 
-        got_tokens = eng.llma_step(n, k)[seq]
-        info = eng.llma_last_step_info()[seq]
-        assert info.k_eff == k_eff, (rep.steps, info.k_eff, k_eff)
-        assert info.pos == (pos if k_eff > 0 else -1), (rep.steps, info.pos, pos)
-        got_rows = eng.llma_debug_logits()[seq * kp1: seq * kp1 + k_eff + 1]
-        for j in range(k_eff + 1):
-            rep.max_logit_err = max(rep.max_logit_err, logits_close(got_rows[j], want_rows[j], mode, eng.shape.n_layers))
-            rep.max_logit_scale = max(rep.max_logit_scale, float(np.abs(want_rows[j]).max()))
-        rep.rows_compared += k_eff + 1
-        # the engine's acceptance must be Algorithm 1 applied to its own argmaxes
-        gouts = got_rows.argmax(1).tolist()
-        ga = 0
-        while ga < k_eff and gouts[ga] == ref[pos + ga]:
-            ga += 1
-        assert got_tokens == gouts[:ga + 1], (rep.steps, got_tokens, gouts, ga)
-        assert info.accepted == ga and info.emitted == ga + 1
-        if got_tokens != want_tokens:
-            common = min(len(got_tokens), len(want_tokens))
-            diff = [i for i in range(common) if got_tokens[i] != want_tokens[i]]
-            # both sides apply Algorithm 1's acceptance rule to their own argmaxes on the same copied
-            # tokens, so two token lists that agree on their common prefix have the same length
-            assert diff, f"step {rep.steps}: equal prefixes but {len(got_tokens)} vs {len(want_tokens)} tokens"
-            j = diff[0]
-            srt = np.sort(want_rows[j])
-            margin = float(srt[-1] - srt[-2])
-            assert margin < tie_margin, f"tokens differ at step {rep.steps} row {j} with oracle margin {margin:.3e}"
-            rep.near_ties += 1
-        y.extend(got_tokens)
-        L += len(got_tokens)
-        pending = got_tokens[-1]
-        assert eng.llma_kv_len(seq) == L
-        rep.steps += 1
-        rep.trigger_steps += int(k_eff > 0)
-        rep.copied_accepted += len(got_tokens) - 1
-    rep.tokens = y
-    return rep
+
+def step_parity_batch(eng, oracle_models, prompts, refs, offs_list, n: int, k: int, n_new: int, mode: str,
+                      tie_margin: float = 1e-3) -> List[ParityReport]:
+    """Several sequences decoded together by ``eng.llma_step`` (one forward pass per step for all of
+    them), each compared with its own oracle run: integer results per step, every logits row, tokens.
+    Runs until every sequence has at least ``n_new`` tokens."""
+    B = len(prompts)
+    reps = [ParityReport() for _ in range(B)]
+    refs = [[int(t) for t in r] for r in refs]
+    kp1 = eng.max_k + 1
+    L, pending, ys = [0] * B, [0] * B, [[] for _ in range(B)]
+    for s in range(B):
+        eng.llma_prefill(s, prompts[s])
+        eng.llma_set_reference(s, refs[s], offs_list[s])
+        L[s], pending[s] = D.prefill(oracle_models[s], prompts[s])
+        assert eng.llma_kv_len(s) == L[s]
+    while min(len(y) for y in ys) < n_new:
+        want = []
+        for s in range(B):
+            ref, offs, y = refs[s], offs_list[s], ys[s]
+            matched, pos, _ = D.match_ngrams(y, ref, offs, n)
+            k_eff = D.copy_length(pos, len(ref), offs, k, eng.max_seq - L[s]) if matched else 0
+            inputs = [pending[s]] + (ref[pos:pos + k_eff] if k_eff > 0 else [])
+            rows = np.stack([oracle_models[s].forward(tok, L[s] + j) for j, tok in enumerate(inputs)])
+            want.append((pos, k_eff, rows))
+        got_all = eng.llma_step(n, k)
+        infos = eng.llma_last_step_info()
+        logits = eng.llma_debug_logits()
+        for s in range(B):
+            rep, ref = reps[s], refs[s]
+            pos, k_eff, want_rows = want[s]
+            outs = want_rows.argmax(1).tolist()
+            a = 0
+            while a < k_eff and outs[a] == ref[pos + a]:
+                a += 1
+            want_tokens = outs[:a + 1]
+            got_tokens, info = got_all[s], infos[s]
+            assert info.k_eff == k_eff, (s, rep.steps, info.k_eff, k_eff)
+            assert info.pos == (pos if k_eff > 0 else -1), (s, rep.steps, info.pos, pos)
+            got_rows = logits[s * kp1: s * kp1 + k_eff + 1]
+            for j in range(k_eff + 1):
+                rep.max_logit_err = max(rep.max_logit_err, logits_close(got_rows[j], want_rows[j], mode, eng.shape.n_layers))
+                rep.max_logit_scale = max(rep.max_logit_scale, float(np.abs(want_rows[j]).max()))
+            rep.rows_compared += k_eff + 1
+            # the engine's acceptance must be Algorithm 1 applied to its own argmaxes
+            gouts = got_rows.argmax(1).tolist()
+            ga = 0
+            while ga < k_eff and gouts[ga] == ref[pos + ga]:
+                ga += 1
+            assert got_tokens == gouts[:ga + 1], (s, rep.steps, got_tokens, gouts, ga)
+            assert info.accepted == ga and info.emitted == ga + 1
+            if got_tokens != want_tokens:
+                common = min(len(got_tokens), len(want_tokens))
+                diff = [i for i in range(common) if got_tokens[i] != want_tokens[i]]
+                # both sides apply Algorithm 1's acceptance rule to their own argmaxes on the same copied
+                # tokens, so two token lists that agree on their common prefix have the same length
+                assert diff, f"seq {s} step {rep.steps}: equal prefixes but {len(got_tokens)} vs {len(want_tokens)} tokens"
+                j = diff[0]
+                srt = np.sort(want_rows[j])
+                margin = float(srt[-1] - srt[-2])
+                assert margin < tie_margin, f"seq {s}: tokens differ at step {rep.steps} row {j} with oracle margin {margin:.3e}"
+                rep.near_ties += 1
+            ys[s].extend(got_tokens)
+            L[s] += len(got_tokens)
+            pending[s] = got_tokens[-1]
+            assert eng.llma_kv_len(s) == L[s]
+            rep.steps += 1
+            rep.trigger_steps += int(k_eff > 0)
+            rep.copied_accepted += len(got_tokens) - 1
+    for s in range(B):
+        reps[s].tokens = ys[s]
+    return reps

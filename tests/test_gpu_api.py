@@ -67,7 +67,7 @@ def test_unsupported_configs_rejected(setup):
     from paper_2304_04487_b200 import LlmaError
     Engine, shape, w = setup
     with pytest.raises(LlmaError) as ei:
-        Engine(shape, w, max_seq=32, max_ref=8, max_k=16, max_batch=2)   # 2 * 17 rows > 32
+        Engine(shape, w, max_seq=32, max_ref=8, max_k=16, max_batch=16)  # 16 * 17 rows > 256
     assert ei.value.status == -2
     with pytest.raises(LlmaError) as ei:
         Engine(shape, w, max_seq=32, max_ref=8, max_k=2, gemm_impl=2)    # tensor-core GEMM needs bf16

@@ -38,6 +38,13 @@ def test_noalloc_matches_allocating_entry_point_twice():
             scale = max(1.0, float(want.abs().max()))
             assert float((got - want).abs().max()) <= 1e-4 * scale, (n_out, k_in, attempt)
             assert torch.equal(got, want), (n_out, k_in, attempt)
+    # the point of the entry point: a warmed-up call leaves the device's free memory where it was
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    llma_gemm_rows32_bf16_noalloc(W, a, got)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
