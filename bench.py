@@ -38,6 +38,9 @@ WORKLOADS = {
     "mid-rag": ("mid-bf16", 256, [128, 128], 0.8, 1, 8, 128),
     "tiny-fp32": ("tiny-fp32", 128, [256], 0.6, 2, 4, 64),
 }
+# workloads with a driver of their own (see the functions of the same name below)
+OTHER_WORKLOADS = ("serve16", "layer-grid", "llama13b-sweep", "llama7b-trace", "serve16-small", "layer-grid-small",
+                   "sweep-small", "trace-small")
 METRIC = "tokens_per_s_llma_b1"
 UNIT = "tokens/s"
 
@@ -74,6 +77,21 @@ def max_over_ranks(values, device="cpu"):
 def replica_throughput(tokens_per_replica: int, world: int, slowest_seconds: float) -> float:
     """Whole-job tokens/s of `world` independent replicas (weak scaling: same work per GPU)."""
     return tokens_per_replica * world / slowest_seconds
+
+
+def per_class_roofline(shape, prof, kvbytes, peak):
+    """Algorithmic bytes, time and fraction of the HBM peak for every kernel class of a step."""
+    e = 2 if shape.dtype == "bf16" else 4
+    L, D, F, V, HD = shape.n_layers, shape.d_model, shape.d_ffn, shape.vocab, shape.n_heads * shape.head_dim
+    nbytes = {"gemm_qkv": L * 3 * HD * D * e, "gemm_o": L * D * HD * e, "gemm_gateup": L * 2 * F * D * e,
+              "gemm_down": L * D * F * e, "gemm_lmhead": V * D * e, "attn": kvbytes}
+    out = {}
+    for name, b in nbytes.items():
+        if name in prof and prof[name]["ms_per_step"] > 0:
+            ms = prof[name]["ms_per_step"]
+            out[name] = {"bytes": int(b), "ms": round(ms, 4), "gbs": round(b / (ms / 1e3) / 1e9, 1),
+                         "frac": round(b / (ms / 1e3) / 1e9 / peak, 3)}
+    return out
 
 
 def load_peaks():
@@ -165,7 +183,9 @@ def cpu_oracle_sample(shape, weights, n, k, budget_s=20.0):
 def run_reference(args, rank):
     if rank != 0:
         return
-    shape_name, P, docs, f, n, k, n_new = WORKLOADS[args.workload]
+    base = {"llama13b-sweep": "llama13b-rag", "sweep-small": "mid-rag", "serve16-small": "mid-rag",
+            "layer-grid-small": "mid-rag", "trace-small": "mid-rag"}.get(args.workload, args.workload)
+    shape_name, P, docs, f, n, k, n_new = WORKLOADS.get(base, WORKLOADS["llama7b-rag"])
     shape = SHAPES[shape_name]
     w = make_weights(shape, seed=0)
     vals = []
@@ -179,8 +199,327 @@ def run_reference(args, rank):
             "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "shape": shape.name, "n": n, "k": k, "n_new": n_new},
             "cpu_baseline": cb,
+            # a step of this arm is a bounded sample (a few dozen tokens after a short prompt); ms_per_step
+            # is that rate scaled to the workload's n_new tokens, not a measured full decode
+            "extrapolated": True,
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+# Further workloads.  Each prints one JSON line with the same keys as the default workload; `value` is
+# the workload's own headline figure, the details sit under a key named after the workload.
+# ---------------------------------------------------------------------------------------------------
+def _launches_per_pass(shape):
+    """Kernels of one decoding step on the tensor-core path: embedding gather, six per layer, LM head, step tail."""
+    return 6 * shape.n_layers + 3
+
+
+def _common_line(args, world, shape, value, unit, ms_per_step, config, launches):
+    return {"metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
+            "gpu_launches": int(launches)}
+
+
+def run_serve16(args, rank, local_rank, world, small=False):
+    """Multi-turn serving shape: 16 sequences with a long history each, a 512-token reference per sequence with
+    its own overlap, decoded together: one forward pass per step over the packed rows of all sequences."""
+    import torch
+    from paper_2304_04487_b200 import Engine
+    shape = SHAPES["mid-bf16" if small else "llama7b-shape"]
+    B, hist, R, n, k, N = (16, 300, 128, 1, 8, 48) if small else (16, 4096, 512, 1, 8, 128)
+    w = make_weights(shape, seed=0)
+    eng = Engine(shape, w, max_seq=hist + N + 32, max_ref=R, max_k=k, max_batch=B, device=f"cuda:{local_rank}")
+    t0 = time.perf_counter()
+    for s in range(B):
+        eng.llma_prefill(s, make_prompt(hist, shape.vocab, seed=100 + s))
+    t_pre = time.perf_counter() - t0
+    y_star, g0 = eng.llma_generate(N, 1, 0)
+    frng = np.random.Generator(np.random.Philox(key=[5, 0]))
+    fs = frng.uniform(0.7, 0.9, size=B)
+    refs = [build_reference(y_star[s], [R], float(fs[s]), shape.vocab, seed=s) for s in range(B)]
+    pinned = [torch.from_numpy(r[0].copy()).pin_memory().numpy() for r in refs]
+
+    def one(kk):
+        for s in range(B):
+            eng.llma_set_reference(s, pinned[s], refs[s][1])
+            eng.llma_rewind(s)
+        return eng.llma_generate(N, n, kk)
+
+    for _ in range(args.warmup):
+        toks, _ = one(k)
+        assert toks == y_star, "batched LLMA output differs from the engine's own greedy decode"
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    torch.cuda.synchronize()
+    dev_ms, passes, launches, trig, acc, wall0 = 0.0, 0, 0, 0, 0, time.perf_counter()
+    for _ in range(args.steps):
+        toks, st = one(k)
+        dev_ms += st.device_ms; launches += st.launches
+        passes += (st.launches - 1) // _launches_per_pass(shape)
+        trig += st.trigger_steps; acc += st.copied_accepted
+    torch.cuda.synchronize()
+    wall_s = time.perf_counter() - wall0
+    g_ms, g_passes = 0.0, 0
+    for _ in range(args.steps):
+        _, st = one(0)
+        g_ms += st.device_ms; g_passes += (st.launches - 1) // _launches_per_pass(shape)
+    clocks = sampler.stop()
+    dev_ms, wall_s, g_ms = max_over_ranks([dev_ms, wall_s, g_ms], device="cuda")
+    peak, peak_kind = load_peaks()
+    wbytes = shape.weight_bytes_per_step()
+    kvbytes = B * shape.kv_bytes_per_position() * (hist + N // 2)
+    step_ms = dev_ms / max(passes, 1)
+    value = replica_throughput(args.steps * B * N, world, dev_ms / 1e3)
+    line = _common_line(args, world, shape, value, UNIT, dev_ms / args.steps,
+                        {"workload": args.workload, "shape": shape.name, "batch": B, "history": hist, "reference": R,
+                         "overlap": "U[0.7,0.9] per sequence", "n": n, "k": k, "n_new": N, "replicas": world,
+                         "l2": "inputs (weights and K/V) larger than L2"}, launches)
+    line.update({"greedy_tokens_per_s": replica_throughput(args.steps * B * N, world, g_ms / 1e3),
+                 "speedup_vs_own_greedy": g_ms / dev_ms, "clocks": clocks, "prefill_s": t_pre,
+                 "e2e": {"value": replica_throughput(args.steps * B * N, world, wall_s), "unit": UNIT,
+                         "h2d_bytes_per_step": int(sum(r[0].nbytes + r[1].nbytes for r in refs)),
+                         "d2h_bytes_per_step": int(4 * B * N)},
+                 "roofline": {"bound": "hbm", "kernel": "whole step (weights once + K/V of 16 sequences)",
+                              "achieved": (wbytes + kvbytes) / (step_ms / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
+                              "frac": (wbytes + kvbytes) / (step_ms / 1e3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
+                              "traffic": None},
+                 "serve16": {"forward_passes_per_decode": passes / args.steps, "ms_per_forward_pass": step_ms,
+                             "greedy_ms_per_forward_pass": g_ms / max(g_passes, 1),
+                             "weight_bytes": wbytes, "kv_bytes_mid_decode": kvbytes,
+                             "tokens_per_pass": args.steps * B * N / max(passes, 1),
+                             "trigger_steps_per_decode": trig / args.steps, "accepted_per_decode": acc / args.steps}})
+    return line
+
+
+def run_layer_grid(args, rank, local_rank, world, small=False):
+    """One decoder layer at the 7B widths: latency of a verification step and HBM GB/s against the rows per
+    sequence (k + 1), the cached length and the batch.  Steps are replayed (every step feeds k + 1 rows per
+    sequence and keeps one token), so the cached length stays where the cell puts it."""
+    import torch
+    from paper_2304_04487_b200 import Engine
+    shape = SHAPES["mid-bf16" if small else "llama7b-1layer"]
+    if small:
+        shape = shape.with_layers(1)
+    kvs, rows_list, batches = ((200, 600), (1, 5, 9), (1, 4)) if small else ((512, 2048, 8192), (1, 2, 5, 9, 17), (1, 4, 16))
+    w = make_weights(shape, seed=0)
+    peak, peak_kind = load_peaks()
+    wbytes = shape.weight_bytes_per_step()
+    n_steps = 24
+    cells, launches, shared = [], 0, None
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_all = 0.0
+    for B in batches:
+        for rows in rows_list:
+            if B * rows > 256:
+                for kv in kvs:
+                    cells.append({"batch": B, "rows": rows, "kv": kv, "unsupported": "more than 256 rows per step"})
+                continue
+            for kv in kvs:
+                eng = Engine(shape, w if shared is None else None, max_seq=kv + n_steps + 8, max_ref=8, max_k=rows - 1,
+                             max_batch=B, device=f"cuda:{local_rank}", share_weights_with=shared)
+                shared = shared or eng
+                for s in range(B):
+                    eng.llma_prefill(s, make_prompt(kv + 1, shape.vocab, seed=200 + s))
+                target = make_prompt(n_steps, shape.vocab, seed=9).tolist()
+                trace = [(rows, 1)] * n_steps
+                best = None
+                for it in range(args.warmup + args.steps):
+                    for s in range(B):
+                        eng.llma_rewind(s)
+                    st = eng.llma_generate_forced(-1, trace, target)
+                    if it >= args.warmup:
+                        best = st.device_ms if best is None else min(best, st.device_ms)
+                        launches += st.launches; t_all += st.device_ms
+                ms = best / n_steps
+                kvb = B * shape.kv_bytes_per_position() * (kv + n_steps // 2)
+                cells.append({"batch": B, "rows": rows, "kv": kv, "us_per_step": 1e3 * ms,
+                              "gbs": (wbytes + kvb) / (ms / 1e3) / 1e9, "frac": (wbytes + kvb) / (ms / 1e3) / 1e9 / peak})
+                if eng is not shared:
+                    eng.llma_destroy()
+    clocks = sampler.stop()
+    ok = [c for c in cells if "gbs" in c]
+    best_cell = max(ok, key=lambda c: c["gbs"])
+    line = _common_line(args, world, shape, float(np.median([c["gbs"] for c in ok])), "GB/s", t_all / max(args.steps, 1),
+                        {"workload": args.workload, "shape": shape.name, "kv_lengths": list(kvs), "rows": list(rows_list),
+                         "batches": list(batches), "steps_per_cell": n_steps,
+                         "l2": "weights of the layer (405 MB) larger than L2"}, launches)
+    line["metric"] = "verify_step_hbm_gbs_median_over_cells"
+    line.update({"clocks": clocks,
+                 "roofline": {"bound": "hbm", "kernel": "one decoder layer (six kernels) + step tail",
+                              "achieved": best_cell["gbs"], "peak": peak, "unit": "GB/s", "frac": best_cell["frac"],
+                              "peak_kind": f"of {peak_kind}", "traffic": None, "cell": best_cell},
+                 "e2e": {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                         "note": "device-timed replay only"},
+                 "layer_grid": cells})
+    return line
+
+
+def run_sweep13b(args, rank, local_rank, world, small=False):
+    """The analogue of the paper's copy-length sweep (Fig. 4, Section 3.5) at the 13B widths: overlap x k."""
+    import torch
+    from paper_2304_04487_b200 import Engine
+    shape = SHAPES["mid-bf16" if small else "llama13b-shape"]
+    P, R, N = (200, 128, 64) if small else (2048, 1024, 256)
+    overlaps, ks = (0.2, 0.5, 0.8, 0.95), (4, 8, 16)
+    w = make_weights(shape, seed=0)
+    prompt = make_prompt(P, shape.vocab, seed=1)
+    max_seq = P + N + 32
+    eng8 = Engine(shape, w, max_seq=max_seq, max_ref=R, max_k=8, device=f"cuda:{local_rank}")
+    eng16 = Engine(shape, None, max_seq=max_seq, max_ref=R, max_k=16, device=f"cuda:{local_rank}", share_weights_with=eng8)
+    t0 = time.perf_counter()
+    eng8.llma_prefill(0, prompt)
+    t_pre = time.perf_counter() - t0
+    eng16.llma_prefill(0, prompt)
+    (y_star,), _ = eng8.llma_generate(N, 1, 0)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    greedy = {}
+    for name, eng in (("16rows", eng8), ("32rows", eng16)):
+        ms = []
+        for it in range(args.warmup + args.steps):
+            eng.llma_rewind(0)
+            (t,), st = eng.llma_generate(N, 1, 0)
+            assert t == y_star
+            if it >= args.warmup:
+                ms.append(st.device_ms)
+        greedy[name] = float(np.mean(ms))
+    table, launches, total_ms = [], 0, 0.0
+    for f in overlaps:
+        ref, offs, info = build_reference(y_star, [R], f, shape.vocab, seed=0)
+        for k in ks:
+            eng, gname = (eng8, "16rows") if k <= 8 else (eng16, "32rows")
+            eng.llma_set_reference(0, ref, offs)
+            ms, st = [], None
+            for it in range(args.warmup + args.steps):
+                eng.llma_rewind(0)
+                (t,), st = eng.llma_generate(N, 1, k)
+                assert t == y_star, "LLMA output differs from the engine's own greedy decode"
+                if it >= args.warmup:
+                    ms.append(st.device_ms); launches += st.launches
+            m = float(np.mean(ms)); total_ms += sum(ms)
+            table.append({"overlap": f, "k": k, "tokens_per_s": N / (m / 1e3), "speedup_vs_own_greedy": greedy["16rows"] / m,
+                          "speedup_vs_same_engine_greedy": greedy[gname] / m, "steps": int(st.steps),
+                          "tokens_per_step": N / st.steps, "trigger_steps": int(st.trigger_steps),
+                          "accepted": int(st.copied_accepted), "ms_per_step": m / st.steps,
+                          "placed_fraction": info["placed_fraction"]})
+    clocks = sampler.stop()
+    peak, peak_kind = load_peaks()
+    wbytes, kvbytes = shape.weight_bytes_per_step(), shape.kv_bytes_per_position() * (P + N // 2)
+    head = next(r for r in table if r["overlap"] == 0.8 and r["k"] == 8)
+    line = _common_line(args, world, shape, head["tokens_per_s"], UNIT, total_ms / max(args.steps, 1),
+                        {"workload": args.workload, "shape": shape.name, "prompt": P, "reference": R, "n": 1,
+                         "overlaps": list(overlaps), "ks": list(ks), "n_new": N, "headline": "overlap 0.8, k 8",
+                         "l2": "inputs (weights) larger than L2"}, launches)
+    line.update({"clocks": clocks, "prefill_s": t_pre, "greedy_tokens_per_s": N / (greedy["16rows"] / 1e3),
+                 "greedy_tokens_per_s_32row_engine": N / (greedy["32rows"] / 1e3),
+                 "roofline": {"bound": "hbm", "kernel": "whole step at overlap 0.8, k 8",
+                              "achieved": (wbytes + kvbytes) / (head["ms_per_step"] / 1e3) / 1e9, "peak": peak, "unit": "GB/s",
+                              "frac": (wbytes + kvbytes) / (head["ms_per_step"] / 1e3) / 1e9 / peak,
+                              "peak_kind": f"of {peak_kind}", "traffic": None},
+                 "e2e": {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                         "note": "device-timed sweep; the end-to-end figure is the default workload's"},
+                 "paper_context": {"fig4b_13b_rag_speedup_n1": {"k4": 2.03, "k8": 2.31, "k14": 2.47, "k18": 2.46},
+                                   "note": "the paper's numbers: LLaMA-13B fp16 on V100s, its own data; context only"},
+                 "sweep": table})
+    eng16.llma_destroy()
+    return line
+
+
+def fig5_like_trace(n_tokens, steps, accepted, plain_steps, k, seed=0):
+    """A step sequence with the paper's Fig. 5 statistics (retrieval-augmented set, n = 1): `plain_steps`
+    one-token steps, the other steps feed k + 1 rows and keep 1 + a_i tokens with the a_i summing to
+    `accepted`; steps + accepted = n_tokens."""
+    rng = np.random.Generator(np.random.Philox(key=[7, seed]))
+    trig = steps - plain_steps
+    a = np.zeros(trig, np.int64)
+    for _ in range(accepted):                       # deal the accepted tokens over the trigger steps, at most k each
+        while True:
+            i = int(rng.integers(0, trig))
+            if a[i] < k:
+                a[i] += 1
+                break
+    kinds = np.array([0] * plain_steps + [1] * trig)
+    rng.shuffle(kinds)
+    out, it = [], iter(a.tolist())
+    for kd in kinds:
+        out.append((1, 1) if kd == 0 else (k + 1, 1 + next(it)))
+    assert sum(o for _, o in out) == n_tokens == steps + accepted
+    return out
+
+
+def run_trace(args, rank, local_rank, world, small=False):
+    """Target-guided replay (Section 3.2, Algorithm 2): the engine is driven along a step sequence with the
+    statistics the paper reports for its retrieval-augmented set at n = 1, k = 8 (Fig. 5: 37.62 steps, 32.11 of
+    them triggered, 73.61 accepted tokens, 111.2 output tokens after a ~900-token prompt), against one-token
+    steps over the same text."""
+    import torch
+    from paper_2304_04487_b200 import Engine
+    shape = SHAPES["mid-bf16" if small else "llama7b-shape"]
+    P, k = (120, 8) if small else (900, 8)
+    steps, accepted, plain = 38, 73, 6                                  # Fig. 5, rounded: 38 + 73 = 111 tokens
+    N = steps + accepted
+    w = make_weights(shape, seed=0)
+    eng = Engine(shape, w, max_seq=P + N + 32, max_ref=8, max_k=k, device=f"cuda:{local_rank}")
+    t0 = time.perf_counter()
+    eng.llma_prefill(0, make_prompt(P, shape.vocab, seed=1))
+    t_pre = time.perf_counter() - t0
+    target = make_prompt(N, shape.vocab, seed=8).tolist()
+    trace = fig5_like_trace(N, steps, accepted, plain, k)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    res, launches = {}, 0
+    for name, tr in (("llma", trace), ("greedy", [(1, 1)] * N)):
+        ms = []
+        for it in range(args.warmup + args.steps):
+            eng.llma_rewind(0)
+            st = eng.llma_generate_forced(0, tr, target)
+            if it >= args.warmup:
+                ms.append(st.device_ms); launches += st.launches
+        res[name] = float(np.mean(ms))
+    clocks = sampler.stop()
+    peak, peak_kind = load_peaks()
+    wbytes, kvbytes = shape.weight_bytes_per_step(), shape.kv_bytes_per_position() * (P + N // 2)
+    step_ms = res["llma"] / steps
+    line = _common_line(args, world, shape, N / (res["llma"] / 1e3), UNIT, res["llma"],
+                        {"workload": args.workload, "shape": shape.name, "prompt": P, "n": 1, "k": k, "n_new": N,
+                         "trace": {"steps": steps, "trigger_steps": steps - plain, "accepted": accepted},
+                         "l2": "inputs (weights) larger than L2"}, launches)
+    line.update({"clocks": clocks, "prefill_s": t_pre, "greedy_tokens_per_s": N / (res["greedy"] / 1e3),
+                 "speedup_vs_own_greedy": res["greedy"] / res["llma"],
+                 "speedup_including_prefill": (res["greedy"] + 1e3 * t_pre) / (res["llma"] + 1e3 * t_pre),
+                 "roofline": {"bound": "hbm", "kernel": "whole step", "achieved": (wbytes + kvbytes) / (step_ms / 1e3) / 1e9,
+                              "peak": peak, "unit": "GB/s", "frac": (wbytes + kvbytes) / (step_ms / 1e3) / 1e9 / peak,
+                              "peak_kind": f"of {peak_kind}", "traffic": None},
+                 "e2e": {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                         "note": "device-timed replay"},
+                 "paper_context": {"fig4a_7b_rag_speedup_n1_k8": 2.61, "table3_7b_rag_tokens_per_s": [23.9, 59.2],
+                                   "note": "the paper's numbers: LLaMA-7B fp16 on one V100, totals include the prompt; context only"}})
+    return line
+
+
+OTHER_RUNNERS = {"serve16": run_serve16, "layer-grid": run_layer_grid, "llama13b-sweep": run_sweep13b,
+                 "llama7b-trace": run_trace}
+
+
+def run_other(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    small = args.workload.endswith("-small")
+    key = {"serve16-small": "serve16", "layer-grid-small": "layer-grid", "sweep-small": "llama13b-sweep",
+           "trace-small": "llama7b-trace"}.get(args.workload, args.workload)
+    line = OTHER_RUNNERS[key](args, rank, local_rank, world, small=small)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def main():
@@ -189,7 +528,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama7b-rag", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="llama7b-rag", choices=sorted(WORKLOADS) + sorted(OTHER_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-steps", type=int, default=6)
     ap.add_argument("--profile-only", action="store_true",
@@ -200,6 +539,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.workload in OTHER_WORKLOADS:
+        run_other(args, rank, local_rank, world)
         return
 
     import torch
@@ -311,7 +653,10 @@ def main():
                 "launches_per_step": gemm_launches,
                 "whole_step": {"bytes": wbytes + kvbytes, "ms": step_ms,
                                "frac": (wbytes + kvbytes) / (step_ms / 1e3) / 1e9 / peak},
-                "per_class_ms_per_step": {x: round(prof[x]["ms_per_step"], 4) for x in prof}}
+                "per_class_ms_per_step": {x: round(prof[x]["ms_per_step"], 4) for x in prof},
+                "per_class": per_class_roofline(shape, prof, kvbytes, peak),
+                "per_class_note": "launched one by one with an event after every kernel (no overlap between "
+                                  "kernels): each class's rate inside the graph is at least this"}
 
     # step latency against k: reference = y* itself, so every step feeds k+1 rows.  k <= 8 on the
     # benchmark's engine (16-row MMA shape); k = 16 needs an engine created for 17 rows (32-row shape)

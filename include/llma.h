@@ -66,10 +66,6 @@ typedef struct {
     int32_t eos_id;       /* -1: none.  Otherwise a sequence stops after emitting this id */
     int32_t gemm_impl;    /* LLMA_GEMM_*; AUTO = tensor-core kernels for bf16, SIMT for fp32 */
     int32_t keep_logits;  /* 1: keep the last step's logits for llma_debug_logits */
-    int32_t kv_proj_terms; /* tensor-core path: bf16 terms the normalised hidden state is split into for the
-                              Q/K/V projection: 2 (16 mantissa bits) or 3 (24 bits); 0 = default (3).  K/V rows
-                              are rounded to bf16 afterwards, so their pre-rounding accuracy decides how often
-                              the stored code differs from an exact computation's */
 } llma_config;
 
 /* Device pointers.  Per-layer arrays are HOST arrays of n_layers device pointers. */
@@ -203,8 +199,9 @@ int llma_debug_buffer(llma_engine *e, int32_t which, float *out, int64_t count);
  * the next trace[2i]-1 tokens of `target`) through the real forward pass and then appends trace[2i+1]
  * tokens of `target` (1 <= trace[2i+1] <= trace[2i] <= max_k+1), whatever the model's own outputs are.
  * trace (host, [n_steps][2]); target (host, n_target ids) is the text to reproduce; the trace's emitted
- * counts must sum to n_target.  Every other sequence must be idle or finished.  Output tokens are the
- * target's; stats (may be NULL) carry steps, launches and device time.
+ * counts must sum to n_target.  seq = -1 replays the same trace and target on every prefilled sequence
+ * at once (one forward pass per step for all of them); otherwise every other sequence must be idle or
+ * finished.  Output tokens are the target's; stats (may be NULL) carry steps, launches and device time.
  * Errors: NULL, ARG, CAPACITY, TOKEN_RANGE, STATE, CUDA, DEVICE_TIMEOUT.
  */
 int llma_generate_forced(llma_engine *e, int32_t seq, const int32_t *trace, int32_t n_steps,

@@ -17,7 +17,7 @@ class LlmaConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab", "dtype",
                                          "max_batch", "max_seq", "max_ref", "max_k")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("eos_id", C.c_int32),
-                ("gemm_impl", C.c_int32), ("keep_logits", C.c_int32), ("kv_proj_terms", C.c_int32)]
+                ("gemm_impl", C.c_int32), ("keep_logits", C.c_int32)]
 
 
 class LlmaWeights(C.Structure):
@@ -142,7 +142,7 @@ class Engine:
 
     def __init__(self, shape, weights: Dict[str, np.ndarray], max_seq: int, max_ref: int, max_k: int,
                  max_batch: int = 1, eos_id: int = -1, gemm_impl: int = LLMA_GEMM_AUTO, keep_logits: bool = False,
-                 device: str = "cuda:0", stream=None, share_weights_with: "Engine" = None, kv_proj_terms: int = 0):
+                 device: str = "cuda:0", stream=None, share_weights_with: "Engine" = None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the LLMA engine has no CPU path")
@@ -179,7 +179,7 @@ class Engine:
                         arr_of("w_down"))
         self.cfg = LlmaConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                               LLMA_DTYPE_BF16 if bf16 else LLMA_DTYPE_F32, max_batch, max_seq, max_ref, max_k,
-                              shape.rms_eps, shape.rope_theta, eos_id, gemm_impl, int(keep_logits), kv_proj_terms)
+                              shape.rms_eps, shape.rope_theta, eos_id, gemm_impl, int(keep_logits))
         self._stream = stream if stream is not None else torch.cuda.Stream(self.device)
         h = C.c_void_p()
         torch.cuda.synchronize(self.device)

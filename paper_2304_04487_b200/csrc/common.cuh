@@ -65,14 +65,12 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-// Activations that feed a projection are kept in one of these layouts (rc = the engine's row capacity):
+// Activations that feed a projection are kept in one of two layouts (rc = the engine's row capacity):
 //   kActF32    fp32 [rc][K]                         (CUDA-core GEMM)
 //   kActSplit  bf16 [2 rc][K]: row r holds hi = bf16(v), row rc + r holds lo = bf16(v - hi), so
-//              hi + lo carries 16 mantissa bits through a bf16 tensor-core product (both halves
-//              are accumulated into the same fp32 accumulator)
-//   kActSplit3 bf16 [3 rc][K]: a third term lo2 = bf16(v - hi - lo) in row 2 rc + r, 24 mantissa
-//              bits in all (used where the product is rounded to bf16 afterwards: the K/V rows)
-enum ActLayout : int32_t { kActF32 = 0, kActSplit = 1, kActSplit3 = 2 };
+//              hi + lo carries 16 mantissa bits through a bf16 tensor-core product (the two halves
+//              are summed in fp32)
+enum ActLayout : int32_t { kActF32 = 0, kActSplit = 1 };
 
 __device__ __forceinline__ void store_act(void* buf, int layout, int rc, int r, int64_t i, int64_t K, float v) {
     if (layout == kActF32) {
@@ -81,10 +79,7 @@ __device__ __forceinline__ void store_act(void* buf, int layout, int rc, int r, 
         __nv_bfloat16* b = reinterpret_cast<__nv_bfloat16*>(buf);
         const __nv_bfloat16 hi = __float2bfloat16_rn(v);
         b[(int64_t)r * K + i] = hi;
-        const float rest = v - __bfloat162float(hi);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(rest);
-        b[(int64_t)(rc + r) * K + i] = lo;
-        if (layout == kActSplit3) b[(int64_t)(2 * rc + r) * K + i] = __float2bfloat16_rn(rest - __bfloat162float(lo));
+        b[(int64_t)(rc + r) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
 }
 

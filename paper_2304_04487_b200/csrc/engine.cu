@@ -73,7 +73,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     if (cfg->max_batch < 1 || cfg->max_batch > kSeqCap || cfg->max_k < 0 ||
         (int64_t)cfg->max_batch * (cfg->max_k + 1) > kRowCap)
         return LLMA_ERR_CONFIG;
-    if (cfg->kv_proj_terms != 0 && cfg->kv_proj_terms != 2 && cfg->kv_proj_terms != 3) return LLMA_ERR_CONFIG;
     if (cfg->max_seq < 2 || cfg->max_ref < 0 || !(cfg->rms_eps >= 0.f) || !(cfg->rope_theta > 0.f)) return LLMA_ERR_CONFIG;
     if (cfg->gemm_impl < LLMA_GEMM_AUTO || cfg->gemm_impl > LLMA_GEMM_TCGEN05) return LLMA_ERR_CONFIG;
     if (!w->tok_emb || !w->lm_head || !w->final_norm || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
@@ -107,7 +106,6 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     e->prefill_rows = std::max(e->decode_rows, e->gemm_impl == LLMA_GEMM_TCGEN05 ? 128 : 32);
     e->row_cap = e->prefill_rows;
     d.row_cap = e->row_cap;
-    e->qkv_terms = cfg->kv_proj_terms == 0 ? 3 : cfg->kv_proj_terms;
     e->tok_emb = w->tok_emb; e->lm_head = w->lm_head; e->final_norm = w->final_norm;
     for (int l = 0; l < L; ++l) {
         e->attn_norm.push_back(w->attn_norm[l]); e->ffn_norm.push_back(w->ffn_norm[l]);
@@ -144,9 +142,8 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
     CREATE_TRY(dalloc(&e->qkv, RC * 3 * HD));
     if (e->gemm_impl != LLMA_GEMM_TCGEN05) CREATE_TRY(dalloc(&e->gate_up, RC * 2 * d.d_ffn));
     if (e->gemm_impl != LLMA_GEMM_TCGEN05 || cfg->keep_logits) CREATE_TRY(dalloc(&e->logits, RC * d.vocab));
-    // activation operands: fp32 [rc][K] (CUDA-core GEMM) or split bf16 [2 rc][K] (tensor cores): 4 bytes per
-    // element; x_hat carries a third bf16 term when the QKV projection multiplies three
-    CREATE_TRY(dalloc((char**)&e->x_hat, RC * d.d_model * 6));
+    // activation operands: fp32 [rc][K] (CUDA-core GEMM) or split bf16 [2 rc][K] (tensor cores): 4 bytes per element
+    CREATE_TRY(dalloc((char**)&e->x_hat, RC * d.d_model * 4));
     CREATE_TRY(dalloc((char**)&e->attn, RC * HD * 4));
     CREATE_TRY(dalloc((char**)&e->h, RC * d.d_ffn * 4));
     const size_t kv_elems = (size_t)L * B * d.n_heads * d.max_seq * d.head_dim;
@@ -205,7 +202,7 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         // activation operands of the wide kernel: one box of nr rows per (buffer, use)
         auto act_maps = [&](llma_engine::ActMaps& m, int nr) {
             int bad2 = 0;
-            bad2 |= make_tensor_map_bf16(&m.x_hat, e->x_hat, 3 * RC, d.d_model, nr);
+            bad2 |= make_tensor_map_bf16(&m.x_hat, e->x_hat, 2 * RC, d.d_model, nr);
             bad2 |= make_tensor_map_bf16(&m.attn, e->attn, 2 * RC, HD, nr);
             bad2 |= make_tensor_map_bf16(&m.h, e->h, 2 * RC, d.d_ffn, nr);
             return bad2;

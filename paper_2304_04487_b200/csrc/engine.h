@@ -37,7 +37,6 @@ struct llma_engine {
     // row capacities (multiples of 16): activation buffers hold row_cap rows; a decoding step uses at most
     // decode_rows = max_batch * (max_k + 1) of them, a prompt pass prefill_rows
     int row_cap = 0, decode_rows = 0, prefill_rows = 0;
-    int qkv_terms = 2;              // bf16 terms of the QKV projection's activation operand (2 or 3)
 
     // tensor-core GEMM path (bf16): TMA descriptors of weights and activation buffers, work buffers
     struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };

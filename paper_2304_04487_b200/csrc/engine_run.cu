@@ -30,9 +30,9 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
     std::memset(&a, 0, sizeof(a));
     a.mode = mode; a.n_out = n_out; a.n_tiles = n_tiles; a.chunks = k_in / 64; a.tiles_per_map = tiles_per_map;
     a.rows = e->rows; a.dev_err = e->dev_err;
-    a.rc = e->row_cap; a.nr = e->cur_nr; a.terms = 2;
+    a.rc = e->row_cap; a.nr = e->cur_nr;
+    a.l2_ahead = e->l2_ahead;
     a.ws = e->cur_wide ? e->gemm_ws_wide : e->gemm_ws;
-    a.xs_layout = kActSplit;
     a.dims = e->dims;
     return a;
 }
@@ -54,9 +54,6 @@ static void with_norm(llma_engine* e, GemmArgs& a) {
     a.norm_dim = e->dims.d_model; a.norm_eps = e->dims.rms_eps;
 }
 
-// layout of x_hat when it feeds a QKV projection
-static int qkv_act_layout(const llma_engine* e) { return e->qkv_terms == 3 ? kActSplit3 : kActSplit; }
-
 static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const ModelDims& d = e->dims;
     cudaStream_t st = e->stream;
@@ -66,7 +63,6 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         const llma_engine::LayerMaps& m = e->maps[l];
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
         with_norm(e, q);
-        q.terms = e->qkv_terms;
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
         run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat, am ? &am->x_hat : nullptr);
@@ -91,7 +87,6 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
-        if (l + 1 < d.n_layers) dn.xs_layout = qkv_act_layout(e);  // feeds the next layer's QKV projection
         run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h, am ? &am->h : nullptr);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 6;
@@ -157,7 +152,7 @@ static void enqueue_forward(llma_engine* e, bool lm_head) {
 static void enqueue_embed(llma_engine* e) {
     if (e->gemm_impl == LLMA_GEMM_TCGEN05)
         launch_embed_norm(e->stream, e->dims, e->cur_rows, e->rows, e->tok_emb, e->attn_norm[0], e->x, e->x_hat,
-                          qkv_act_layout(e), e->norm_ss, e->dev_err);
+                          e->norm_ss, e->dev_err);
     else
         launch_embed(e->stream, e->dims, e->bf16, e->cur_rows, e->rows, e->tok_emb, e->x, e->dev_err);
 }
@@ -183,7 +178,7 @@ static void enqueue_tail(llma_engine* e, int n, int k, bool accept, bool plan) {
     if (e->gemm_impl == LLMA_GEMM_TCGEN05) {
         t.part_max = e->part_max; t.part_idx = e->part_idx; t.n_tiles = (e->dims.vocab + 127) / 128;
     }
-    t.out_tok = e->out_tok;
+    t.out_tok = e->out_tok; t.n_rows = e->decode_rows;
     t.trace = e->trace; t.target = e->target; t.trace_cap = e->trace_cap;
     t.dev_err = e->dev_err;
     launch_step_tail(e->stream, t);
@@ -465,7 +460,7 @@ extern "C" int llma_generate_forced(llma_engine* e, int32_t seq, const int32_t* 
                                     const int32_t* target, int32_t n_target, llma_stats* stats) {
     if (!e || !trace || !target) return LLMA_ERR_NULL;
     const ModelDims& d = e->dims;
-    if (seq < 0 || seq >= d.max_batch) return LLMA_ERR_CAPACITY;
+    if (seq < -1 || seq >= d.max_batch) return LLMA_ERR_CAPACITY;
     if (n_steps < 1 || n_target < 1 || n_steps > e->trace_cap) return LLMA_ERR_ARG;
     int64_t total = 0;
     for (int i = 0; i < n_steps; ++i) {
@@ -478,19 +473,29 @@ extern "C" int llma_generate_forced(llma_engine* e, int32_t seq, const int32_t* 
         if (target[i] < 0 || target[i] >= d.vocab) return LLMA_ERR_TOKEN_RANGE;
     int rc = read_state(e);
     if (rc) return rc;
-    for (int s = 0; s < d.max_batch; ++s)
-        if (s != seq && e->h_state[s].active && !e->h_state[s].done) return LLMA_ERR_STATE;
-    const SeqState s0 = e->h_state[seq];
-    if (!s0.active) return LLMA_ERR_STATE;
-    if (s0.kv_len + n_target > d.max_seq || s0.y_len + n_target > e->y_cap) return LLMA_ERR_CAPACITY;
-    CU_TRY(cudaMemcpyAsync(e->trace + (size_t)seq * e->trace_cap * 2, trace, (size_t)n_steps * 2 * sizeof(int32_t),
-                           cudaMemcpyHostToDevice, e->stream));
-    CU_TRY(cudaMemcpyAsync(e->target + (size_t)seq * e->y_cap + s0.y_len, target, (size_t)n_target * sizeof(int32_t),
-                           cudaMemcpyHostToDevice, e->stream));
-    SeqState& S = e->h_state[seq];
-    S.target_len = S.y_len + n_target; S.done = 0; S.forced_rows = 1; S.forced_emit = 1; S.trace_step = 0;
-    rc = write_state(e, seq);  // synchronises: the host arrays may go after this
-    if (rc) return rc;
+    // the sequences that replay: the given one, or (seq = -1) every prefilled one; all others must be at rest
+    std::vector<int> who;
+    for (int s = 0; s < d.max_batch; ++s) {
+        const SeqState& S = e->h_state[s];
+        if (s == seq || (seq < 0 && S.active)) who.push_back(s);
+        else if (S.active && !S.done) return LLMA_ERR_STATE;
+    }
+    if (who.empty()) return LLMA_ERR_STATE;
+    std::vector<SeqState> s0(e->h_state, e->h_state + d.max_batch);
+    for (int s : who) {
+        if (!s0[s].active) return LLMA_ERR_STATE;
+        if (s0[s].kv_len + n_target > d.max_seq || s0[s].y_len + n_target > e->y_cap) return LLMA_ERR_CAPACITY;
+    }
+    for (int s : who) {
+        CU_TRY(cudaMemcpyAsync(e->trace + (size_t)s * e->trace_cap * 2, trace, (size_t)n_steps * 2 * sizeof(int32_t),
+                               cudaMemcpyHostToDevice, e->stream));
+        CU_TRY(cudaMemcpyAsync(e->target + (size_t)s * e->y_cap + s0[s].y_len, target, (size_t)n_target * sizeof(int32_t),
+                               cudaMemcpyHostToDevice, e->stream));
+        SeqState& S = e->h_state[s];
+        S.target_len = S.y_len + n_target; S.done = 0; S.forced_rows = 1; S.forced_emit = 1; S.trace_step = 0;
+        rc = write_state(e, s);  // synchronises: the host arrays may go after this
+        if (rc) return rc;
+    }
     cudaGraphExec_t graph = nullptr;
     rc = get_step_graph(e, 1, 0, &graph);
     if (rc) return rc;
@@ -505,19 +510,23 @@ extern "C" int llma_generate_forced(llma_engine* e, int32_t seq, const int32_t* 
     if (rc) return rc;
     rc = read_state(e);
     if (rc) return rc;
-    SeqState& T = e->h_state[seq];
     llma_stats st;
     std::memset(&st, 0, sizeof(st));
-    st.steps = T.steps - s0.steps; st.trigger_steps = T.trigger_steps - s0.trigger_steps;
-    st.copied_accepted = T.copied_accepted - s0.copied_accepted; st.tokens = T.y_len - s0.y_len;
+    bool complete = true;
+    for (int s : who) {
+        SeqState& T = e->h_state[s];
+        st.steps += T.steps - s0[s].steps; st.trigger_steps += T.trigger_steps - s0[s].trigger_steps;
+        st.copied_accepted += T.copied_accepted - s0[s].copied_accepted; st.tokens += T.y_len - s0[s].y_len;
+        complete = complete && T.y_len - s0[s].y_len == n_target;
+        T.forced_rows = 0; T.forced_emit = 0; T.trace_step = 0;
+        rc = write_state(e, s);
+        if (rc) return rc;
+    }
     st.launches = tail_launches + (int64_t)n_steps * e->launches_per_step;
     CU_TRY(cudaEventElapsedTime(&st.device_ms, e->ev0, e->ev1));
-    T.forced_rows = 0; T.forced_emit = 0; T.trace_step = 0;
-    rc = write_state(e, seq);
-    if (rc) return rc;
     if (stats) *stats = st;
     e->last_step_valid = false;
-    return st.tokens == n_target ? LLMA_OK : LLMA_ERR_STATE;
+    return complete ? LLMA_OK : LLMA_ERR_STATE;
 }
 
 extern "C" int llma_debug_set_device_error(llma_engine* e, int32_t code) {

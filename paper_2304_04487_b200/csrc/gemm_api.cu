@@ -17,7 +17,7 @@ int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, 
     g.mode = kGemmStore; g.n_out = n_out; g.n_tiles = (n_out + 127) / 128; g.chunks = k_in / 64;
     g.tiles_per_map = g.n_tiles; g.rows = nullptr; g.ws = ws; g.dev_err = dev_err;
     g.out_f32 = out; g.ld = n_out; g.act = a;
-    g.rc = 32; g.nr = 32; g.terms = 2;  // the operand is [64][k_in]: 32 rows, then their low halves
+    g.rc = 32; g.nr = 32;  // the operand is [64][k_in]: 32 rows, then their low halves
     launch_gemm_tcgen05(st, grid, false, g, ma, ma, ma);
     CU_TRY(cudaGetLastError());
     return LLMA_OK;

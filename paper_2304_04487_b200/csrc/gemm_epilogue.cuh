@@ -57,7 +57,7 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
         const float xn = valid ? stage[row][j] : 0.f;
         if (valid) g.out_f32[(int64_t)(jb + j) * g.ld + col] = xn;
         if (fold) {
-            if (valid) store_act(g.xs_out, g.xs_layout, g.rc, jb + j, col, g.n_out, xn * gain);
+            if (valid) store_act(g.xs_out, kActSplit, g.rc, jb + j, col, g.n_out, xn * gain);
             const float sq = warp_sum(xn * xn);
             if (lane == 0) red_f[warp * 32 + j] = sq;
         }

@@ -26,15 +26,17 @@ namespace llma {
 
 using namespace ptx;
 
-// NR = activation rows: 16 or 32 = MMA N.  NT = bf16 terms of the activation operand (2 or 3): each weight
-// tile is multiplied by every term, all into the same accumulator.  MODE = GemmMode: one kernel per fused
+// NR = activation rows: 16 or 32.  The hi and lo halves of the activations are the MMA's N = 2 NR columns
+// (one MMA per k-slice: an MMA this narrow costs the same issue time whatever its N, so two N = NR MMAs into
+// one accumulator measured 15 % slower); the epilogue adds the two halves.  MODE = GemmMode: one kernel per fused
 // epilogue, so that each carries only the code it runs (the end of a launch is instruction-fetch-bound).
-template <int NR, int NT, int MODE>
+template <int NR, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2) {
-    using Cfg = GemmCfg<NR, NT>;
-    constexpr uint32_t kTmemCols = 2 * NR;  // two accumulators of NR columns (32 is the smallest allocation)
+    using Cfg = GemmCfg<NR>;
+    constexpr int NT = 2;                   // bf16 terms of the activation operand: hi, lo
+    constexpr uint32_t kTmemCols = 4 * NR;  // two accumulators of 2 NR columns
     constexpr int S = Cfg::kStages;
     constexpr uint32_t kBBytes = Cfg::kBBytes;
 
@@ -120,7 +122,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else if (warp == 5) {
         // ------------------------------- MMA issuer ---------------------------------------------
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_m128(NR);
+            constexpr uint32_t idesc = idesc_bf16_m128(2 * NR);
             int64_t it = 0;
             int seg = 0;
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
@@ -130,7 +132,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const uint32_t use = (uint32_t)(seg >> 1);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * NR;
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (2 * NR);
                 for (int c = c0; c < c1; ++c, ++it) {
                     const int s = (int)(it % S);
                     const uint32_t ph = (uint32_t)((it / S) & 1);
@@ -139,12 +141,8 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
                     const uint64_t db = smem_desc_sw128(sB + s * kBBytes);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-#pragma unroll
-                        for (int t = 0; t < NT; ++t)  // term t of the activations: NR rows of 128 bytes further on
-                            umma_bf16(d_tmem, da + 2 * kk, db + (uint64_t)(t * NR * 8) + 2 * kk, idesc,
-                                      (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                        umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0) ? 1u : 0u);
                     umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
                 }
                 if (sh[1]) break;
@@ -250,7 +248,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             }
         };
         // stage the tile in shared memory (scaled by the folded RMSNorm), then the fused epilogue
-        auto finish_tile = [&](int tile, float (&acc)[NR], const float (&xpre)[kXPre]) {
+        auto finish_tile = [&](int tile, float (&acc)[32], const float (&xpre)[kXPre]) {
             if (g.ss_in) {
 #pragma unroll
                 for (int j = 0; j < NR; ++j) stage[row][j] = acc[j] * rscale[j];
@@ -294,11 +292,20 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             epi_sync();
             if (!ok) { aborted = true; break; }
             tc_fence_after();
-            float acc[NR];
+            float acc[32];
             {
-                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * NR;
-                if constexpr (NR == 32) tmem_ld_32cols(t0, acc);
-                else tmem_ld_16cols(t0, acc);
+                const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (2 * NR);
+                if (NR == 32) {
+                    float lo[32];
+                    tmem_ld_32cols(t0, acc);
+                    tmem_ld_32cols(t0 + 32, lo);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+                } else {
+                    tmem_ld_32cols(t0, acc);  // columns 0..15 hi, 16..31 lo
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { acc[j] += acc[16 + j]; acc[16 + j] = 0.f; }
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -324,9 +331,9 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         if (own_tile >= 0 && !aborted) {
             float xpre[kXPre];
             prefetch_x(own_tile, xpre);
-            float acc[NR];
+            float acc[32];
 #pragma unroll
-            for (int j = 0; j < NR; ++j) acc[j] = 0.f;
+            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
             // this CTA's own partial (parked in slot 0 by these same threads) is requested now and added last
             float4 own[NR / 4];
             {
@@ -430,20 +437,19 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-template <int NR, int NT, int MODE>
+template <int NR, int MODE>
 static cudaError_t opt_in() {
-    return cudaFuncSetAttribute(gemm_ws_kernel<NR, NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)GemmCfg<NR, NT>::kSmemBytes);
+    return cudaFuncSetAttribute(gemm_ws_kernel<NR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)GemmCfg<NR>::kSmemBytes);
 }
 template <int NR>
 static cudaError_t opt_in_all() {
     cudaError_t e;
-    if ((e = opt_in<NR, 2, kGemmQKV>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, 3, kGemmQKV>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, 2, kGemmResid>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, 2, kGemmSwiGLU>()) != cudaSuccess) return e;
-    if ((e = opt_in<NR, 2, kGemmLmHead>()) != cudaSuccess) return e;
-    return opt_in<NR, 2, kGemmStore>();
+    if ((e = opt_in<NR, kGemmQKV>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmResid>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmSwiGLU>()) != cudaSuccess) return e;
+    if ((e = opt_in<NR, kGemmLmHead>()) != cudaSuccess) return e;
+    return opt_in<NR, kGemmStore>();
 }
 
 cudaError_t init_gemm_tcgen05() {
@@ -452,23 +458,15 @@ cudaError_t init_gemm_tcgen05() {
     return opt_in_all<32>();
 }
 
-// three terms exist for the QKV projection only (its K/V rows are rounded to bf16 afterwards)
 template <int NR>
 static void launch_mode(cudaLaunchConfig_t* cfg, const GemmArgs& args, const CUtensorMap& a0, const CUtensorMap& a1,
                         const CUtensorMap& a2) {
     switch (args.mode) {
-        case kGemmQKV:
-            if (args.terms == 3) {
-                cfg->dynamicSmemBytes = GemmCfg<NR, 3>::kSmemBytes;
-                cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 3, kGemmQKV>, args, a0, a1, a2);
-            } else {
-                cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmQKV>, args, a0, a1, a2);
-            }
-            break;
-        case kGemmResid: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmResid>, args, a0, a1, a2); break;
-        case kGemmSwiGLU: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmSwiGLU>, args, a0, a1, a2); break;
-        case kGemmLmHead: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmLmHead>, args, a0, a1, a2); break;
-        default: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, 2, kGemmStore>, args, a0, a1, a2); break;
+        case kGemmQKV: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmQKV>, args, a0, a1, a2); break;
+        case kGemmResid: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmResid>, args, a0, a1, a2); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmSwiGLU>, args, a0, a1, a2); break;
+        case kGemmLmHead: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmLmHead>, args, a0, a1, a2); break;
+        default: cudaLaunchKernelEx(cfg, gemm_ws_kernel<NR, kGemmStore>, args, a0, a1, a2); break;
     }
 }
 
@@ -477,7 +475,7 @@ void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& ar
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = args.nr == 16 ? GemmCfg<16, 2>::kSmemBytes : GemmCfg<32, 2>::kSmemBytes;
+    cfg.dynamicSmemBytes = args.nr == 16 ? GemmCfg<16>::kSmemBytes : GemmCfg<32>::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -2,10 +2,9 @@
 //
 //   out[r, n] = sum_k W[n, k] * a[r, k],  r < rows (up to 256 activation rows), W bf16 [n_out, k_in].
 //
-// The activations arrive split into bf16 terms (ActLayout kActSplit / kActSplit3: hi rows, lo rows,
-// optionally a third term); every term is multiplied by the same weight tile and accumulated into
-// the same fp32 accumulator, so the product keeps 16 (24) mantissa bits of the activations at no
-// cost in weight traffic.
+// The activations arrive split into two bf16 terms (ActLayout kActSplit: hi rows, then lo rows); both
+// are multiplied by the same weight tile and summed in fp32, so the product keeps 16 mantissa bits
+// of the activations at no cost in weight traffic.
 //
 // The weight matrix is the MMA's M operand (128 output features per tile) and the
 // activation rows are its N operand, so every weight byte crosses HBM exactly once per
@@ -39,10 +38,9 @@ struct GemmArgs {
     int32_t chunks;         // k_in / 64
     int32_t tiles_per_map;  // tiles per A map
     const RowDesc* rows;    // nullptr: all nr rows are in use
-    const void* act;        // activation operand, ActLayout kActSplit(3) [terms * rc][k_in] bf16
+    const void* act;        // activation operand, ActLayout kActSplit [2 rc][k_in] bf16
     int32_t rc;             // row capacity of the activation buffers and per-row scratch arrays
     int32_t nr;             // rows the launch is shaped for (wide kernel: multiple of 16, <= 256)
-    int32_t terms;          // bf16 terms of the activation operand that are multiplied (2 or 3)
     float* ws;              // partial tiles [grid][2][nr / 4][128] float4; slot 1 of every CTA all-ones (empty) at launch
     int32_t* dev_err;
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
@@ -57,8 +55,7 @@ struct GemmArgs {
     int32_t norm_dim;
     float norm_eps;
     const float* gain_next; // Resid producer: gain of the next norm [n_out], with xs_out / ss_out
-    void* xs_out;           // ActLayout xs_layout [terms * rc][n_out], or nullptr
-    int32_t xs_layout;      // kActSplit or kActSplit3
+    void* xs_out;           // ActLayout kActSplit [2 rc][n_out], or nullptr
     float* ss_out;          // [n_tiles][rc]
     // QKV
     ModelDims dims;
@@ -74,8 +71,7 @@ constexpr int kGemmThreads = 320;  // 4 epilogue warps, TMA producer, MMA issuer
 constexpr int kGemmWideThreads = 224;  // 4 epilogue warps, weight producer, MMA issuer, activation producer
 constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 
-// gemm_ws_kernel exists for NR = 16 or 32 activation rows and NT = 2 or 3 terms (MMA N = NR, issued once
-// per term).  Ring depths are the ones measured fastest inside a decoding step (deeper rings only
+// gemm_ws_kernel exists for NR = 16 or 32 activation rows (MMA N = 2 NR: hi and lo columns).  Ring depths are the ones measured fastest inside a decoding step (deeper rings only
 // lengthen the queues that the epilogue's traffic also waits in).  The activation tile of a stage
 // is NOT fetched by TMA here: a second, small TMA copy per stage slowed the weight stream by a
 // quarter wherever it came from (shared buffer, per-CTA replica, one hot 4 KB block), whereas
@@ -83,9 +79,9 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 // the rows from global memory into the 128-byte-swizzled layout the MMA expects.
 // The request is padded to more than half an SM's shared memory so that the CTAs of two
 // consecutive projections never share an SM (measured 10 % slower when they do).
-template <int NR, int NT> struct GemmCfg {
-    static constexpr uint32_t kBBytes = NT * NR * 64 * 2;
-    static constexpr int kStages = NR == 16 ? 8 : (NT == 2 ? 7 : 6);
+template <int NR> struct GemmCfg {
+    static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
+    static constexpr int kStages = NR == 16 ? 8 : 7;
     static constexpr size_t kRopeBytes = 32 * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
     static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
@@ -111,12 +107,12 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-// args.nr = 16 or 32 rows, args.terms = 2 or 3; pdl = launch with programmatic stream serialization
+// args.nr = 16 or 32 rows; pdl = launch with programmatic stream serialization
 // (the kernel before it must be one of this library's)
 void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2);
 
-// args.nr = 16 .. 256 (multiple of 16); map_b covers the activation buffer [terms * rc][k_in] with a
+// args.nr = 32 .. 256 (multiple of 16); map_b covers the activation buffer [2 rc][k_in] with a
 // {64, nr} box
 cudaError_t init_gemm_wide();
 void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,

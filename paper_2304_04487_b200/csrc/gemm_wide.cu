@@ -1,8 +1,8 @@
 // Weight-streaming GEMM for up to 256 activation rows (batched decoding steps, prompt passes).
 // Same contract, work split and fused epilogues as gemm_ws_kernel (see gemm_tcgen05.cuh); what differs:
 //   * the activation tiles are large enough for TMA to pay: a second producer thread streams them
-//     through a ring of their own (one slot = nr rows x 64 columns of ONE bf16 term), so the number of
-//     terms does not change the depth of the weight ring;
+//     through a ring of their own (one slot = nr rows x 64 columns of ONE bf16 term, hi or lo); both terms
+//     are accumulated into the same TMEM columns, so 256 rows fit two accumulators;
 //   * MMA N = the rows in use rounded up to 16 (a run-time field of the instruction descriptor);
 //   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
 //
@@ -35,7 +35,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const int nr = g.nr, NT = g.terms;
+    const int nr = g.nr;
+    constexpr int NT = 2;  // bf16 terms of the activation operand: hi, lo
     const uint32_t b_slot = (uint32_t)nr * 128u;
     const uint32_t sA = base, sB = base + (uint32_t)SA * kGemmABytes;
     uint8_t* after = gen_base + (size_t)SA * kGemmABytes + (size_t)SB * b_slot;

@@ -21,6 +21,7 @@ struct TailArgs {
     const int32_t* part_idx;
     int32_t n_tiles;
     int32_t* out_tok;          // [row_cap]
+    int32_t n_rows;            // row slots of a decoding step (decode_rows)
     // replay
     const int32_t* trace;      // [max_batch][trace_cap][2] = (rows, emitted) of every step, or nullptr
     const int32_t* target;     // [max_batch][y_cap] the text to reproduce
@@ -35,7 +36,7 @@ void launch_embed(cudaStream_t st, const ModelDims& dims, bool bf16, int n_rows,
                   float* x, int32_t* dev_err);
 // bf16 embedding gather with the first RMSNorm folded in: x, xs = split(x * gain), ss[tile][row]
 void launch_embed_norm(cudaStream_t st, const ModelDims& dims, int n_rows, const RowDesc* rows, const void* emb,
-                       const float* gain, float* x, void* xs, int xs_layout, float* ss, int32_t* dev_err);
+                       const float* gain, float* x, void* xs, float* ss, int32_t* dev_err);
 
 // ---- SIMT (CUDA-core) kernels, fp32 or bf16 storage (kernels_simt.cu) -------------------
 // x_hat[r,:] = rmsnorm(x[r,:]) * g in the given ActLayout (rc = row capacity); unused rows are zero-filled

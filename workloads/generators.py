@@ -67,6 +67,8 @@ SHAPES: Dict[str, ModelShape] = {
     "llama7b-shape": ModelShape("llama7b-shape", 32, 4096, 32, 128, 11008, 32000, "bf16"),
     # two layers at the 7B widths: the same kernels and tile shapes at a size a profiler capture can hold
     "llama7b-2layer": ModelShape("llama7b-2layer", 2, 4096, 32, 128, 11008, 32000, "bf16"),
+    # one layer of the 7B-shaped decoder with a token table too small to matter: what a step costs is the layer
+    "llama7b-1layer": ModelShape("llama7b-1layer", 1, 4096, 32, 128, 11008, 256, "bf16"),
     "llama13b-shape": ModelShape("llama13b-shape", 40, 5120, 40, 128, 13824, 32000, "bf16"),
     "llama13b-2layer": ModelShape("llama13b-2layer", 2, 5120, 40, 128, 13824, 32000, "bf16"),
 }
