@@ -40,8 +40,9 @@ struct llma_engine {
 
     // tensor-core GEMM path (bf16): TMA descriptors of weights and activation buffers, work buffers
     struct LayerMaps { CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down; };
-    std::vector<LayerMaps> maps;
-    CUtensorMap map_lm_head;
+    std::vector<LayerMaps> maps;    // 2-D views (gemm_wide_kernel; gate/up of both kernels)
+    std::vector<LayerMaps> maps2;   // chunk-pair views (gemm_ws_kernel; gate/up entries are the 2-D ones)
+    CUtensorMap map_lm_head, map_lm_head2;
     struct ActMaps { CUtensorMap x_hat, attn, h; };  // activation operands of gemm_wide_kernel, box of nr rows
     ActMaps act_decode, act_prefill;
     bool decode_wide = false;       // decoding steps of more than 32 rows use gemm_wide_kernel

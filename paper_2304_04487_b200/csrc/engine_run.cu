@@ -59,7 +59,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
     const int HD = d.hd_total, F = d.d_ffn, D = d.d_model;
     const llma_engine::ActMaps* am = e->cur_maps;
     for (int l = 0; l < d.n_layers; ++l) {
-        const llma_engine::LayerMaps& m = e->maps[l];
+        const llma_engine::LayerMaps& m = e->cur_wide ? e->maps[l] : e->maps2[l];
         GemmArgs q = gemm_args(e, kGemmQKV, HD, 3 * HD / 128, D, HD / 128);
         with_norm(e, q);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
@@ -96,7 +96,8 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         with_norm(e, lm);
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
-        run_gemm(e, lm, e->map_lm_head, e->map_lm_head, e->map_lm_head, e->x_hat, am ? &am->x_hat : nullptr);
+        const CUtensorMap& lmm = e->cur_wide ? e->map_lm_head : e->map_lm_head2;
+        run_gemm(e, lm, lmm, lmm, lmm, e->x_hat, am ? &am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_LMHEAD);
         e->launch_counter += 1;
     }

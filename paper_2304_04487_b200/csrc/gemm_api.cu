@@ -11,7 +11,7 @@ namespace llma {
 int gemm_rows32_launch(const void* W, const void* a, float* out, int32_t n_out, int32_t k_in, float* ws,
                        int32_t* dev_err, int grid, cudaStream_t st) {
     CUtensorMap ma;
-    if (make_tensor_map_bf16(&ma, W, (uint64_t)n_out, (uint64_t)k_in, 128) != 0) return LLMA_ERR_ARG;
+    if (make_tensor_map_bf16_chunks(&ma, W, (uint64_t)n_out, (uint64_t)k_in, 128) != 0) return LLMA_ERR_ARG;
     GemmArgs g;
     std::memset(&g, 0, sizeof(g));
     g.mode = kGemmStore; g.n_out = n_out; g.n_tiles = (n_out + 127) / 128; g.chunks = k_in / 64;

@@ -34,17 +34,18 @@ template <int NR, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2) {
-    using Cfg = GemmCfg<NR>;
+    constexpr int KC = gemm_ws_chunks_per_stage(MODE);  // 64-wide k-chunks per ring stage (one TMA copy)
+    using Cfg = GemmCfg<NR, KC>;
     constexpr int NT = 2;                   // bf16 terms of the activation operand: hi, lo
     constexpr uint32_t kTmemCols = 4 * NR;  // two accumulators of 2 NR columns
     constexpr int S = Cfg::kStages;
-    constexpr uint32_t kBBytes = Cfg::kBBytes;
+    constexpr uint32_t kABytes = Cfg::kABytes, kBBytes = Cfg::kBBytes, kBTile = Cfg::kBTile;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t sA = base, sB = base + S * kGemmABytes;
-    float (*stage)[33] = reinterpret_cast<float (*)[33]>(gen_base + S * (kGemmABytes + kBBytes));
+    const uint32_t sA = base, sB = base + S * kABytes;
+    float (*stage)[33] = reinterpret_cast<float (*)[33]>(gen_base + S * (kABytes + kBBytes));
     uint8_t* tail = reinterpret_cast<uint8_t*>(stage) + 128 * 33 * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full[S], empty[S], acc_full[2], acc_empty[2]
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + (2 * S + 4) * 8);
@@ -61,14 +62,15 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, b = blockIdx.x;
-    const int C = g.chunks;
+    const int C = (g.chunks + KC - 1) / KC;  // work items (ring stages) per tile
     const int64_t work = (int64_t)g.n_tiles * C;
     const int64_t w_beg = cta_begin(work, b, G), w_end = cta_begin(work, b + 1, G);
 
     grid_launch_dependents();  // the next kernel may begin its own prologue now
     if (threadIdx.x == 0) {
-        // a stage is full once its weight tile has landed (producer's expect_tx) and its loader warp has arrived
-        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
+        // a stage is full once its weight tile has landed (producer's expect_tx) and the loader warps of its
+        // KC activation tiles have arrived
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1 + KC); mbar_init(empty_bar(s), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(accf_bar(i), 1); mbar_init(acce_bar(i), 4); }
         sh[1] = 0; sh[2] = 0;
         fence_mbar_init();
@@ -92,14 +94,15 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         if (lane == 0) {
             auto load_a = [&](int64_t w, int s) {
                 const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
-                const uint32_t dstA = sA + s * kGemmABytes;
+                const uint32_t dstA = sA + s * kABytes;
                 if (MODE == kGemmSwiGLU) {
                     tma_load_2d(dstA, &map_a0, full_bar(s), c * 64, tile * 64);
                     tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_bar(s), c * 64, tile * 64);
                 } else {
+                    // chunks 2c and 2c+1 of the tile in one copy (a chunk past the matrix arrives as zeros)
                     const int m = tile / g.tiles_per_map, r0 = (tile % g.tiles_per_map) * 128;
                     const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
-                    tma_load_2d(dstA, mp, full_bar(s), c * 64, r0);
+                    tma_load_3d(dstA, mp, full_bar(s), 0, r0, c * KC);
                 }
             };
             // weights are written by no kernel of the step: the whole range streams without waiting for
@@ -109,7 +112,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 const int s = (int)(it % S);
                 const uint32_t ph = (uint32_t)((it / S) & 1);
                 if (it >= S && !mbar_wait(empty_bar(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                mbar_arrive_expect_tx(full_bar(s), kGemmABytes);
+                mbar_arrive_expect_tx(full_bar(s), kABytes);
                 load_a(w, s);
             }
             if (sh[1]) {
@@ -138,11 +141,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const uint32_t ph = (uint32_t)((it / S) & 1);
                     if (!mbar_wait(full_bar(s), ph)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                     tc_fence_after();
-                    const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
-                    const uint64_t db = smem_desc_sw128(sB + s * kBBytes);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-                        umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0) ? 1u : 0u);
+                    for (int h = 0; h < KC; ++h) {  // the stage's k-chunks: a weight tile and an activation tile each
+                        const uint64_t da = smem_desc_sw128(sA + s * kABytes + h * kGemmABytes);
+                        const uint64_t db = smem_desc_sw128(sB + s * kBBytes + h * kBTile);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || h > 0 || kk > 0) ? 1u : 0u);
+                    }
                     umma_commit(empty_bar(s));  // stage is free once these MMAs have read it
                 }
                 if (sh[1]) break;
@@ -156,31 +162,35 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         // swizzled descriptor reads): row r = 0..NT*NR-1 (NR rows per term) at r * 128 bytes, its
         // 16-byte unit j stored at position j ^ (r & 7).  Rows past those in use are left as they are:
         // their columns of the accumulator are never read.
-        constexpr int NW = 4;  // loader warps: warp 6 + i takes items i, i + NW, ...
+        constexpr int NW = 4;  // loader warps: warp 6 + i takes activation tiles i, i + NW, ... (KC tiles per stage)
         const int sw = warp - 6;
         grid_dependency_wait();  // activations are written by the kernel before this one
         const int rows_used = g.rows ? min(__ldcg(&g.rows->rows_used), NR) : NR;
-        const int64_t n_items = w_end - w_beg;
-        const int64_t ld_bytes = (int64_t)C * 128;  // one activation row: k_in bf16
+        const int64_t n_sub = (w_end - w_beg) * KC;
+        const int64_t ld_bytes = (int64_t)g.chunks * 128;  // one activation row: k_in bf16
         const char* act = reinterpret_cast<const char*>(g.act);
         constexpr int kUnits = NT * NR * 8 / 32;    // 16-byte units per lane
         // rows of the next tile are requested before waiting for its stage to come free, so the
         // latency of the loads hides behind the MMAs of the tiles in between
         uint4 v[kUnits];
-        auto fetch = [&](int64_t it, int row_limit) {
-            const int c = (int)((w_beg + it) % C);
+        auto fetch = [&](int64_t q, int row_limit) {
+            const int64_t it = q / KC;
+            const int chunk = (int)((w_beg + it) % C) * KC + (int)(q % KC);  // 64-wide chunk of the activations
+            const bool inside = chunk < g.chunks;                            // past the matrix: zeros
 #pragma unroll
             for (int u = 0; u < kUnits; ++u) {
                 const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
                 const int t = r / NR, rr = r - t * NR;                // term, row inside it
                 const int src_row = t * g.rc + rr;                    // term t starts at row t * rc
                 v[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (rr < row_limit)
-                    v[u] = __ldcg(reinterpret_cast<const uint4*>(act + src_row * ld_bytes + (int64_t)c * 128 + j * 16));
+                if (rr < row_limit && inside)
+                    v[u] = __ldcg(reinterpret_cast<const uint4*>(act + src_row * ld_bytes + (int64_t)chunk * 128 + j * 16));
             }
         };
-        if (sw < n_items) fetch(sw, NR);  // every row: the count of rows in use is still on its way
-        for (int64_t it = sw; it < n_items && !sh[1]; it += NW) {
+        if (sw < n_sub) fetch(sw, NR);  // every row: the count of rows in use is still on its way
+        for (int64_t q = sw; q < n_sub && !sh[1]; q += NW) {
+            const int64_t it = q / KC;
+            const int h = (int)(q % KC);
             const int st = (int)(it % S);
             const uint32_t ph = (uint32_t)((it / S) & 1);
             if (it >= S) {
@@ -193,12 +203,13 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             for (int u = 0; u < kUnits; ++u) {
                 const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
                 const int rr = r % NR;
-                if (rr < rows_used) st_shared_v4(sB + st * kBBytes + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
+                if (rr < rows_used)
+                    st_shared_v4(sB + st * kBBytes + h * kBTile + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4), v[u]);
             }
             fence_proxy_async_shared();  // make the stores visible to the tensor core's reads
             __syncwarp();
             if (lane == 0) mbar_arrive(full_bar(st));
-            if (it + NW < n_items) fetch(it + NW, rows_used);
+            if (q + NW < n_sub) fetch(q + NW, rows_used);
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
@@ -420,14 +431,32 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+static EncodeTiledFn encode_fn() {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return -1;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return nullptr;
         fn = (EncodeTiledFn)p;
     }
+    return fn;
+}
+
+int make_tensor_map_bf16_chunks(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || cols % 64) return -1;
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {cols * 2, 128};
+    const cuuint32_t box[3] = {64, box_rows, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return (int)fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return -1;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
     const cuuint32_t box[2] = {64, box_rows};
@@ -440,7 +469,7 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 template <int NR, int MODE>
 static cudaError_t opt_in() {
     return cudaFuncSetAttribute(gemm_ws_kernel<NR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)GemmCfg<NR>::kSmemBytes);
+                                (int)GemmCfg<NR, gemm_ws_chunks_per_stage(MODE)>::kSmemBytes);
 }
 template <int NR>
 static cudaError_t opt_in_all() {
@@ -475,7 +504,9 @@ void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& ar
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = args.nr == 16 ? GemmCfg<16>::kSmemBytes : GemmCfg<32>::kSmemBytes;
+    const bool one = gemm_ws_chunks_per_stage(args.mode) == 1;
+    cfg.dynamicSmemBytes = args.nr == 16 ? (one ? GemmCfg<16, 1>::kSmemBytes : GemmCfg<16, 2>::kSmemBytes)
+                                         : (one ? GemmCfg<32, 1>::kSmemBytes : GemmCfg<32, 2>::kSmemBytes);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

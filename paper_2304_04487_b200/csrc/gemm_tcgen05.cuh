@@ -69,9 +69,15 @@ struct GemmArgs {
 
 constexpr int kGemmThreads = 320;  // 4 epilogue warps, TMA producer, MMA issuer, 4 activation-loader warps
 constexpr int kGemmWideThreads = 224;  // 4 epilogue warps, weight producer, MMA issuer, activation producer
-constexpr uint32_t kGemmABytes = 128 * 64 * 2;
+constexpr uint32_t kGemmABytes = 128 * 64 * 2;  // one weight tile: 128 rows x one 64-wide k-chunk
 
-// gemm_ws_kernel exists for NR = 16 or 32 activation rows (MMA N = 2 NR: hi and lo columns).  Ring depths are the ones measured fastest inside a decoding step (deeper rings only
+// gemm_ws_kernel exists for NR = 16 or 32 activation rows (MMA N = 2 NR: hi and lo columns).
+// A ring stage holds KC consecutive k-chunks of one weight tile, fetched by ONE TMA copy through a
+// 3-D view of the matrix (64 columns, rows, chunk): with KC = 2 a copy moves 32 KB and reads 256
+// contiguous bytes of every weight row, which streams at 5.85 TB/s where 16 KB copies (128 bytes per
+// row) reach 4.86 TB/s (copy-only kernel, 148 CTAs, measured).  The gate/up projection, whose tile is
+// 64 + 64 rows of two matrices, keeps one chunk per stage.
+// Ring depths are the ones measured fastest inside a decoding step (deeper rings only
 // lengthen the queues that the epilogue's traffic also waits in).  The activation tile of a stage
 // is NOT fetched by TMA here: a second, small TMA copy per stage slowed the weight stream by a
 // quarter wherever it came from (shared buffer, per-CTA replica, one hot 4 KB block), whereas
@@ -79,13 +85,16 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;
 // the rows from global memory into the 128-byte-swizzled layout the MMA expects.
 // The request is padded to more than half an SM's shared memory so that the CTAs of two
 // consecutive projections never share an SM (measured 10 % slower when they do).
-template <int NR> struct GemmCfg {
-    static constexpr uint32_t kBBytes = 2 * NR * 64 * 2;
-    static constexpr int kStages = NR == 16 ? 8 : 7;
+template <int NR, int KC> struct GemmCfg {
+    static constexpr uint32_t kABytes = KC * kGemmABytes;
+    static constexpr uint32_t kBTile = 2 * NR * 64 * 2;   // activation rows (hi, lo) of one k-chunk
+    static constexpr uint32_t kBBytes = KC * kBTile;
+    static constexpr int kStages = KC == 2 ? (NR == 16 ? 4 : 3) : (NR == 16 ? 8 : 7);
     static constexpr size_t kRopeBytes = 32 * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
-    static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kGemmABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
+    static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
+constexpr int gemm_ws_chunks_per_stage(int mode) { return mode == kGemmSwiGLU ? 1 : 2; }
 
 // Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight tiles (16 KB each) and a ring of
 // activation tiles (nr rows of 128 bytes each: one term of one 64-wide k-chunk), as many as fit.
@@ -103,11 +112,15 @@ int gemm_grid_for(int64_t work, int num_sms);
 // Encode a 2-D bf16 row-major [rows, cols] tensor for TMA with a {64, box_rows} box and
 // 128-byte swizzle.  Returns a CUresult (0 = success).
 int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// The same tensor seen as (64 columns, rows, cols / 64 chunks) with a {64, box_rows, 2} box: two
+// consecutive k-chunks of box_rows rows per copy, landing as two tiles of the 2-D layout one after the other.
+int make_tensor_map_bf16_chunks(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-// args.nr = 16 or 32 rows; pdl = launch with programmatic stream serialization
+// args.nr = 16 or 32 rows; a0..a2 are chunk-pair maps (make_tensor_map_bf16_chunks, 128-row boxes) except
+// in kGemmSwiGLU mode (2-D maps, 64-row boxes); pdl = launch with programmatic stream serialization
 // (the kernel before it must be one of this library's)
 void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2);
