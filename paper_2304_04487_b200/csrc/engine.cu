@@ -185,6 +185,8 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         CREATE_TRY(dalloc(&e->norm_ss, (size_t)((d.d_model + 127) / 128) * RC));
         e->maps.resize(L);
         e->maps2.resize(L);
+        e->gate_up_map.resize(L);
+        bool pair_ok = true;
         int bad = 0;
         for (int l = 0; l < L; ++l) {
             llma_engine::LayerMaps& m = e->maps[l];
@@ -202,12 +204,16 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
             bad |= make_tensor_map_bf16_chunks(&m2.wo, e->wo[l], d.d_model, HD, 128);
             bad |= make_tensor_map_bf16_chunks(&m2.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
             m2.w_gate = m.w_gate; m2.w_up = m.w_up;
+            // one view over both matrices; if they lie too far apart for one, every pass uses the wide kernel
+            if (make_tensor_map_bf16_pair(&e->gate_up_map[l].map, e->w_gate[l], e->w_up[l], d.d_ffn, d.d_model,
+                                          &e->gate_up_map[l].gate_second) != 0)
+                pair_ok = false;
         }
         bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
         bad |= make_tensor_map_bf16_chunks(&e->map_lm_head2, e->lm_head, d.vocab, d.d_model, 128);
         // the MMA shape of decoding steps is fixed per engine (by its row capacity), never per step
-        e->decode_wide = e->decode_rows > 32;
-        e->decode_nr = e->decode_wide ? e->decode_rows : (e->decode_rows <= 16 ? 16 : 32);
+        e->decode_wide = e->decode_rows > 32 || !pair_ok;
+        e->decode_nr = e->decode_wide ? std::max(e->decode_rows, 32) : (e->decode_rows <= 16 ? 16 : 32);
         // activation operands of the wide kernel: one box of nr rows per (buffer, use)
         auto act_maps = [&](llma_engine::ActMaps& m, int nr) {
             int bad2 = 0;
@@ -217,7 +223,7 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
             return bad2;
         };
         bad |= act_maps(e->act_prefill, e->prefill_rows);
-        if (e->decode_wide) bad |= act_maps(e->act_decode, e->decode_rows);
+        if (e->decode_wide) bad |= act_maps(e->act_decode, e->decode_nr);
         if (bad) { free_engine(e); return LLMA_ERR_CONFIG; }  // misaligned weight pointer or bad shape
         CREATE_TRY(init_gemm_tcgen05());
         CREATE_TRY(init_gemm_wide());

@@ -43,6 +43,8 @@ struct llma_engine {
     std::vector<LayerMaps> maps;    // 2-D views (gemm_wide_kernel; gate/up of both kernels)
     std::vector<LayerMaps> maps2;   // chunk-pair views (gemm_ws_kernel; gate/up entries are the 2-D ones)
     CUtensorMap map_lm_head, map_lm_head2;
+    struct PairMap { CUtensorMap map; int gate_second; };   // gate and up matrices of a layer in one view (gemm_ws_kernel)
+    std::vector<PairMap> gate_up_map;
     struct ActMaps { CUtensorMap x_hat, attn, h; };  // activation operands of gemm_wide_kernel, box of nr rows
     ActMaps act_decode, act_prefill;
     bool decode_wide = false;       // decoding steps of more than 32 rows use gemm_wide_kernel

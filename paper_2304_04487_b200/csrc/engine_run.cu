@@ -81,7 +81,12 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         with_norm(e, gu);
         gu.out_act = e->h;
-        run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat, am ? &am->x_hat : nullptr);
+        if (e->cur_wide) {
+            run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat, &am->x_hat);
+        } else {  // one view over both matrices; whichever lies lower in memory fills the tile's first 64 rows
+            gu.gate_second = e->gate_up_map[l].gate_second;
+            run_gemm(e, gu, e->gate_up_map[l].map, e->gate_up_map[l].map, e->gate_up_map[l].map, e->x_hat, nullptr);
+        }
         mark(e, LLMA_K_GEMM_GATEUP);
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;

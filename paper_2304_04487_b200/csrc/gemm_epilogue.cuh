@@ -125,7 +125,7 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
     if (f < g.n_out) {
 #pragma unroll 1
         for (int j = row >> 6; j < nj; j += 2) {
-            const float gate = stage[fi][j], up = stage[64 + fi][j];
+            const float gate = stage[g.gate_second ? 64 + fi : fi][j], up = stage[g.gate_second ? fi : 64 + fi][j];
             store_act(g.out_act, kActSplit, g.rc, jb + j, f, g.n_out, gate / (1.f + expf(-gate)) * up);
         }
     }

@@ -34,8 +34,8 @@ template <int NR, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_a2) {
-    constexpr int KC = gemm_ws_chunks_per_stage(MODE);  // 64-wide k-chunks per ring stage (one TMA copy)
-    using Cfg = GemmCfg<NR, KC>;
+    constexpr int KC = kGemmKC;             // 64-wide k-chunks per ring stage (one TMA copy)
+    using Cfg = GemmCfg<NR>;
     constexpr int NT = 2;                   // bf16 terms of the activation operand: hi, lo
     constexpr uint32_t kTmemCols = 4 * NR;  // two accumulators of 2 NR columns
     constexpr int S = Cfg::kStages;
@@ -82,7 +82,6 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     if (warp == 4 && lane == 0) {
         tma_prefetch_desc(&map_a0);
         if (MODE == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
-        if (MODE == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
     }
     tc_fence_before();
     __syncthreads();
@@ -95,11 +94,10 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             auto load_a = [&](int64_t w, int s) {
                 const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
                 const uint32_t dstA = sA + s * kABytes;
-                if (MODE == kGemmSwiGLU) {
-                    tma_load_2d(dstA, &map_a0, full_bar(s), c * 64, tile * 64);
-                    tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_bar(s), c * 64, tile * 64);
+                // chunks 2c and 2c+1 of the tile in one copy (a chunk past the matrix arrives as zeros)
+                if (MODE == kGemmSwiGLU) {  // 64 rows of each of the two matrices per chunk
+                    tma_load_4d(dstA, &map_a0, full_bar(s), 0, tile * 64, 0, c * KC);
                 } else {
-                    // chunks 2c and 2c+1 of the tile in one copy (a chunk past the matrix arrives as zeros)
                     const int m = tile / g.tiles_per_map, r0 = (tile % g.tiles_per_map) * 128;
                     const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
                     tma_load_3d(dstA, mp, full_bar(s), 0, r0, c * KC);
@@ -454,6 +452,23 @@ int make_tensor_map_bf16_chunks(CUtensorMap* out, const void* base, uint64_t row
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+int make_tensor_map_bf16_pair(CUtensorMap* out, const void* base0, const void* base1, uint64_t rows, uint64_t cols,
+                              int* swapped) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || cols % 64 || base0 == base1) return -1;
+    const uintptr_t p0 = (uintptr_t)base0, p1 = (uintptr_t)base1;
+    *swapped = p1 < p0 ? 1 : 0;
+    const uintptr_t lo = *swapped ? p1 : p0, diff = *swapped ? p0 - p1 : p1 - p0;
+    if (diff % 16 || diff >= (1ull << 40) || diff < rows * cols * 2) return -1;
+    const cuuint64_t dims[4] = {64, rows, 2, cols / 64};
+    const cuuint64_t strides[3] = {cols * 2, (cuuint64_t)diff, 128};
+    const cuuint32_t box[4] = {64, 64, 2, 2};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return (int)fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, reinterpret_cast<void*>(lo), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return -1;
@@ -469,7 +484,7 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 template <int NR, int MODE>
 static cudaError_t opt_in() {
     return cudaFuncSetAttribute(gemm_ws_kernel<NR, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)GemmCfg<NR, gemm_ws_chunks_per_stage(MODE)>::kSmemBytes);
+                                (int)GemmCfg<NR>::kSmemBytes);
 }
 template <int NR>
 static cudaError_t opt_in_all() {
@@ -504,9 +519,7 @@ void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& ar
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kGemmThreads);
-    const bool one = gemm_ws_chunks_per_stage(args.mode) == 1;
-    cfg.dynamicSmemBytes = args.nr == 16 ? (one ? GemmCfg<16, 1>::kSmemBytes : GemmCfg<16, 2>::kSmemBytes)
-                                         : (one ? GemmCfg<32, 1>::kSmemBytes : GemmCfg<32, 2>::kSmemBytes);
+    cfg.dynamicSmemBytes = args.nr == 16 ? GemmCfg<16>::kSmemBytes : GemmCfg<32>::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

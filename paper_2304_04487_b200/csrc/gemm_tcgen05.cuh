@@ -26,7 +26,7 @@ namespace llma {
 enum GemmMode : int32_t {
     kGemmQKV = 0,     // A maps = {wq, wk, wv}; rotary embedding; q -> qkv buffer, k/v -> cache
     kGemmResid = 1,   // x[r, n] += acc
-    kGemmSwiGLU = 2,  // A maps = {w_gate, w_up}, 64 + 64 rows per tile; h = silu(g) * u (bf16)
+    kGemmSwiGLU = 2,  // A maps = {w_gate, w_up}, 64 + 64 rows per tile; h = silu(g) * u (split bf16)
     kGemmLmHead = 3,  // per-tile (max, argmax) per row; optional logits store
     kGemmStore = 4,   // out[r, n] = acc for all rows (stand-alone product)
 };
@@ -46,6 +46,7 @@ struct GemmArgs {
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
     int32_t ld;             // leading dimension of out_f32
     void* out_act;          // SwiGLU: h in ActLayout kActSplit [2 rc][d_ffn]
+    int32_t gate_second;    // SwiGLU: 1 when the tile's rows 0..63 are the up features and 64..127 the gate features
     // RMSNorm folded into the projections: the producer of the residual stream x writes
     // xs = split(x * gain) and, per 128-column tile, the rows' sums of squares; the consumer
     // multiplies its accumulators by rsqrt(sum / norm_dim + eps), which equals projecting the
@@ -76,7 +77,8 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;  // one weight tile: 128 rows x o
 // 3-D view of the matrix (64 columns, rows, chunk): with KC = 2 a copy moves 32 KB and reads 256
 // contiguous bytes of every weight row, which streams at 5.85 TB/s where 16 KB copies (128 bytes per
 // row) reach 4.86 TB/s (copy-only kernel, 148 CTAs, measured).  The gate/up projection, whose tile is
-// 64 + 64 rows of two matrices, keeps one chunk per stage.
+// 64 + 64 rows of two matrices, does the same through a 4-D view that spans both matrices (64 columns,
+// rows, matrix, chunk): one copy lands, for each of the two chunks, the 64 gate rows followed by the 64 up rows.
 // Ring depths are the ones measured fastest inside a decoding step (deeper rings only
 // lengthen the queues that the epilogue's traffic also waits in).  The activation tile of a stage
 // is NOT fetched by TMA here: a second, small TMA copy per stage slowed the weight stream by a
@@ -85,16 +87,16 @@ constexpr uint32_t kGemmABytes = 128 * 64 * 2;  // one weight tile: 128 rows x o
 // the rows from global memory into the 128-byte-swizzled layout the MMA expects.
 // The request is padded to more than half an SM's shared memory so that the CTAs of two
 // consecutive projections never share an SM (measured 10 % slower when they do).
-template <int NR, int KC> struct GemmCfg {
-    static constexpr uint32_t kABytes = KC * kGemmABytes;
+constexpr int kGemmKC = 2;  // 64-wide k-chunks per ring stage
+template <int NR> struct GemmCfg {
+    static constexpr uint32_t kABytes = kGemmKC * kGemmABytes;
     static constexpr uint32_t kBTile = 2 * NR * 64 * 2;   // activation rows (hi, lo) of one k-chunk
-    static constexpr uint32_t kBBytes = KC * kBTile;
-    static constexpr int kStages = KC == 2 ? (NR == 16 ? 4 : 3) : (NR == 16 ? 8 : 7);
+    static constexpr uint32_t kBBytes = kGemmKC * kBTile;
+    static constexpr int kStages = NR == 16 ? 4 : 3;
     static constexpr size_t kRopeBytes = 32 * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
     static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
-constexpr int gemm_ws_chunks_per_stage(int mode) { return mode == kGemmSwiGLU ? 1 : 2; }
 
 // Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight tiles (16 KB each) and a ring of
 // activation tiles (nr rows of 128 bytes each: one term of one 64-wide k-chunk), as many as fit.
@@ -115,12 +117,17 @@ int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 // The same tensor seen as (64 columns, rows, cols / 64 chunks) with a {64, box_rows, 2} box: two
 // consecutive k-chunks of box_rows rows per copy, landing as two tiles of the 2-D layout one after the other.
 int make_tensor_map_bf16_chunks(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// Two matrices [rows, cols] of equal shape seen as (64 columns, rows, matrix, chunk) with a {64, 64, 2, 2} box: one
+// copy lands [chunk][matrix][64 rows].  The matrix at the lower address comes first: *swapped = 1 if that is
+// base1.  Fails (non-zero) when the two allocations are more than 2^40 bytes apart.
+int make_tensor_map_bf16_pair(CUtensorMap* out, const void* base0, const void* base1, uint64_t rows, uint64_t cols,
+                              int* swapped);
 
 // Opt the kernel into its dynamic shared-memory size (once per process, outside any capture).
 cudaError_t init_gemm_tcgen05();
 
-// args.nr = 16 or 32 rows; a0..a2 are chunk-pair maps (make_tensor_map_bf16_chunks, 128-row boxes) except
-// in kGemmSwiGLU mode (2-D maps, 64-row boxes); pdl = launch with programmatic stream serialization
+// args.nr = 16 or 32 rows; a0..a2 are chunk-pair maps (make_tensor_map_bf16_chunks, 128-row boxes); in
+// kGemmSwiGLU mode a0 is the map over both matrices (make_tensor_map_bf16_pair); pdl = launch with programmatic stream serialization
 // (the kernel before it must be one of this library's)
 void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2);
