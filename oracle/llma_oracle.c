@@ -58,6 +58,10 @@ typedef struct {
     float *kcache, *vcache; /* [layer][pos][H*hd] */
     float *x, *h, *q, *k, *v, *att, *gate, *up, *tmp;
     double *scores;
+    /* prescribed cache codes for the next forward call (see oracle_prescribe_kv), or NULL */
+    const float *given_k, *given_v;
+    double given_tol;
+    double *given_stats;
 } oracle_model;
 
 /* ---- scalar helpers ------------------------------------------------------- */
@@ -153,6 +157,54 @@ void oracle_silu_mul(const float *g, const float *u, int32_t n, float *out) {
     }
 }
 
+/* ---- prescribed cache codes -------------------------------------------------
+ * The cache is bf16 by definition, so a cached element is a quantised code decided by an
+ * fp32 value.  Two correct computations whose values differ in their last bits can fall on
+ * different sides of a rounding boundary, and the two codes then differ by a whole bf16 step,
+ * a difference thousands of times larger than its cause.  A comparison may therefore
+ * PRESCRIBE the codes.  A prescribed code g is accepted for an element whose unrounded value
+ * here is x iff
+ *        |g - x| <= step(x) / 2 + tol * max(1, max |row|)
+ * i.e. iff g is what rounding to nearest gives for SOME value within the stated absolute
+ * tolerance of x (step = spacing of bf16 values at the larger of |x|, |g|; the tolerance is the
+ * one the projection itself is held to).  Anything else is counted as a violation and the
+ * oracle keeps its own code.  stats[0] counts elements whose prescribed code differs from the
+ * oracle's own rounding, stats[1] the violations, stats[2] is the largest share of the
+ * tolerance an accepted difference needed, (|g - x| - step / 2) / (tol * max(1, max|row|)),
+ * stats[3] counts all elements seen. */
+static void adopt_codes(const float *own, const float *given, float *dst, int64_t n, double tol, double *stats) {
+    double rowmax = 1.0;
+    for (int64_t i = 0; i < n; ++i)
+        if (fabs((double)own[i]) > rowmax) rowmax = fabs((double)own[i]);
+    const double slack = tol * rowmax;
+    for (int64_t i = 0; i < n; ++i) {
+        const float r = oracle_round_bf16(own[i]);
+        const float g = given[i];
+        stats[3] += 1.0;
+        if (g == r) { dst[i] = r; continue; }
+        stats[0] += 1.0;
+        const double x = own[i];
+        const double big = fabs((double)g) > fabs(x) ? fabs((double)g) : fabs(x);
+        int e;
+        (void)frexp(big, &e);
+        const double step = ldexp(1.0, e - 8); /* spacing of bf16 values at this magnitude */
+        const double excess = fabs((double)g - x) - 0.5 * step;
+        if (excess <= slack) {
+            if (excess / slack > stats[2]) stats[2] = excess / slack;
+            dst[i] = g;
+        } else {
+            stats[1] += 1.0;
+            dst[i] = r;
+        }
+    }
+}
+
+/* k_rows, v_rows: [n_layers][H*hd] codes for the position of the NEXT oracle_forward call (used once);
+ * tol: the relative tolerance above; stats: double[4], accumulated into (the caller zeroes it). */
+void oracle_prescribe_kv(oracle_model *m, const float *k_rows, const float *v_rows, double tol, double *stats) {
+    m->given_k = k_rows; m->given_v = v_rows; m->given_tol = tol; m->given_stats = stats;
+}
+
 /* ---- model ---------------------------------------------------------------- */
 
 oracle_model *oracle_create(const oracle_config *cfg, const oracle_weights *w) {
@@ -215,9 +267,14 @@ int32_t oracle_forward(oracle_model *m, int32_t token, int32_t pos, float *logit
             oracle_rope(m->q + (int64_t)hI * hd, hd, pos, c->rope_theta);
             oracle_rope(m->k + (int64_t)hI * hd, hd, pos, c->rope_theta);
         }
-        for (int64_t i = 0; i < hh; ++i) {
-            Kl[(int64_t)pos * hh + i] = c->kv_round_bf16 ? oracle_round_bf16(m->k[i]) : m->k[i];
-            Vl[(int64_t)pos * hh + i] = c->kv_round_bf16 ? oracle_round_bf16(m->v[i]) : m->v[i];
+        if (m->given_k && c->kv_round_bf16) {
+            adopt_codes(m->k, m->given_k + (int64_t)l * hh, Kl + (int64_t)pos * hh, hh, m->given_tol, m->given_stats);
+            adopt_codes(m->v, m->given_v + (int64_t)l * hh, Vl + (int64_t)pos * hh, hh, m->given_tol, m->given_stats);
+        } else {
+            for (int64_t i = 0; i < hh; ++i) {
+                Kl[(int64_t)pos * hh + i] = c->kv_round_bf16 ? oracle_round_bf16(m->k[i]) : m->k[i];
+                Vl[(int64_t)pos * hh + i] = c->kv_round_bf16 ? oracle_round_bf16(m->v[i]) : m->v[i];
+            }
         }
         for (int32_t hI = 0; hI < H; ++hI)
             oracle_attention(m->q + (int64_t)hI * hd, Kl + (int64_t)hI * hd, Vl + (int64_t)hI * hd, pos + 1, hh, hd,
@@ -232,6 +289,7 @@ int32_t oracle_forward(oracle_model *m, int32_t token, int32_t pos, float *logit
         oracle_matvec(m->w.w_down[l], wb, d, F, m->gate, m->tmp);
         for (int32_t i = 0; i < d; ++i) m->x[i] += m->tmp[i];
     }
+    m->given_k = m->given_v = NULL;
     if (hidden) memcpy(hidden, m->x, (size_t)d * sizeof(float));
     if (logits) {
         oracle_rmsnorm(m->x, m->w.final_norm, d, c->rms_eps, m->h);

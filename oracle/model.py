@@ -44,6 +44,7 @@ def lib() -> C.CDLL:
         L.oracle_destroy.argtypes = [C.c_void_p]
         L.oracle_forward.restype = C.c_int32
         L.oracle_forward.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.oracle_prescribe_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_void_p]
         L.oracle_read_cache.restype = C.c_int32
         L.oracle_read_cache.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         L.oracle_round_bf16.restype = C.c_float
@@ -136,12 +137,23 @@ class OracleModel:
                      arr_of("ffn_norm"), arr_of("w_gate"), arr_of("w_up"), arr_of("w_down"))
         cfg = _Cfg(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                    int(bf16), int(bool(kv_round_bf16)), max_seq, shape.rms_eps, shape.rope_theta)
+        self.code_stats = np.zeros(4, np.float64)
         self._h = lib().oracle_create(C.byref(cfg), C.byref(w))
         if not self._h:
             raise MemoryError("oracle_create failed")
 
-    def forward(self, token: int, pos: int, want_logits: bool = True) -> Optional[np.ndarray]:
+    def forward(self, token: int, pos: int, want_logits: bool = True, given_kv=None, code_tol: float = 1e-4
+                ) -> Optional[np.ndarray]:
+        """``given_kv = (K, V)``, float32 [n_layers, H*hd]: prescribed bf16 cache codes of this position.  A code
+        is adopted only if rounding some value within ``code_tol * max(1, max|row|)`` of the oracle's own unrounded
+        value gives it; ``self.code_stats`` = differing elements, violations, largest share of the tolerance used,
+        elements seen."""
         out = np.empty(self.vocab, np.float32) if want_logits else None
+        if given_kv is not None:
+            gk = np.ascontiguousarray(given_kv[0], np.float32); gv = np.ascontiguousarray(given_kv[1], np.float32)
+            assert gk.shape == gv.shape == (self.shape.n_layers, self.shape.n_heads * self.shape.head_dim)
+            self._given = (gk, gv)                      # kept alive across the call
+            lib().oracle_prescribe_kv(self._h, _p(gk), _p(gv), float(code_tol), _p(self.code_stats))
         rc = lib().oracle_forward(self._h, int(token), int(pos), _p(out) if want_logits else None, None)
         if rc != 0:
             raise ValueError(f"oracle_forward({token}, {pos}) rejected its arguments")

@@ -84,20 +84,21 @@ extern "C" int llma_debug_kv_row(llma_engine* e, int32_t layer, int32_t seq, int
     CU_TRY(cudaStreamSynchronize(e->stream));
     const char* base = (const char*)(which ? e->vcache : e->kcache);
     const size_t es = e->bf16 ? 2 : 4;
-    std::vector<unsigned char> tmp((size_t)d.head_dim * es);
-    for (int h = 0; h < d.n_heads; ++h) {
-        const size_t off = (size_t)kv_row_index(d, layer, seq, h, pos) * d.head_dim * es;
-        CU_TRY(cudaMemcpy(tmp.data(), base + off, tmp.size(), cudaMemcpyDeviceToHost));
-        for (int i = 0; i < d.head_dim; ++i) {
-            float v;
-            if (e->bf16) {
-                uint32_t u = (uint32_t)(((const uint16_t*)tmp.data())[i]) << 16;
-                std::memcpy(&v, &u, 4);
-            } else {
-                v = ((const float*)tmp.data())[i];
-            }
-            out[(size_t)h * d.head_dim + i] = v;
+    // one strided copy: the row of every head (heads are max_seq rows apart in the cache)
+    std::vector<unsigned char> tmp((size_t)d.n_heads * d.head_dim * es);
+    const size_t off = (size_t)kv_row_index(d, layer, seq, 0, pos) * d.head_dim * es;
+    CU_TRY(cudaMemcpy2D(tmp.data(), (size_t)d.head_dim * es, base + off, (size_t)d.max_seq * d.head_dim * es,
+                        (size_t)d.head_dim * es, (size_t)d.n_heads, cudaMemcpyDeviceToHost));
+    const size_t n = (size_t)d.n_heads * d.head_dim;
+    for (size_t i = 0; i < n; ++i) {
+        float v;
+        if (e->bf16) {
+            uint32_t u = (uint32_t)(((const uint16_t*)tmp.data())[i]) << 16;
+            std::memcpy(&v, &u, 4);
+        } else {
+            v = ((const float*)tmp.data())[i];
         }
+        out[i] = v;
     }
     return LLMA_OK;
 }

@@ -6,7 +6,7 @@ from oracle import decoding as D
 from oracle import model as OM
 from workloads import SHAPES, ModelShape, build_reference, make_prompt, make_weights
 
-from parity import bf16_logit_tolerance, step_parity, step_parity_batch
+from parity import BF16_LOGIT_TOL, step_parity, step_parity_batch
 
 pytestmark = pytest.mark.gpu
 
@@ -66,6 +66,26 @@ def test_bf16_stepwise_parity(name, n, k, P, N):
     assert rep.max_logit_err <= 2e-2
     assert rep.near_ties <= 3, rep.near_ties
     assert rep.trigger_steps > 0
+
+
+def test_bf16_parity_with_prescribed_cache_codes():
+    """The same comparison with the cache's quantisation decisions taken alike on both sides: every code the engine
+    stored must be the rounding of a value within 1e-4 of the row scale of the oracle's unrounded value, differing
+    codes must be rare, and the logits then agree far inside the tolerance."""
+    shape = SHAPES["small-bf16"]
+    w = _weights(shape)
+    P, N, k = 150, 24, 8
+    prompt = make_prompt(P, shape.vocab, seed=2)
+    max_seq = P + N + 40
+    y_star = _greedy_star(shape, w, prompt, N, max_seq)
+    ref, offs, _ = build_reference(y_star, [60, 60, 40], 0.7, shape.vocab, seed=1)
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=200, max_k=k, keep_logits=True)
+    rep = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, offs, 1, k, N, "bf16",
+                      prescribe_kv=True)
+    assert rep.code_violations == 0 and rep.codes_seen > 100000
+    assert rep.code_flips <= 0.01 * rep.codes_seen
+    assert rep.max_logit_err <= 5e-3 and rep.near_ties <= 1
+    eng.llma_destroy()
 
 
 # ---- the whole loop: llma_generate vs Algorithm 1 on the oracle, LLMA == greedy on the GPU -----------
@@ -334,7 +354,14 @@ def test_wide_two_layer_stepwise_parity(name, k):
 def test_llama7b_shape_sampled_parity():
     """Full-size check in the configuration the benchmark times (7B-shaped bf16 decoder, engine created
     for k = 8): a short prompt, then LLMA steps whose every logits row is compared with the oracle.  The
-    oracle needs about a second per position at this size, so only a few dozen positions are sampled."""
+    oracle needs about a second per position at this size, so only a few dozen positions are sampled.
+
+    Two runs.  (1) Both sides take the cache's quantisation decisions alike (the oracle adopts the engine's bf16
+    code wherever it is the rounding of a value within 1e-4 of the row scale of its own unrounded value): logits
+    within the flat 2e-2, no code outside that rule, differing codes rare.  (2) Free-running: every layer's flips feed
+    the next layer, the effect on the logits grows with depth (about 2.4e-2 at 32 layers with tensor-core
+    accumulation, 1.3e-2 with fp32 FMA accumulation, unchanged by a third bf16 term of the activations); the
+    figure is printed, tokens must still agree except at near-ties."""
     shape = SHAPES["llama7b-shape"]
     w = _weights(shape)
     prompt = make_prompt(20, shape.vocab, seed=11)
@@ -344,10 +371,19 @@ def test_llama7b_shape_sampled_parity():
     ref = y_star[:8] + [shape.vocab - 1, shape.vocab - 2]                 # one span that is accepted, then junk
     eng = _engine(shape, w, max_seq=max_seq, max_ref=32, max_k=8, keep_logits=True)
     assert eng.llma_gemm_impl() == 2
-    om2 = OM.OracleModel(shape, w, max_seq=max_seq)
-    rep = step_parity(eng, om2, prompt, ref, None, 1, 8, 10, "bf16")
-    assert rep.max_logit_err <= bf16_logit_tolerance(shape.n_layers)
+    rep = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, None, 1, 8, 10, "bf16",
+                      prescribe_kv=True)
+    assert rep.max_logit_err <= BF16_LOGIT_TOL
+    assert rep.code_violations == 0
+    assert rep.code_flips <= 0.05 * rep.codes_seen                        # about 2 % at these widths (k = 4096 products per element)
     assert rep.rows_compared >= 10 and rep.trigger_steps >= 1 and rep.copied_accepted >= 4
     assert rep.tokens[:10] == y_star or rep.near_ties > 0
-    print(f"7B-shape parity: rows {rep.rows_compared}, max |dlogit| {rep.max_logit_err:.2e}, near ties {rep.near_ties}")
+    eng.llma_reset(0)
+    free = step_parity(eng, OM.OracleModel(shape, w, max_seq=max_seq), prompt, ref, None, 1, 8, 10, "bf16",
+                       check_logits=False)
+    assert free.tokens[:10] == y_star or free.near_ties > 0
+    assert free.max_logit_err <= 5e-2                                     # a gross error would not hide behind the drift
+    print(f"7B-shape parity: rows {rep.rows_compared}; cache codes prescribed: max |dlogit| {rep.max_logit_err:.2e}, "
+          f"{rep.code_flips} of {rep.codes_seen} codes differ ({rep.code_boundary_dist:.2f} of the code tolerance used); "
+          f"free-running: max |dlogit| {free.max_logit_err:.2e}, near ties {free.near_ties}")
     _cache.clear()                                                        # 13 GB of host weights

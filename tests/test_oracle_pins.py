@@ -456,3 +456,50 @@ def test_llma_equals_greedy_real_model(shape):
             assert D.simulate_decoding_sequence(y, ref, offs, n, k) == [(1 + s.k_eff, s.emitted) for s in r.trace]
     r = D.llma_decode(OM.OracleModel(shape, w, max_seq=80), prompt, y, None, 1, 4, N)
     assert r.steps < N / 2       # with the output itself as reference most steps emit several tokens
+
+
+def test_prescribed_cache_codes_are_checked():
+    """oracle_prescribe_kv: a prescribed bf16 code g is adopted for an unrounded value x iff
+    |g - x| <= step / 2 + tol * max(1, max|row|); the rule is restated here in numpy and compared element by element.
+    The oracle's own codes change nothing; refused codes leave the oracle's own in place."""
+    shape, w = MICRO_BF16, make_weights(MICRO_BF16, seed=3, std=0.3)
+    HD = shape.n_heads * shape.head_dim
+    tok, pos, tol = 5, 0, 4e-4
+    exact = OM.OracleModel(shape, w, max_seq=4, kv_round_bf16=False)      # cache rows unrounded
+    exact.forward(tok, pos)
+    own = OM.OracleModel(shape, w, max_seq=4)
+    base = own.forward(tok, pos)
+    # layer 0's unrounded rows are the same in both models (nothing upstream of them is rounded)
+    k_un = exact.read_cache(0, pos, 0)
+    k_own = np.stack([own.read_cache(l, pos, 0) for l in range(shape.n_layers)])
+    v_own = np.stack([own.read_cache(l, pos, 1) for l in range(shape.n_layers)])
+    assert np.array_equal(bf16_bits_from_f32(k_un), bf16_bits_from_f32(k_own[0]))
+
+    def neighbour(codes_f32, towards):                                    # the bf16 value next to each code, on the side of `towards`
+        bits = bf16_bits_from_f32(codes_f32).astype(np.int32)
+        step = np.where(codes_f32 >= 0, 1, -1) * np.where(towards > codes_f32, 1, -1)
+        return f32_from_bf16_bits((bits + step).astype(np.uint16))
+
+    def rule(g, x):                                                       # the acceptance rule, restated
+        big = np.maximum(np.abs(g.astype(np.float64)), np.abs(x.astype(np.float64)))
+        step = 2.0 ** (np.floor(np.log2(big)) + 1 - 8)
+        return np.abs(g.astype(np.float64) - x) - 0.5 * step <= tol * max(1.0, float(np.abs(x).max()))
+
+    # (1) the oracle's own codes: nothing differs, same logits
+    m = OM.OracleModel(shape, w, max_seq=4)
+    got = m.forward(tok, pos, given_kv=(k_own, v_own), code_tol=tol)
+    assert np.array_equal(got, base) and m.code_stats[0] == 0 and m.code_stats[3] == 2 * shape.n_layers * HD
+    # (2) layer 0: every K element replaced by the code on the other side of its unrounded value, then (3) by the
+    # neighbouring code on the wrong side: adopted exactly where the rule says so
+    sel = k_un != k_own[0]
+    for towards in (k_un, 2 * k_own[0] - k_un):
+        given = k_own.copy()
+        given[0] = np.where(sel, neighbour(k_own[0], towards), k_own[0])
+        want_accept = rule(given[0], k_un) & sel
+        m = OM.OracleModel(shape, w, max_seq=4)
+        m.forward(tok, pos, given_kv=(given, v_own), code_tol=tol)
+        assert np.array_equal(m.read_cache(0, pos, 0), np.where(want_accept, given[0], k_own[0]))
+        assert m.code_stats[1] >= (sel & ~want_accept).sum() and m.code_stats[2] <= 1.0
+    given = k_own.copy()
+    given[0] = np.where(sel, neighbour(k_own[0], k_un), k_own[0])
+    assert 5 < (rule(given[0], k_un) & sel).sum() < sel.sum() - 5          # both branches of the rule were exercised
