@@ -49,7 +49,7 @@ def measured_traffic_ratio():
     """DRAM traffic / algorithmic bytes of the GEMM kernel from the committed ncu summary, or None
     when the kernel's sources have changed since those counters were taken."""
     import hashlib
-    prof = os.path.join(ROOT, "profiles", "gemm_ws_kernel_ncu_full_22016x4096.md")
+    prof = os.path.join(ROOT, "profiles", "gemm_ws_kernel_ncu_full_llama7b_2layer.md")
     src = [os.path.join(ROOT, "paper_2304_04487_b200", "csrc", f)
            for f in ("gemm_tcgen05.cu", "gemm_epilogue.cuh", "gemm_tcgen05.cuh", "ptx_sm100.cuh")]
     try:
@@ -646,7 +646,8 @@ def main():
     step_ms = dev_ms / max(steps_taken, 1)
     roofline = {"bound": "hbm", "kernel": "gemm_ws_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                # per launch, scaled from the ncu capture of a 180 MB launch (traffic grows with the matrix size)
+                # per launch, scaled from the ncu capture of three projections of the 2-layer model of the same
+                # widths (DRAM traffic grows in proportion to the matrix size)
                 "traffic": (None if measured_traffic_ratio() is None
                             else measured_traffic_ratio() * wbytes / max(gemm_launches, 1)),
                 "bytes_per_launch": wbytes / max(gemm_launches, 1), "us_per_launch": 1e3 * gemm_ms / max(gemm_launches, 1),
