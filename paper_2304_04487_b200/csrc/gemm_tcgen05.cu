@@ -272,15 +272,15 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, 0, rows_used, stage);
             else epilogue_lmhead(g, tile, row, 0, rows_used, stage, red_f, red_i);
         };
-        // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks
-        // its own partial (slot 0 of its workspace) and completes the tile after its last segment.  Every
-        // other CTA of the tile hands its partial over through slot 1, whose words hold the bit pattern
-        // kEmpty (a NaN no arithmetic here produces) while nothing has been handed over: the owner polls
-        // the words it needs until none is kEmpty, adds the partials in ascending k order, and puts kEmpty
-        // back.  No fence, counter or second pass: one store and one load stand between the last MMA of a
-        // neighbour and the owner's epilogue.
+        // Tiles cut by a range boundary.  The CTA whose range holds the tile's FIRST chunks owns it: that is
+        // the last thing it works on, so it completes the tile at once.  Every other CTA of the tile hands its
+        // partial over through its slot of the workspace, whose words hold the bit pattern kEmpty (a NaN no
+        // arithmetic here produces) while nothing has been handed over: the owner polls the words it needs
+        // until none is kEmpty, adds the partials in ascending k order (its own first), and puts kEmpty back.
+        // No fence, counter or second pass.  The CTA that holds a tile's LAST chunks works on them first, long
+        // before the owner asks: a tile cut in two costs its owner no wait at all; only CTAs whose whole range
+        // lies inside one tile finish together with the owner.
         constexpr uint32_t kEmpty = 0xFFFFFFFFu;
-        int own_tile = -1, own_first = 0;
         bool aborted = false;
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
@@ -321,93 +321,69 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
 
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
-            if (w_beg > t_lo || w_end < t_hi) {  // the tile is shared with a neighbour
-                const bool owner = w_end >= t_hi;
-                float4* dst = ws_slot(g.ws, NR / 4, b, owner ? 0 : 1, row);
+            if (w_beg > t_lo) {  // another CTA holds the tile's first chunks: hand this partial over to it
+                float4* dst = ws_slot(g.ws, NR / 4, b, 1, row);
 #pragma unroll
                 for (int q = 0; q < NR / 4; ++q)  // only the columns of rows in use travel
                     if (4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-                if (owner) {
-                    int b_first = (int)(t_lo * G / work);
-                    while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
-                    while (cta_begin(work, b_first, G) > t_lo) --b_first;
-                    own_tile = tile; own_first = b_first;
-                }
                 continue;
             }
-            finish_tile(tile, acc, xpre);
-        }
-        if (own_tile >= 0 && !aborted) {
-            float xpre[kXPre];
-            prefetch_x(own_tile, xpre);
-            float acc[32];
+            if (w_end < t_hi) {  // this CTA owns the tile; the CTAs after it hold the rest of its chunks
+                int b_last = (int)((t_hi - 1) * G / work);
+                while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
+                while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
+                const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
+                constexpr int kBatch = 2;
+                for (int bb = b + 1; bb <= b_last; bb += kBatch) {  // ascending k: a fixed summation order
+                    float4 p[kBatch][NR / 4];
+                    bool valid;
+                    do {
+                        valid = true;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-            // this CTA's own partial (parked in slot 0 by these same threads) is requested now and added last
-            float4 own[NR / 4];
-            {
-                const float4* src = ws_slot(g.ws, NR / 4, b, 0, row);
+                        for (int u = 0; u < kBatch; ++u) {
+                            if (bb + u <= b_last) {
+                                const float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
 #pragma unroll
-                for (int q = 0; q < NR / 4; ++q)
-                    if (4 * q < rows_used) own[q] = src[q * 128];
-            }
-            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
-            constexpr int kBatch = 2;
-            for (int bb = own_first; bb < b; bb += kBatch) {  // ascending k: a fixed summation order
-                float4 p[kBatch][NR / 4];
-                bool valid;
-                do {
-                    valid = true;
-#pragma unroll
-                    for (int u = 0; u < kBatch; ++u) {
-                        if (bb + u < b) {
-                            const float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
-#pragma unroll
-                            for (int q = 0; q < NR / 4; ++q)
-                                if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q * 128);
+                                for (int q = 0; q < NR / 4; ++q)
+                                    if (4 * q < rows_used) p[u][q] = ld_poll_f4(src + q * 128);
+                            }
                         }
-                    }
+#pragma unroll
+                        for (int u = 0; u < kBatch; ++u) {
+                            if (bb + u <= b_last) {
+#pragma unroll
+                                for (int q = 0; q < NR / 4; ++q) {
+                                    if (4 * q < rows_used) {
+                                        valid = valid && __float_as_uint(p[u][q].x) != kEmpty;
+                                        if (4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[u][q].y) != kEmpty;
+                                        if (4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[u][q].z) != kEmpty;
+                                        if (4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[u][q].w) != kEmpty;
+                                    }
+                                }
+                            }
+                        }
+                        if (!valid && globaltimer_ns() > give_up) { atomicExch(g.dev_err, kDevErrTimeout); break; }
+                    } while (!valid);
+                    const float e = __uint_as_float(kEmpty);
 #pragma unroll
                     for (int u = 0; u < kBatch; ++u) {
-                        if (bb + u < b) {
+                        if (bb + u <= b_last) {
+                            float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
 #pragma unroll
                             for (int q = 0; q < NR / 4; ++q) {
                                 if (4 * q < rows_used) {
-                                    valid = valid && __float_as_uint(p[u][q].x) != kEmpty;
-                                    if (4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[u][q].y) != kEmpty;
-                                    if (4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[u][q].z) != kEmpty;
-                                    if (4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[u][q].w) != kEmpty;
+                                    src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
+                                    acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
+                                    acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
                                 }
                             }
                         }
                     }
-                    if (!valid && globaltimer_ns() > give_up) { atomicExch(g.dev_err, kDevErrTimeout); break; }
-                } while (!valid);
-                const float e = __uint_as_float(kEmpty);
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    if (bb + u < b) {
-                        float4* src = ws_slot(g.ws, NR / 4, bb + u, 1, row);
-#pragma unroll
-                        for (int q = 0; q < NR / 4; ++q) {
-                            if (4 * q < rows_used) {
-                                src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
-                                acc[4 * q] += p[u][q].x; acc[4 * q + 1] += p[u][q].y;
-                                acc[4 * q + 2] += p[u][q].z; acc[4 * q + 3] += p[u][q].w;
-                            }
-                        }
-                    }
                 }
             }
-            // this CTA's own partial comes last (it holds the highest k)
-#pragma unroll
-            for (int q = 0; q < NR / 4; ++q) {
-                if (4 * q < rows_used) {
-                    acc[4 * q] += own[q].x; acc[4 * q + 1] += own[q].y; acc[4 * q + 2] += own[q].z; acc[4 * q + 3] += own[q].w;
-                }
-            }
-            finish_tile(own_tile, acc, xpre);
+            finish_tile(tile, acc, xpre);
         }
+        (void)aborted;
     }
     tc_fence_before();
     __syncthreads();

@@ -222,9 +222,13 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             else epilogue_lmhead(g, tile, row, jb, nj, stage, red_f, red_i);
             epi_sync();  // the staging area is rewritten by the next block
         };
-        // Tiles cut by a range boundary: see gemm_ws_kernel.  The hand-over slots hold nr / 4 row groups.
+        // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks its own
+        // partial in slot 0 of its workspace and completes the tile after its last segment; every other CTA of the tile
+        // hands its partial over through slot 1 (all-ones words while empty, see gemm_ws_kernel).
         constexpr uint32_t kEmpty = 0xFFFFFFFFu;
-        const int qn = nr >> 2;
+        // slots are laid out for the engine's row capacity whatever nr is: a prompt pass and a decoding step (different nr)
+        // then agree on where every CTA's slots are, and the never-emptied slot 0 of one cannot sit in a slot 1 of the other
+        const int qn = g.rc >> 2;
         int own_tile = -1, own_first = 0;
         bool aborted = false;
         int seg = 0;
