@@ -211,6 +211,14 @@ int llma_generate_forced(llma_engine *e, int32_t seq, const int32_t *trace, int3
  * 3 token range), as a kernel that gave up would have left it; the next step reports it.  Errors: ARG, CUDA. */
 int llma_debug_set_device_error(llma_engine *e, int32_t code);
 
+/* Measurement aid: in-kernel timestamps of the last decoding step's kernels (globaltimer, ns), copied to `out`
+ * (host, 512 x 160 x 8 words) when out != NULL and reset when clear != 0.  Block i < 300 belongs to the i-th
+ * projection launch of the step (one 8-word slot per CTA: CTA start, dependency released, first stage ready,
+ * last MMA issued, last accumulator ready, CTA end); blocks 300 + layer and 400 + layer hold (min, max) pairs
+ * of the attention kernel (CTA start, dependency released, K tile landed, CTA end) and of its merge kernel.
+ * Only a library built with -DLLMA_STAMPS records anything; otherwise LLMA_ERR_STATE.  Errors: NULL, STATE, CUDA. */
+int llma_debug_timeline(llma_engine *e, int32_t clear, unsigned long long *out);
+
 /* Rows the engine's activation buffers hold (the leading dimension of llma_debug_buffer), or a negative
  * status. */
 int llma_row_capacity(llma_engine *e);

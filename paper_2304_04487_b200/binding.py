@@ -57,7 +57,7 @@ _lib = None
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
            "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16",
-           "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity",
+           "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity", "llma_debug_timeline",
            "llma_last_cuda_error", "llma_strerror")
 
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
         L.llma_row_capacity.argtypes = [vp]
+        L.llma_debug_timeline.argtypes = [vp, i32, vp]
         L.llma_debug_set_device_error.argtypes = [vp, i32]
         L.llma_generate_forced.argtypes = [vp, i32, pi32, i32, pi32, i32, C.POINTER(LlmaStats)]
         L.llma_debug_buffer.argtypes = [vp, i32, C.POINTER(C.c_float), C.c_int64]
@@ -267,6 +268,12 @@ class Engine:
 
     def llma_row_capacity(self) -> int:
         return self._check(lib().llma_row_capacity(self._h), "llma_row_capacity")
+
+    def llma_debug_timeline(self, clear: bool = True) -> np.ndarray:
+        """Timestamps of the last step's kernels, uint64 [512, 160, 8] (a library built with LLMA_STAMPS only)."""
+        out = np.zeros((512, 160, 8), np.uint64)
+        self._check(lib().llma_debug_timeline(self._h, int(clear), out.ctypes.data), "llma_debug_timeline")
+        return out
 
     def llma_debug_set_device_error(self, code: int) -> None:
         self._check(lib().llma_debug_set_device_error(self._h, code), "llma_debug_set_device_error")

@@ -8,11 +8,14 @@ from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-OBJ = os.path.join(HERE, "_build")
+# LLMA_BUILD_STAMPS=1 builds the measurement variant (in-kernel timestamps, see LLMA_STAMPS in csrc/common.cuh)
+# into the same library name but a build folder of its own; switch back by rebuilding without the variable.
+STAMPS = os.environ.get("LLMA_BUILD_STAMPS") == "1"
+OBJ = os.path.join(HERE, "_build_stamps" if STAMPS else "_build")
 LIB = os.path.join(HERE, "libllma_b200.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
+         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"] + (["-DLLMA_STAMPS"] if STAMPS else [])
 
 
 def _sources():
@@ -48,8 +51,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=8) as ex:
         list(ex.map(run, jobs))
-    if force or jobs or _stale(LIB, objs):
+    marker = os.path.join(OBJ, ".linked")
+    if force or jobs or _stale(LIB, objs) or not os.path.exists(marker):
         run([NVCC, "-shared", "-o", LIB] + objs + ["-cudart", "static"])
+        for d in (os.path.join(HERE, "_build"), os.path.join(HERE, "_build_stamps")):   # the library now holds THIS variant
+            if os.path.exists(os.path.join(d, ".linked")):
+                os.remove(os.path.join(d, ".linked"))
+        open(marker, "w").close()
     return LIB
 
 

@@ -57,6 +57,9 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     using L = AttnSmem<HD>;
     pdl_trigger();
     const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    // timeline (min, max over the CTAs): 0/1 CTA start, 2/3 dependency released, 4/5 K tile landed, 6/7 CTA end
+    [[maybe_unused]] unsigned long long* stp = LLMA_STAMP_PTR(a.stamps, 300 + a.layer, 0);
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
     const int c0 = chunk * kAttnChunk;
@@ -89,6 +92,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
         if (early) fetch_kv();
     }
     pdl_wait();  // row descriptors, q and the K/V rows of this step come from the kernels before
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 2);
 
     // rows of this sequence in the step (contiguous; summarised by the planning kernel)
     const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
@@ -132,6 +136,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     }
     __syncthreads();
     if (flag[0]) return;  // the copy never landed: give up (error word is set)
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 4);
 
     const float scale = rsqrtf((float)HD);
     const int n_mt = (cnt + 15) >> 4;
@@ -311,6 +316,7 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
         }
         __syncthreads();
     }
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 6);
 }
 
 // Second pass: one warp per (head, row) combines the row's chunk partials in ascending chunk
@@ -319,24 +325,47 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
 template <int HD>
 __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) {
     pdl_trigger();
+    // timeline (min, max over the warps): 2/3 dependency released, 6/7 warp end
+    [[maybe_unused]] unsigned long long* stp = LLMA_STAMP_PTR(a.stamps, 400 + a.layer, 0);
     pdl_wait();
+    if ((threadIdx.x & 31) == 0) LLMA_STAMP_MINMAX(stp, 2);
     extern __shared__ float s_w[];  // [4 warps][n_chunks] weights, then [4][n_chunks] weighted sums
     const int head = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const ModelDims& d = a.dims;
-    const int r = blockIdx.y * 4 + warp;  // row slot of the step
-    if (r >= __ldcg(&a.rows->rows_used)) return;
-    const int pos = __ldcg(&a.rows->pos[r]);
-    if (pos < 0) return;
-    const int nc = pos / kAttnChunk + 1;
+    const int r = blockIdx.y * 4 + warp;  // row slot of the step (below the pass's row slots: they come in fours)
     const int64_t head_base = (int64_t)head * a.n_chunks * d.row_cap;
     float* w_c = s_w + warp * a.n_chunks;
     float* wl_c = s_w + (4 + warp) * a.n_chunks;
+    // The kernel is a chain of dependent loads, so everything whose address is known is requested at once:
+    // the row's position, the (max, sum) pairs of every chunk slot and the first sixteen chunk partials.
+    // Slots past the row's last chunk hold older (finite) values; they are read but never used.
+    const int rows_used = __ldcg(&a.rows->rows_used);
+    const int pos = __ldcg(&a.rows->pos[r]);
+    const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + (lane < HD / 4 ? lane : 0);
+    float2 ml[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int c = lane + 32 * u;
+        ml[u] = c < a.n_chunks ? __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * d.row_cap + r)
+                               : make_float2(-INFINITY, 0.f);
+    }
+    float4 p0[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u)
+        p0[u] = u < a.n_chunks ? __ldcg(src + (int64_t)u * d.row_cap * (HD / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r >= rows_used || pos < 0) return;
+    const int nc = pos / kAttnChunk + 1;
     float M = -INFINITY;
-    for (int c = lane; c < nc; c += 32) {
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * d.row_cap + r);
-        w_c[c] = ml.x; wl_c[c] = ml.y;
-        M = fmaxf(M, ml.x);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int c = lane + 32 * u;
+        if (c < nc) { w_c[c] = ml[u].x; wl_c[c] = ml[u].y; M = fmaxf(M, ml[u].x); }
+    }
+    for (int c = lane + 64; c < nc; c += 32) {  // contexts beyond 64 chunks
+        const float2 m2 = __ldcg(reinterpret_cast<const float2*>(a.ws_ml) + head_base + (int64_t)c * d.row_cap + r);
+        w_c[c] = m2.x; wl_c[c] = m2.y;
+        M = fmaxf(M, m2.x);
     }
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     __syncwarp();
@@ -350,8 +379,14 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
     for (int c = 0; c < nc; ++c) den += wl_c[c];  // ascending order, the same in every lane
     if (lane < HD / 4) {
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + lane;
-        for (int c = 0; c < nc; c += 16) {  // sixteen partials requested together
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            if (u < nc) {
+                const float f = w_c[u];
+                num.x += f * p0[u].x; num.y += f * p0[u].y; num.z += f * p0[u].z; num.w += f * p0[u].w;
+            }
+        }
+        for (int c = 16; c < nc; c += 16) {  // sixteen partials requested together
             float4 p[16];
 #pragma unroll
             for (int u = 0; u < 16; ++u)
@@ -370,6 +405,7 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
         store_act(a.attn_out, kActSplit, d.row_cap, r, col + 2, d.hd_total, num.z / den);
         store_act(a.attn_out, kActSplit, d.row_cap, r, col + 3, d.hd_total, num.w / den);
     }
+    if (lane == 0) LLMA_STAMP_MINMAX(stp, 6);
 }
 
 constexpr size_t kAttnPad = 0;  // extra shared memory per CTA (a knob for the number of CTAs per SM)

@@ -20,6 +20,7 @@ struct AttnArgs {
     void* attn_out;          // ActLayout kActSplit [2 rc][H*hd]
     float* ws_o;             // chunk partials [head][chunk][rc][hd] fp32
     float* ws_ml;            // [head][chunk][rc][2] = (max, sum)
+    unsigned long long* stamps;  // measurement builds: timeline block (see LLMA_STAMPS), else unused
     int32_t* dev_err;
 };
 

@@ -42,6 +42,21 @@ struct RowDesc {
     int32_t max_pos;       // highest position among used rows (-1 if none)
 };
 
+// In-kernel timeline (measurement builds only: compile with -DLLMA_STAMPS).  Every stamped kernel gets a
+// block of kStampSlots x 8 words per launch: the projections write one slot per CTA (word i = time of event
+// i), the attention kernels keep (min, max) pairs over their CTAs in slot 0.  Without the flag the macros
+// expand to nothing and the kernels carry no trace of them.
+constexpr int kStampLaunches = 512, kStampSlots = 160;
+#ifdef LLMA_STAMPS
+#define LLMA_STAMP_PTR(base, launch, slot) ((base) ? (base) + ((size_t)(launch) * llma::kStampSlots + (slot)) * 8 : nullptr)
+#define LLMA_STAMP(ptr, i) do { if (ptr) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); (ptr)[i] = _t; } } while (0)
+#define LLMA_STAMP_MINMAX(ptr, i) do { if (ptr) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); atomicMin(&(ptr)[i], _t); atomicMax(&(ptr)[(i) + 1], _t); } } while (0)
+#else
+#define LLMA_STAMP_PTR(base, launch, slot) nullptr
+#define LLMA_STAMP(ptr, i) do { } while (0)
+#define LLMA_STAMP_MINMAX(ptr, i) do { } while (0)
+#endif
+
 enum : int32_t {
     kDevErrNone = 0,
     kDevErrTimeout = 1,   // a bounded wait ran out

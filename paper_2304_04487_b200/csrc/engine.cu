@@ -51,7 +51,7 @@ static void free_engine(llma_engine* e) {
     cudaFree(e->gate_up); cudaFree(e->logits); cudaFree(e->x_hat); cudaFree(e->attn); cudaFree(e->h);
     cudaFree(e->rope_cos); cudaFree(e->rope_sin); cudaFree(e->kcache); cudaFree(e->vcache);
     cudaFree(e->attn_ws_o); cudaFree(e->attn_ws_ml); cudaFree(e->trace); cudaFree(e->target);
-    cudaFree(e->gemm_ws); cudaFree(e->gemm_ws_wide); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss);
+    cudaFree(e->gemm_ws); cudaFree(e->stamps); cudaFree(e->gemm_ws_wide); cudaFree(e->part_max); cudaFree(e->part_idx); cudaFree(e->norm_ss);
     if (e->h_state) cudaFreeHost(e->h_state);
     if (e->h_rows) cudaFreeHost(e->h_rows);
     if (e->h_err) cudaFreeHost(e->h_err);
@@ -183,6 +183,9 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         CREATE_TRY(dalloc(&e->part_max, (size_t)vt * RC));
         CREATE_TRY(dalloc(&e->part_idx, (size_t)vt * RC));
         CREATE_TRY(dalloc(&e->norm_ss, (size_t)((d.d_model + 127) / 128) * RC));
+#ifdef LLMA_STAMPS
+        CREATE_TRY(dalloc(&e->stamps, (size_t)kStampLaunches * kStampSlots * 8));
+#endif
         e->maps.resize(L);
         e->maps2.resize(L);
         e->gate_up_map.resize(L);

@@ -54,6 +54,8 @@ struct llma_engine {
     int cur_nr = 32, cur_rows = 32;
     const ActMaps* cur_maps = nullptr;
     int num_sms = 0;
+    unsigned long long* stamps = nullptr;  // timeline blocks (allocated in measurement builds only)
+    int stamp_id = 0;                      // projections enqueued since the step began
     float* gemm_ws = nullptr;       // partial tiles of gemm_ws_kernel [num_sms][2][8][128] float4
     float* gemm_ws_wide = nullptr;  // partial tiles of gemm_wide_kernel [num_sms][2][wide_nr / 4][128] float4
     size_t gemm_ws_bytes = 0, gemm_ws_wide_bytes = 0;

@@ -112,6 +112,21 @@ extern "C" int llma_kv_len(llma_engine* e, int32_t seq) {
     return e->h_state[seq].kv_len;
 }
 
+extern "C" int llma_debug_timeline(llma_engine* e, int32_t clear, unsigned long long* out) {
+    if (!e) return LLMA_ERR_NULL;
+    if (!e->stamps) return LLMA_ERR_STATE;  // not a measurement build
+    const size_t n = (size_t)kStampLaunches * kStampSlots * 8;
+    CU_TRY(cudaStreamSynchronize(e->stream));
+    if (out) CU_TRY(cudaMemcpy(out, e->stamps, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    if (clear) {  // even words of the (min, max) blocks start at all-ones, everything else at zero
+        std::vector<unsigned long long> h(n, 0ull);
+        for (int l = 300; l < kStampLaunches; ++l)
+            for (int j = 0; j < 8; j += 2) h[(size_t)l * kStampSlots * 8 + j] = ~0ull;
+        CU_TRY(cudaMemcpy(e->stamps, h.data(), n * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    }
+    return LLMA_OK;
+}
+
 extern "C" int llma_row_capacity(llma_engine* e) {
     if (!e) return LLMA_ERR_NULL;
     return e->row_cap;

@@ -31,6 +31,7 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
     a.mode = mode; a.n_out = n_out; a.n_tiles = n_tiles; a.chunks = k_in / 64; a.tiles_per_map = tiles_per_map;
     a.rows = e->rows; a.dev_err = e->dev_err;
     a.rc = e->row_cap; a.nr = e->cur_nr;
+    a.stamps = e->cur_wide ? nullptr : e->stamps; a.launch_id = (e->stamp_id++) % kStampLaunches;
     a.ws = e->cur_wide ? e->gemm_ws_wide : e->gemm_ws;
     a.dims = e->dims;
     return a;
@@ -71,6 +72,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         at.n_rows = e->cur_rows;
         at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml;
         at.dev_err = e->dev_err;
+        at.stamps = e->cur_wide ? nullptr : e->stamps;
         at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0;  // prompt passes: the device-side length is stale
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
@@ -195,6 +197,7 @@ static void enqueue_tail(llma_engine* e, int n, int k, bool accept, bool plan) {
 // llma_generate's graph) the plan of the next step in the same launch.
 static void enqueue_step_body(llma_engine* e, int n, int k, bool plan_next) {
     shape_for_decode(e);
+    e->stamp_id = 0;
     enqueue_embed(e);
     mark(e, LLMA_K_EMBED);
     e->launch_counter += 1;

@@ -67,6 +67,9 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     const int64_t w_beg = cta_begin(work, b, G), w_end = cta_begin(work, b + 1, G);
 
     grid_launch_dependents();  // the next kernel may begin its own prologue now
+    // timeline events: 0 CTA start, 1 dependency released, 2 first stage ready, 3 last MMA issued, 4 last accumulator ready, 5 CTA end
+    [[maybe_unused]] unsigned long long* stp = LLMA_STAMP_PTR(g.stamps, g.launch_id, blockIdx.x);
+    if (threadIdx.x == 0) LLMA_STAMP(stp, 0);
     if (threadIdx.x == 0) {
         // a stage is full once its weight tile has landed (producer's expect_tx) and the loader warps of its
         // KC activation tiles have arrived
@@ -138,6 +141,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     const int s = (int)(it % S);
                     const uint32_t ph = (uint32_t)((it / S) & 1);
                     if (!mbar_wait(full_bar(s), ph)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    if (it == 0) LLMA_STAMP(stp, 2);
                     tc_fence_after();
 #pragma unroll
                     for (int h = 0; h < KC; ++h) {  // the stage's k-chunks: a weight tile and an activation tile each
@@ -151,6 +155,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 }
                 if (sh[1]) break;
                 umma_commit(accf_bar(buf));  // accumulator complete
+                LLMA_STAMP(stp, 3);
                 w += c1 - c0;
             }
         }
@@ -212,6 +217,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
+        if (threadIdx.x == 0) LLMA_STAMP(stp, 1);
         const int rows_used = g.rows ? min(g.rows->rows_used, NR) : NR;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
         if (g.ss_in && row < NR) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
@@ -300,6 +306,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             const bool ok = sh[2] != 0;
             epi_sync();
             if (!ok) { aborted = true; break; }
+            if (threadIdx.x == 0) LLMA_STAMP(stp, 4);
             tc_fence_after();
             float acc[32];
             {
@@ -384,6 +391,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             finish_tile(tile, acc, xpre);
         }
         (void)aborted;
+        if (threadIdx.x == 0) LLMA_STAMP(stp, 5);
     }
     tc_fence_before();
     __syncthreads();

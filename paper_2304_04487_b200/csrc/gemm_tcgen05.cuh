@@ -41,6 +41,8 @@ struct GemmArgs {
     const void* act;        // activation operand, ActLayout kActSplit [2 rc][k_in] bf16
     int32_t rc;             // row capacity of the activation buffers and per-row scratch arrays
     int32_t nr;             // rows the launch is shaped for (wide kernel: multiple of 16, <= 256)
+    unsigned long long* stamps;  // measurement builds: timeline block (see LLMA_STAMPS), else unused
+    int32_t launch_id;           // ... which launch of the step this is
     float* ws;              // partial tiles [grid][2][nr / 4][128] float4; slot 1 of every CTA all-ones (empty) at launch
     int32_t* dev_err;
     float* out_f32;         // Resid: x; QKV: qkv buffer; LmHead: logits or nullptr
