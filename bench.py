@@ -210,9 +210,10 @@ def run_reference(args, rank):
 # Further workloads.  Each prints one JSON line with the same keys as the default workload; `value` is
 # the workload's own headline figure, the details sit under a key named after the workload.
 # ---------------------------------------------------------------------------------------------------
-def _launches_per_pass(shape):
-    """Kernels of one decoding step on the tensor-core path: embedding gather, six per layer, LM head, step tail."""
-    return 6 * shape.n_layers + 3
+def _launches_per_pass(stats, forward_passes):
+    """Kernels of one decoding step, from a run whose number of forward passes is known (a greedy decode of N tokens
+    takes N passes; the call's first launch is the stand-alone plan)."""
+    return (int(stats.launches) - 1) // forward_passes
 
 
 def _common_line(args, world, shape, value, unit, ms_per_step, config, launches):
@@ -236,6 +237,7 @@ def run_serve16(args, rank, local_rank, world, small=False):
         eng.llma_prefill(s, make_prompt(hist, shape.vocab, seed=100 + s))
     t_pre = time.perf_counter() - t0
     y_star, g0 = eng.llma_generate(N, 1, 0)
+    per_pass = _launches_per_pass(g0, N)
     frng = np.random.Generator(np.random.Philox(key=[5, 0]))
     fs = frng.uniform(0.7, 0.9, size=B)
     refs = [build_reference(y_star[s], [R], float(fs[s]), shape.vocab, seed=s) for s in range(B)]
@@ -257,14 +259,14 @@ def run_serve16(args, rank, local_rank, world, small=False):
     for _ in range(args.steps):
         toks, st = one(k)
         dev_ms += st.device_ms; launches += st.launches
-        passes += (st.launches - 1) // _launches_per_pass(shape)
+        passes += (st.launches - 1) // per_pass
         trig += st.trigger_steps; acc += st.copied_accepted
     torch.cuda.synchronize()
     wall_s = time.perf_counter() - wall0
     g_ms, g_passes = 0.0, 0
     for _ in range(args.steps):
         _, st = one(0)
-        g_ms += st.device_ms; g_passes += (st.launches - 1) // _launches_per_pass(shape)
+        g_ms += st.device_ms; g_passes += (st.launches - 1) // per_pass
     clocks = sampler.stop()
     dev_ms, wall_s, g_ms = max_over_ranks([dev_ms, wall_s, g_ms], device="cuda")
     peak, peak_kind = load_peaks()
