@@ -193,26 +193,26 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         int bad = 0;
         for (int l = 0; l < L; ++l) {
             llma_engine::LayerMaps& m = e->maps[l];
-            // wide kernel: 256-row boxes (two tiles per copy); gate and up: 128 rows of each
-            bad |= make_tensor_map_bf16(&m.wq, e->wq[l], HD, d.d_model, 256);
-            bad |= make_tensor_map_bf16(&m.wk, e->wk[l], HD, d.d_model, 256);
-            bad |= make_tensor_map_bf16(&m.wv, e->wv[l], HD, d.d_model, 256);
-            bad |= make_tensor_map_bf16(&m.wo, e->wo[l], d.d_model, HD, 256);
-            bad |= make_tensor_map_bf16(&m.w_gate, e->w_gate[l], d.d_ffn, d.d_model, 128);
-            bad |= make_tensor_map_bf16(&m.w_up, e->w_up[l], d.d_ffn, d.d_model, 128);
-            bad |= make_tensor_map_bf16(&m.w_down, e->w_down[l], d.d_model, d.d_ffn, 256);
+            bad |= make_tensor_map_bf16(&m.wq, e->wq[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wk, e->wk[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wv, e->wv[l], HD, d.d_model, 128);
+            bad |= make_tensor_map_bf16(&m.wo, e->wo[l], d.d_model, HD, 128);
+            bad |= make_tensor_map_bf16(&m.w_gate, e->w_gate[l], d.d_ffn, d.d_model, 64);
+            bad |= make_tensor_map_bf16(&m.w_up, e->w_up[l], d.d_ffn, d.d_model, 64);
+            bad |= make_tensor_map_bf16(&m.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
             llma_engine::LayerMaps& m2 = e->maps2[l];
             bad |= make_tensor_map_bf16_chunks(&m2.wq, e->wq[l], HD, d.d_model, 128);
             bad |= make_tensor_map_bf16_chunks(&m2.wk, e->wk[l], HD, d.d_model, 128);
             bad |= make_tensor_map_bf16_chunks(&m2.wv, e->wv[l], HD, d.d_model, 128);
             bad |= make_tensor_map_bf16_chunks(&m2.wo, e->wo[l], d.d_model, HD, 128);
             bad |= make_tensor_map_bf16_chunks(&m2.w_down, e->w_down[l], d.d_model, d.d_ffn, 128);
+            m2.w_gate = m.w_gate; m2.w_up = m.w_up;
             // one view over both matrices; if they lie too far apart for one, every pass uses the wide kernel
             if (make_tensor_map_bf16_pair(&e->gate_up_map[l].map, e->w_gate[l], e->w_up[l], d.d_ffn, d.d_model,
                                           &e->gate_up_map[l].gate_second) != 0)
                 pair_ok = false;
         }
-        bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 256);
+        bad |= make_tensor_map_bf16(&e->map_lm_head, e->lm_head, d.vocab, d.d_model, 128);
         bad |= make_tensor_map_bf16_chunks(&e->map_lm_head2, e->lm_head, d.vocab, d.d_model, 128);
         // the MMA shape of decoding steps is fixed per engine (by its row capacity), never per step
         e->decode_wide = e->decode_rows > 32 || !pair_ok;

@@ -80,9 +80,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
         run_gemm(e, o, m.wo, m.wo, m.wo, e->attn, am ? &am->attn : nullptr);
         mark(e, LLMA_K_GEMM_O);
-        // narrow kernel: tiles of 64 gate + 64 up rows; wide kernel: pairs of 128 gate + 128 up rows
-        const int gu_tiles = e->cur_wide ? (F + 127) / 128 : (F + 63) / 64;
-        GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, gu_tiles, D, gu_tiles);
+        GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         with_norm(e, gu);
         gu.out_act = e->h;
         if (e->cur_wide) {

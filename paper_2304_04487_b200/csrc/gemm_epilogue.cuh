@@ -132,19 +132,6 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
     epi_sync();
 }
 
-// SwiGLU on a pair of tiles: gate[f][j] and up[f][j] hold features [128 tile, +128) of the two projections,
-// rows jb .. jb + nj - 1.
-__device__ __forceinline__ void epilogue_swiglu_pair(const GemmArgs& g, int tile, int row, int jb, int nj,
-                                                     float (*gate)[33], float (*up)[33]) {
-    const int f = tile * 128 + row;
-    if (f >= g.n_out) return;
-#pragma unroll 1
-    for (int j = 0; j < nj; ++j) {
-        const float gv = gate[row][j], uv = up[row][j];
-        store_act(g.out_act, kActSplit, g.rc, jb + j, f, g.n_out, gv / (1.f + expf(-gv)) * uv);
-    }
-}
-
 // LM head: optional logits store, then the tile's (max, lowest argmax) for every used row.
 __device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33], float* red_f, int* red_i) {

@@ -100,12 +100,12 @@ template <int NR> struct GemmCfg {
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
 };
 
-// Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight stages (256 rows, 32 KB each) and a ring of
+// Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight tiles (16 KB each) and a ring of
 // activation tiles (nr rows of 128 bytes each: one term of one 64-wide k-chunk), as many as fit.
 struct GemmWideCfg {
     uint32_t b_slot;    // bytes of one activation tile
     int sa, sb;         // ring depths (each at most 8)
-    uint32_t tmem_cols; // power of two >= 4 nr (two sets of two accumulators) or, past 128 rows, >= 2 nr (one set)
+    uint32_t tmem_cols; // power of two >= 2 nr (two accumulators)
     size_t smem_bytes;
 };
 GemmWideCfg gemm_wide_cfg(int nr);

@@ -2,9 +2,7 @@
 // Same contract, work split and fused epilogues as gemm_ws_kernel (see gemm_tcgen05.cuh); what differs:
 //   * the activation tiles are large enough for TMA to pay: a second producer thread streams them
 //     through a ring of their own (one slot = nr rows x 64 columns of ONE bf16 term, hi or lo); both terms
-//     are accumulated into the same TMEM columns;
-//   * a ring stage of weights holds 256 rows (two 128-row tiles, or 128 gate + 128 up rows), multiplied by the same
-//     activation tile into two accumulators: every activation byte fetched from L2 serves twice the weights;
+//     are accumulated into the same TMEM columns, so 256 rows fit two accumulators;
 //   * MMA N = the rows in use rounded up to 16 (a run-time field of the instruction descriptor);
 //   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
 //
@@ -28,7 +26,6 @@ using namespace ptx;
 
 constexpr size_t kWideStageBytes = 128 * 33 * 4;
 constexpr size_t kWideTailBytes = 5120;  // barriers, flags, per-row scales, reduction scratch, row positions and slots
-constexpr uint32_t kWideABytes = 2 * kGemmABytes;  // a stage of weights: 256 rows x one 64-wide k-chunk
 
 template <int MODE>
 __global__ void __launch_bounds__(kGemmWideThreads, 1)
@@ -41,11 +38,10 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const int nr = g.nr;
     constexpr int NT = 2;  // bf16 terms of the activation operand: hi, lo
     const uint32_t b_slot = (uint32_t)nr * 128u;
-    const uint32_t sA = base, sB = base + (uint32_t)SA * kWideABytes;
-    uint8_t* after = gen_base + (size_t)SA * kWideABytes + (size_t)SB * b_slot;
+    const uint32_t sA = base, sB = base + (uint32_t)SA * kGemmABytes;
+    uint8_t* after = gen_base + (size_t)SA * kGemmABytes + (size_t)SB * b_slot;
     float (*stage)[33] = reinterpret_cast<float (*)[33]>(after);
-    float (*stage_g)[33] = stage + 128;  // gate half of a gate/up pair
-    uint8_t* tail = after + 2 * kWideStageBytes;
+    uint8_t* tail = after + kWideStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full_a[8], empty_a[8], full_b[8], empty_b[8], acc_full[2], acc_empty[2]
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + 36 * 8);  // [0] TMEM base, [1] abort, [2] broadcast
     float* rscale = reinterpret_cast<float*>(tail + 36 * 8 + 16);                 // [256] per-row norm scales
@@ -64,20 +60,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, b = blockIdx.x;
     const int C = g.chunks;
-    // A work tile is 256 weight rows: two 128-row tiles of one matrix (QKV: never across two of the three
-    // matrices), or, for gate/up, 128 gate rows and the same 128 up rows (g.n_tiles counts those pairs).
-    const int tpm = g.tiles_per_map;
-    const int spm = MODE == kGemmSwiGLU ? tpm : (tpm + 1) / 2;          // work tiles per matrix
-    const int n_super = MODE == kGemmSwiGLU ? g.n_tiles : (g.n_tiles / tpm) * spm;
-    const int64_t work = (int64_t)n_super * C;
+    const int64_t work = (int64_t)g.n_tiles * C;
     const int64_t w_beg = cta_begin(work, b, G), w_end = cta_begin(work, b + 1, G);
-    const int n_buf = 4 * nr <= 512 ? 2 : 1;  // accumulator sets (of two accumulators of nr columns) that fit TMEM
-    // the 128-row tile that half h of work tile S is (an index the epilogues understand), or -1 if past its matrix
-    auto sub_tile = [&](int S, int h) {
-        if (MODE == kGemmSwiGLU) return S;
-        const int m = S / spm, lt = 2 * (S - m * spm) + h;
-        return lt < tpm ? m * tpm + lt : -1;
-    };
+    const int64_t n_items = w_end - w_beg;
 
     grid_launch_dependents();  // the next kernel may begin its own prologue now
     if (threadIdx.x == 0) {
@@ -111,14 +96,14 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 const int s = (int)(it % SA);
                 const uint32_t ph = (uint32_t)((it / SA) & 1);
                 if (it >= SA && !mbar_wait(empty_a(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                mbar_arrive_expect_tx(full_a(s), kWideABytes);
-                const int S = (int)(w / C), c = (int)(w - (int64_t)S * C);
-                const uint32_t dstA = sA + s * kWideABytes;
+                mbar_arrive_expect_tx(full_a(s), kGemmABytes);
+                const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
+                const uint32_t dstA = sA + s * kGemmABytes;
                 if (MODE == kGemmSwiGLU) {
-                    tma_load_2d(dstA, &map_a0, full_a(s), c * 64, S * 128);
-                    tma_load_2d(dstA + kGemmABytes, &map_a1, full_a(s), c * 64, S * 128);
-                } else {  // one copy of 256 rows (rows past the matrix arrive as zeros)
-                    const int m = S / spm, r0 = (S - m * spm) * 256;
+                    tma_load_2d(dstA, &map_a0, full_a(s), c * 64, tile * 64);
+                    tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_a(s), c * 64, tile * 64);
+                } else {
+                    const int m = tile / g.tiles_per_map, r0 = (tile % g.tiles_per_map) * 128;
                     const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
                     tma_load_2d(dstA, mp, full_a(s), c * 64, r0);
                 }
@@ -161,36 +146,32 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             int64_t ia = 0, ib = 0;
             int seg = 0;
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
-                const int S = (int)(w / C), c0 = (int)(w - (int64_t)S * C);
+                const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
                 const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
-                const int buf = seg % n_buf;
-                const uint32_t use = (uint32_t)(seg / n_buf);
+                const int buf = seg & 1;
+                const uint32_t use = (uint32_t)(seg >> 1);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2) * (uint32_t)nr;  // the set's two accumulators
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)nr;
                 for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
                     const int s = (int)(ia % SA);
                     if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
                     for (int t = 0; t < NT; ++t, ++ib) {
                         const int sb = (int)(ib % SB);
                         if (!mbar_wait(full_b(sb), (uint32_t)((ib / SB) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                         tc_fence_after();
                         const uint64_t db = smem_desc_sw128(sB + (uint32_t)sb * b_slot);
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {  // the two 128-row halves of the weight stage share the activation tile
-                            const uint64_t da = smem_desc_sw128(sA + s * kWideABytes + h * kGemmABytes);
-#pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-                                umma_bf16(d_tmem + (uint32_t)h * (uint32_t)nr, da + 2 * kk, db + 2 * kk, idesc,
-                                          (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
-                        }
+                        for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
                         umma_commit(empty_b(sb));  // slot is free once these MMAs have read it
                     }
                     if (sh[1]) break;
                     umma_commit(empty_a(s));
                 }
                 if (sh[1]) break;
-                umma_commit(accf_bar(buf));  // accumulators complete
+                umma_commit(accf_bar(buf));  // accumulator complete
                 w += c1 - c0;
             }
         }
@@ -223,41 +204,40 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         }
         epi_sync();
         const float xnone[kXPre] = {};
-        // a 32-row block of one accumulator goes to shared memory (scaled by the folded RMSNorm)
-        auto stage_block = [&](float (*dst)[33], int jb, const float (&acc)[32]) {
+        // stage a 32-row block in shared memory (scaled by the folded RMSNorm), then the fused epilogue
+        auto finish_block = [&](int tile, int rb, float (&acc)[32]) {
+            const int jb = rb * 32, nj = min(32, rows_used - jb);
             if (g.ss_in) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) dst[row][j] = acc[j] * rscale[min(jb + j, kRowCap - 1)];
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[min(jb + j, kRowCap - 1)];
             } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) dst[row][j] = acc[j];
+                for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
             }
-        };
-        // the fused epilogue of a staged block (gate/up: of the pair of staged blocks)
-        auto run_block = [&](int tile, int rb) {
-            const int jb = rb * 32, nj = min(32, rows_used - jb);
             epi_sync();
             if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, jb, nj, stage, s_pos, s_seq, nullptr);
             else if constexpr (MODE == kGemmResid) epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
-            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu_pair(g, tile, row, jb, nj, stage_g, stage);
+            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, jb, nj, stage);
             else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, jb, nj, stage);
             else epilogue_lmhead(g, tile, row, jb, nj, stage, red_f, red_i);
             epi_sync();  // the staging area is rewritten by the next block
         };
-        // Tiles cut by a range boundary (see gemm_ws_kernel): the CTA that holds a work tile's FIRST chunks owns
-        // it and completes it at the end of its range; every other CTA of the tile hands its two partial
-        // accumulators over through its slot pair of the workspace (all-ones words while empty).  The slots are
-        // laid out for the engine's row capacity whatever nr is, so that prompt passes and decoding steps agree on them.
+        // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks its own
+        // partial in slot 0 of its workspace and completes the tile after its last segment; every other CTA of the tile
+        // hands its partial over through slot 1 (all-ones words while empty, see gemm_ws_kernel).
         constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+        // slots are laid out for the engine's row capacity whatever nr is: a prompt pass and a decoding step (different nr)
+        // then agree on where every CTA's slots are, and the never-emptied slot 0 of one cannot sit in a slot 1 of the other
         const int qn = g.rc >> 2;
+        int own_tile = -1, own_first = 0;
         bool aborted = false;
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
-            const int S = (int)(w / C), c0 = (int)(w - (int64_t)S * C);
+            const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
             const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
             w += c1 - c0;
-            const int buf = seg % n_buf;
-            const uint32_t use = (uint32_t)(seg / n_buf);
+            const int buf = seg & 1;
+            const uint32_t use = (uint32_t)(seg >> 1);
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
                 if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
@@ -268,75 +248,84 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             epi_sync();
             if (!ok) { aborted = true; break; }
             tc_fence_after();
-            const int64_t t_lo = (int64_t)S * C, t_hi = t_lo + C;
-            const bool hand_over = w_beg > t_lo;            // another CTA holds the tile's first chunks
-            const bool owner = !hand_over && w_end < t_hi;  // this one does, and others hold the rest
-            int b_last = b;
-            if (owner) {
-                b_last = (int)((t_hi - 1) * G / work);
-                while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
-                while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
-            }
-            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
-            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 2) * (uint32_t)nr;
+            const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
+            const bool shared_tile = w_beg > t_lo || w_end < t_hi;
+            const bool owner = w_end >= t_hi;
+            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)nr;
             for (int rb = 0; rb < nblk; ++rb) {
-                const int jb = rb * 32;
+                float acc[32];
+                tmem_ld_32cols(t0 + (uint32_t)rb * 32u, acc);
+                if (shared_tile) {
+                    float4* dst = ws_slot(g.ws, qn, b, owner ? 0 : 1, row) + (int64_t)rb * 8 * 128;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int tile = sub_tile(S, h);
-                    if (tile < 0) continue;  // past the matrix (uniform over the CTA)
-                    float acc[32];
-                    tmem_ld_32cols(t0 + (uint32_t)h * (uint32_t)nr + (uint32_t)rb * 32u, acc);
-                    if (hand_over) {
-                        float4* dst = ws_slot(g.ws, qn, b, h, row) + (int64_t)rb * 8 * 128;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q)  // only the columns of rows in use travel
-                            if (jb + 4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-                        continue;
-                    }
-                    for (int bb = b + 1; bb <= b_last; ++bb) {  // owner: the later CTAs' partials in ascending k
-                        float4* src = ws_slot(g.ws, qn, bb, h, row) + (int64_t)rb * 8 * 128;
-                        float4 p[8];
-                        bool valid;
-                        do {
-                            valid = true;
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                if (jb + 4 * q < rows_used) {
-                                    valid = valid && __float_as_uint(p[q].x) != kEmpty;
-                                    if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
-                                    if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
-                                    if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
-                                }
-                            }
-                            if (!valid && globaltimer_ns() > give_up) { atomicExch(g.dev_err, kDevErrTimeout); break; }
-                        } while (!valid);
-                        const float e = __uint_as_float(kEmpty);
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            if (jb + 4 * q < rows_used) {
-                                src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
-                                acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
-                            }
-                        }
-                    }
-                    if (MODE == kGemmSwiGLU) {
-                        stage_block(h == 0 ? stage_g : stage, jb, acc);
-                        if (h == 1) run_block(tile, rb);
-                    } else {
-                        stage_block(stage, jb, acc);
-                        run_block(tile, rb);
-                    }
+                    for (int q = 0; q < 8; ++q)  // only the columns of rows in use travel
+                        if (rb * 32 + 4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                } else {
+                    finish_block(tile, rb, acc);
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator set
+            if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
+            if (shared_tile && owner) {
+                int b_first = (int)(t_lo * G / work);
+                while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
+                while (cta_begin(work, b_first, G) > t_lo) --b_first;
+                own_tile = tile; own_first = b_first;
+            }
         }
-        (void)aborted;
+        if (own_tile >= 0 && !aborted) {
+            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
+            bool timed_out = false;
+            for (int rb = 0; rb < nblk; ++rb) {
+                const int jb = rb * 32;
+                float acc[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                for (int bb = own_first; bb < b; ++bb) {  // ascending k: a fixed summation order
+                    const float4* src = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
+                    float4 p[8];
+                    bool valid;
+                    do {
+                        valid = true;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            if (jb + 4 * q < rows_used) {
+                                valid = valid && __float_as_uint(p[q].x) != kEmpty;
+                                if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
+                                if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
+                                if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
+                            }
+                        }
+                        if (!valid && (timed_out || globaltimer_ns() > give_up)) {
+                            atomicExch(g.dev_err, kDevErrTimeout); timed_out = true; break;
+                        }
+                    } while (!valid);
+                    const float e = __uint_as_float(kEmpty);
+                    float4* wr = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (jb + 4 * q < rows_used) {
+                            wr[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
+                            acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
+                        }
+                    }
+                }
+                // this CTA's own partial comes last (it holds the highest k)
+                const float4* mine = ws_slot(g.ws, qn, b, 0, row) + (int64_t)rb * 8 * 128;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (jb + 4 * q < rows_used) {
+                        const float4 o = mine[q * 128];
+                        acc[4 * q] += o.x; acc[4 * q + 1] += o.y; acc[4 * q + 2] += o.z; acc[4 * q + 3] += o.w;
+                    }
+                }
+                finish_block(own_tile, rb, acc);
+            }
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -350,19 +339,16 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
 GemmWideCfg gemm_wide_cfg(int nr) {
     GemmWideCfg c;
     c.b_slot = (uint32_t)nr * 128u;
-    const size_t budget = (size_t)227 * 1024 - 1024 - 2 * kWideStageBytes - kWideTailBytes;
-    // three weight stages first, then as many activation tiles as fit (at least three), then more weight stages
-    c.sa = 3;
-    c.sb = (int)((budget - (size_t)c.sa * kWideABytes) / c.b_slot);
-    if (c.sb < 3) { c.sa = 2; c.sb = (int)((budget - (size_t)c.sa * kWideABytes) / c.b_slot); }
+    const size_t budget = (size_t)227 * 1024 - 1024 - kWideStageBytes - kWideTailBytes;
+    // four weight tiles in flight first, then as many activation tiles as fit, then more weight tiles
+    c.sb = (int)((budget - 4 * kGemmABytes) / c.b_slot);
     if (c.sb > 8) c.sb = 8;
-    c.sa = (int)((budget - (size_t)c.sb * c.b_slot) / kWideABytes);
-    if (c.sa > 6) c.sa = 6;
+    c.sa = (int)((budget - (size_t)c.sb * c.b_slot) / kGemmABytes);
+    if (c.sa > 8) c.sa = 8;
     uint32_t cols = 32;
-    const uint32_t need = 4u * (uint32_t)nr <= 512u ? 4u * (uint32_t)nr : 2u * (uint32_t)nr;  // two sets of two accumulators, or one
-    while (cols < need) cols <<= 1;
+    while (cols < 2u * (uint32_t)nr) cols <<= 1;
     c.tmem_cols = cols;
-    c.smem_bytes = 1024 + (size_t)c.sa * kWideABytes + (size_t)c.sb * c.b_slot + 2 * kWideStageBytes + kWideTailBytes;
+    c.smem_bytes = 1024 + (size_t)c.sa * kGemmABytes + (size_t)c.sb * c.b_slot + kWideStageBytes + kWideTailBytes;
     if (c.smem_bytes < 120 * 1024) c.smem_bytes = 120 * 1024;  // one CTA per SM, as for the narrow kernel
     return c;
 }
