@@ -31,7 +31,7 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
     a.mode = mode; a.n_out = n_out; a.n_tiles = n_tiles; a.chunks = k_in / 64; a.tiles_per_map = tiles_per_map;
     a.rows = e->rows; a.dev_err = e->dev_err;
     a.rc = e->row_cap; a.nr = e->cur_nr;
-    a.stamps = e->cur_wide ? nullptr : e->stamps; a.launch_id = (e->stamp_id++) % kStampLaunches;
+    a.stamps = e->stamps; a.launch_id = (e->stamp_id++) % kStampLaunches;
     a.ws = e->cur_wide ? e->gemm_ws_wide : e->gemm_ws;
     a.dims = e->dims;
     return a;

@@ -65,6 +65,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const int64_t n_items = w_end - w_beg;
 
     grid_launch_dependents();  // the next kernel may begin its own prologue now
+    [[maybe_unused]] unsigned long long* stp = LLMA_STAMP_PTR(g.stamps, g.launch_id, blockIdx.x);
+    if (threadIdx.x == 0) LLMA_STAMP(stp, 0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
             mbar_init(full_a(s), 1); mbar_init(empty_a(s), 1); mbar_init(full_b(s), 1); mbar_init(empty_b(s), 1);
@@ -88,11 +90,16 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     tc_fence_after();
     const uint32_t tmem_base = sh[0];
 
+    // One thread gets a TMA copy under way about every 0.5 us, whatever the copy's size (measured: 16 KB boxes from one
+    // thread stream 31 GB/s per CTA, from two threads 59, from four 95, L2-resident).  A work item needs three copies
+    // (a weight tile and the two terms of the activation tile), so the copies are dealt over several issuing threads.
+    constexpr int kPA = 2, kPB = 4;  // issuing lanes of the weight producer warp / of the activation producer warp
     if (warp == 4) {
-        // ------------------------------- weight producer -----------------------------------------
-        if (lane == 0) {
-            int64_t it = 0;
-            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w, ++it) {
+        // ------------------------------- weight producers (lane p takes items p, p + kPA, ...) -----------------
+        if (lane < kPA) {
+            int64_t it = lane;
+            for (; it < n_items && !sh[1]; it += kPA) {
+                const int64_t w = w_beg + it;
                 const int s = (int)(it % SA);
                 const uint32_t ph = (uint32_t)((it / SA) & 1);
                 if (it >= SA && !mbar_wait(empty_a(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
@@ -108,31 +115,29 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                     tma_load_2d(dstA, mp, full_a(s), c * 64, r0);
                 }
             }
-            if (sh[1]) {  // give up: let the copies already issued land before the CTA's memory goes away
-                const int64_t first = it > SA ? it - SA : 0;
-                for (int64_t j = first; j < it; ++j)
+            if (sh[1]) {  // give up: let this lane's copies already issued land before the CTA's memory goes away
+                for (int64_t j = it - kPA; j >= 0 && j > it - kPA * (SA + 1); j -= kPA)
                     (void)mbar_wait(full_a((int)(j % SA)), (uint32_t)((j / SA) & 1), 100000000ull);
             }
         }
     } else if (warp == 6) {
-        // ------------------------------- activation producer ---------------------------------------
-        if (lane == 0) {
+        // ------------------------------- activation producers (lane p takes (item, term) pairs p, p + kPB, ...) --
+        if (lane < kPB) {
             grid_dependency_wait();  // activations are written by the kernel before this one
-            int64_t it = 0;          // counts (item, term) pairs
-            for (int64_t w = w_beg; w < w_end && !sh[1]; ++w) {
+            const int64_t n_pairs = n_items * NT;
+            int64_t q = lane;
+            for (; q < n_pairs && !sh[1]; q += kPB) {
+                const int64_t w = w_beg + q / NT;
+                const int t = (int)(q % NT);
                 const int c = (int)(w % C);
-                for (int t = 0; t < NT; ++t, ++it) {
-                    const int s = (int)(it % SB);
-                    const uint32_t ph = (uint32_t)((it / SB) & 1);
-                    if (it >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                    mbar_arrive_expect_tx(full_b(s), b_slot);
-                    tma_load_2d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, t * g.rc);
-                }
-                if (sh[1]) break;
+                const int s = (int)(q % SB);
+                const uint32_t ph = (uint32_t)((q / SB) & 1);
+                if (q >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                mbar_arrive_expect_tx(full_b(s), b_slot);
+                tma_load_2d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, t * g.rc);
             }
             if (sh[1]) {
-                const int64_t first = it > SB ? it - SB : 0;
-                for (int64_t j = first; j < it; ++j)
+                for (int64_t j = q - kPB; j >= 0 && j > q - kPB * (SB + 1); j -= kPB)
                     (void)mbar_wait(full_b((int)(j % SB)), (uint32_t)((j / SB) & 1), 100000000ull);
             }
         }
@@ -156,6 +161,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
                     const int s = (int)(ia % SA);
                     if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    if (ia == 0) LLMA_STAMP(stp, 2);
                     const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
                     for (int t = 0; t < NT; ++t, ++ib) {
                         const int sb = (int)(ib % SB);
@@ -172,12 +178,14 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 }
                 if (sh[1]) break;
                 umma_commit(accf_bar(buf));  // accumulator complete
+                LLMA_STAMP(stp, 3);
                 w += c1 - c0;
             }
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
+        if (threadIdx.x == 0) LLMA_STAMP(stp, 1);
         const int rows_used = g.rows ? min(g.rows->rows_used, nr) : nr;
         const int nblk = (rows_used + 31) >> 5;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
@@ -247,6 +255,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             const bool ok = sh[2] != 0;
             epi_sync();
             if (!ok) { aborted = true; break; }
+            if (threadIdx.x == 0) LLMA_STAMP(stp, 4);
             tc_fence_after();
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
             const bool shared_tile = w_beg > t_lo || w_end < t_hi;
@@ -327,6 +336,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             }
         }
     }
+    if (threadIdx.x == 0) LLMA_STAMP(stp, 5);
     tc_fence_before();
     __syncthreads();
     if (warp == 5) {

@@ -136,22 +136,28 @@ __global__ void __launch_bounds__(kTailThreads) step_tail_kernel(const TailArgs 
         // ---- trigger search: every thread takes reference positions of every live sequence ---------------------
         // key = (ext << 32) | (0x7fffffff - pos): the maximum is the longest agreement, then the earliest position
         if (a.k > 0 && a.n >= 1) {
-            for (int s = 0; s < B; ++s) {
+            // the 32 warps are dealt over the sequences (all of them on one sequence at batch 1, two per sequence at
+            // batch 16, one warp for several sequences beyond 32), so that every sequence's loads are in flight at once
+            const int per_seq = B >= n_warps ? 1 : n_warps / B;      // warps that share a sequence
+            const int groups = n_warps / per_seq;                    // sequences scanned at a time
+            const int sub = warp % per_seq;
+            for (int s = warp / per_seq; s < B; s += groups) {
                 const SeqState& S = s_st[s];
                 const int ylen = S.y_len, ref_len = S.ref_len;
                 const bool live = S.active && !S.done && ylen < S.target_len;
-                if (!live || S.forced_rows != 0 || ylen < a.n || ref_len <= 0) continue;   // uniform over the CTA
+                if (!live || S.forced_rows != 0 || ylen < a.n || ref_len <= 0) continue;   // uniform over the warp
                 const int* ys = a.y + (int64_t)s * a.y_cap;
                 const int* rs = a.ref + (int64_t)s * dims.max_ref;
                 const int* ds = a.doc_start + (int64_t)s * dims.max_ref;
                 const int* de = a.doc_end + (int64_t)s * dims.max_ref;
                 const int last = S.pending;  // the newest generated token (ylen >= 1 here)
-                for (int p0 = 1 + threadIdx.x; p0 < ref_len; p0 += 2 * kTailThreads) {
+                const int stride = 32 * per_seq;
+                for (int p0 = 1 + sub * 32 + lane; p0 < ref_len; p0 += 2 * stride) {
                     // two candidates per round, their loads in flight together
                     int tokv[2], endv[2], begv[2];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int p = p0 + u * kTailThreads;
+                        const int p = p0 + u * stride;
                         const bool in = p < ref_len;
                         tokv[u] = in ? __ldg(&rs[p - 1]) : -1;
                         endv[u] = in ? __ldg(&de[p - 1]) : 0;
@@ -159,7 +165,7 @@ __global__ void __launch_bounds__(kTailThreads) step_tail_kernel(const TailArgs 
                     }
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int p = p0 + u * kTailThreads;
+                        const int p = p0 + u * stride;
                         // candidate: ref[p-1] is the last matched token; p must stay inside its document
                         if (p >= ref_len || tokv[u] != last || p >= endv[u]) continue;
                         int t = 1;
