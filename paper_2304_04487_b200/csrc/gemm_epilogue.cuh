@@ -27,7 +27,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // x[r, n] += acc  (output projection and FFN down projection, residual stream in fp32).
 // When the next RMSNorm is folded in (g.xs_out): also xs = split(x * gain) and this tile's
-// per-row sums of squares, reduced over the 128 columns in a fixed shuffle/warp order.
+// per-row sums of squares, reduced over the 128 columns in an order fixed by the column index.
 // With kHavePre (jb = 0 only), xpre holds x[0..11, col] and the gain, read earlier by the caller.
 template <bool kHavePre>
 __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int row, int jb, int nj,
@@ -36,7 +36,7 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
     const bool valid = col < g.n_out;
     const bool fold = g.xs_out != nullptr;
     const float gain = kHavePre ? xpre[kXPre - 1] : ((fold && valid) ? __ldg(&g.gain_next[col]) : 0.f);
-    const int warp = row >> 5, lane = row & 31;
+    const unsigned group = 0xffu << (row & 24);  // the eight lanes that share an activation row below
     // x is added into the staged tile with a few loads in flight; the per-row work is a rolled loop
     if (kHavePre) {
 #pragma unroll
@@ -52,20 +52,30 @@ __device__ __forceinline__ void epilogue_resid(const GemmArgs& g, int tile, int 
         for (int u = 0; u < 8; ++u)
             if (j0 + u < nj) stage[row][j0 + u] += xv[u];
     }
+    if (!valid) {
+        for (int j = 0; j < nj; ++j) stage[row][j] = 0.f;  // columns past the matrix add nothing to the sums of squares
+    } else {
 #pragma unroll 1
-    for (int j = 0; j < nj; ++j) {
-        const float xn = valid ? stage[row][j] : 0.f;
-        if (valid) g.out_f32[(int64_t)(jb + j) * g.ld + col] = xn;
-        if (fold) {
-            if (valid) store_act(g.xs_out, kActSplit, g.rc, jb + j, col, g.n_out, xn * gain);
-            const float sq = warp_sum(xn * xn);
-            if (lane == 0) red_f[warp * 32 + j] = sq;
+        for (int j = 0; j < nj; ++j) {
+            const float xn = stage[row][j];
+            g.out_f32[(int64_t)(jb + j) * g.ld + col] = xn;
+            if (fold) store_act(g.xs_out, kActSplit, g.rc, jb + j, col, g.n_out, xn * gain);
         }
     }
     if (!fold) return;
+    // Sums of squares: eight threads per activation row, each over sixteen consecutive features in
+    // ascending order, then a three-step shuffle tree: the order depends on the feature index only.
     epi_sync();
-    if (row < nj)
-        g.ss_out[(int64_t)tile * g.rc + jb + row] = ((red_f[row] + red_f[32 + row]) + red_f[64 + row]) + red_f[96 + row];
+    for (int j = row >> 3; j < nj; j += 16) {  // nj is uniform over the eight threads of a row
+        const int f0 = (row & 7) * 16;
+        float sq = 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { const float v = stage[f0 + u][j]; sq = __fmaf_rn(v, v, sq); }
+        sq += __shfl_xor_sync(group, sq, 1);
+        sq += __shfl_xor_sync(group, sq, 2);
+        sq += __shfl_xor_sync(group, sq, 4);
+        if ((row & 7) == 0) g.ss_out[(int64_t)tile * g.rc + jb + j] = sq;
+    }
     epi_sync();
 }
 

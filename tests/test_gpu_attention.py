@@ -43,5 +43,8 @@ def test_attention_rows_match_oracle(name, P, k):
             want = OM.attention(q, K[:L0 + j + 1, h], V[:L0 + j + 1, h])
             got = att[j, h * hd:(h + 1) * hd]
             worst = max(worst, float(np.abs(got - want).max() / max(1e-6, np.abs(want).max())))
-    # fp32 softmax with split bf16 operands: errors near 1e-6 of the row's scale; 2e-5 leaves headroom
-    assert worst < 2e-5, worst
+    # Split bf16 operands carry 2^-18 relative error each (hi = bf16(x), lo = bf16(x - hi)).  Through q that is
+    # 2^-18 * sum|q_i k_i| / sqrt(hd) on a score, i.e. the same relative amount on its softmax weight (sums of
+    # |q_i k_i| / sqrt(hd) reach about 5 with these weights: 1.9e-5); the weights P and the stored output are
+    # split once more each (2 * 3.8e-6).  Bound 2.7e-5 of the row's scale; measured 1e-5 to 2.1e-5.
+    assert worst < 5e-5, worst
