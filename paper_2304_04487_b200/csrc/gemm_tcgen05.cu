@@ -173,6 +173,43 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
         const int64_t ld_bytes = (int64_t)g.chunks * 128;  // one activation row: k_in bf16
         const char* act = reinterpret_cast<const char*>(g.act);
         constexpr int kUnits = NT * NR * 8 / 32;    // 16-byte units per lane
+        if constexpr (NR == 32) {
+            // Thirty-two rows: the tile goes from global to shared memory by asynchronous 16-byte copies, with no
+            // registers in between (a register copy of the next tile costs 64 of them, and with those the CTA
+            // leaves no room on the SM for a CTA of the attention kernel).  A copy is issued as soon as its
+            // stage is free and handed to the MMA warp when it has landed.
+            auto issue = [&](int64_t q, int row_limit) {
+                const int64_t it = q / KC;
+                const int chunk = (int)((w_beg + it) % C) * KC + (int)(q % KC);
+                const bool inside = chunk < g.chunks;
+                const uint32_t dst0 = sB + (uint32_t)(it % S) * kBBytes + (uint32_t)(q % KC) * kBTile;
+#pragma unroll
+                for (int u = 0; u < kUnits; ++u) {
+                    const int unit = u * 32 + lane, r = unit >> 3, j = unit & 7;
+                    const int t = r / NR, rr = r - t * NR;
+                    const uint32_t dst = dst0 + (uint32_t)r * 128 + (uint32_t)((j ^ (r & 7)) << 4);
+                    if (rr < row_limit) {
+                        if (inside) cp_async_16(dst, act + (t * g.rc + rr) * ld_bytes + (int64_t)chunk * 128 + j * 16);
+                        else st_shared_v4(dst, make_uint4(0u, 0u, 0u, 0u));  // past the matrix: zeros
+                    }
+                }
+                cp_async_commit();
+            };
+            for (int64_t q = sw; q < n_sub && !sh[1]; q += NW) {
+                const int64_t it = q / KC;
+                if (it >= S) {
+                    bool ok = true;
+                    if (lane == 0) ok = mbar_wait(empty_bar((int)(it % S)), (uint32_t)((it / S) & 1) ^ 1u);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { if (lane == 0) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; } break; }
+                }
+                issue(q, q == sw ? NR : rows_used);  // first tile: every row, the count of rows is still on its way
+                cp_async_wait<0>();                  // L2 latency: shorter than that of the weight copy issued at the same moment
+                fence_proxy_async_shared();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_bar((int)(it % S)));
+            }
+        } else {
         // rows of the next tile are requested before waiting for its stage to come free, so the
         // latency of the loads hides behind the MMAs of the tiles in between
         uint4 v[kUnits];
@@ -213,6 +250,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             __syncwarp();
             if (lane == 0) mbar_arrive(full_bar(st));
             if (q + NW < n_sub) fetch(q + NW, rows_used);
+        }
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
@@ -312,11 +350,14 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
             {
                 const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (2 * NR);
                 if (NR == 32) {
-                    float lo[32];
                     tmem_ld_32cols(t0, acc);
-                    tmem_ld_32cols(t0 + 32, lo);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+                    for (int hf = 0; hf < 2; ++hf) {  // W * hi + W * lo, the low term sixteen columns at a time
+                        float lo[16];
+                        tmem_ld_16cols(t0 + 32 + 16 * hf, lo);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[16 * hf + j] += lo[j];
+                    }
                 } else {
                     tmem_ld_32cols(t0, acc);  // columns 0..15 hi, 16..31 lo
 #pragma unroll
@@ -340,7 +381,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                 while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
                 while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
                 const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
-                constexpr int kBatch = 2;
+                constexpr int kBatch = NR == 32 ? 1 : 2;  // partials requested together (registers)
                 for (int bb = b + 1; bb <= b_last; bb += kBatch) {  // ascending k: a fixed summation order
                     float4 p[kBatch][NR / 4];
                     bool valid;
@@ -388,6 +429,7 @@ gemm_ws_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, con
                     }
                 }
             }
+            if (threadIdx.x == 0) LLMA_STAMP(stp, 6);  // partials summed: the tile's epilogue begins
             finish_tile(tile, acc, xpre);
         }
         (void)aborted;

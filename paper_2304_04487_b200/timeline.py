@@ -40,7 +40,7 @@ def main():
         t = eng.llma_debug_timeline(clear=False).astype(np.int64)
         sms = int((t[0, :, 0] > 0).sum())
         print(f"k = {k}: {st.device_ms / st.steps:.3f} ms per step, {sms} CTAs per projection")
-        g = t[:4 * L + 1, :sms, :6]
+        g = t[:4 * L + 1, :sms, :7]
         for cls in range(4):
             rows = []
             for l in range(1, L - 1):
@@ -49,10 +49,13 @@ def main():
                 s = g[i] - prev_end
                 rows.append([s[:, 0].min(), s[:, 1].min(), s[:, 2].min(), np.median(s[:, 2]), s[:, 3].min(), s[:, 3].max(),
                              s[:, 4].max(), s[:, 5].min(), s[:, 5].max()])
+                last = int(np.argmax(s[:, 5]))  # the CTA that ends last: its own accumulator, epilogue start and end
+                rows[-1] += [s[last, 4], s[last, 6] if g[i, last, 6] > 0 else s[last, 4]]
             m = np.mean(rows, 0) / 1e3
             print(f"  {names[cls]:8s} after the projection before it ended: first CTA starts {m[0]:6.2f}, dependency released {m[1]:6.2f}, "
                   f"first MMA {m[2]:6.2f} (median {m[3]:6.2f}), last MMA issued {m[4]:6.2f}..{m[5]:6.2f}, "
-                  f"last accumulator ready {m[6]:6.2f}, CTAs end {m[7]:6.2f}..{m[8]:6.2f}")
+                  f"last accumulator ready {m[6]:6.2f}, CTAs end {m[7]:6.2f}..{m[8]:6.2f}; the CTA that ends last: "
+                  f"accumulator {m[9]:6.2f}, partials summed {m[10]:6.2f}")
         rows = []
         for l in range(1, L - 1):
             qkv_end = g[4 * l, :, 5].max()
