@@ -678,6 +678,22 @@ def main():
         eng16.llma_rewind(0)
         _, st = eng16.llma_generate(n_new, 1, kk)
         lat[f"{kk}@32rows"] = {"ms_per_step": st.device_ms / st.steps, "tokens_per_step": st.tokens / st.steps}
+    # the adaptive copy length (a variant beyond the paper) on the workload's own reference: tokens/s of one decode
+    # next to the fixed k of the same engine (16-row engine: k <= 8; 32-row engine: k <= 16)
+    adaptive = {}
+    for tag, e_, kcap, (kmin, kstart) in (("16rows", eng, k, (2, 4)), ("32rows", eng16, 16, (2, 8))):
+        if kcap < kstart:
+            continue
+        e_.llma_set_reference(0, ref, offs)
+        res = {}
+        for name, setting in (("fixed", (0, 0)), ("adaptive", (kmin, kstart))):
+            e_.llma_set_adaptive_k(0, *setting)
+            e_.llma_rewind(0)
+            _, st = e_.llma_generate(n_new, n, kcap)
+            res[name] = {"tokens_per_s": st.tokens / (st.device_ms / 1e3), "steps": int(st.steps),
+                         "ms_per_step": st.device_ms / st.steps}
+        e_.llma_set_adaptive_k(0, 0, 0)
+        adaptive[tag] = {"k_cap": kcap, "k_min": kmin, "k_start": kstart, **res}
     eng16.llma_destroy()
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -690,7 +706,7 @@ def main():
             "greedy_tokens_per_s": greedy_value, "speedup_vs_own_greedy": value / greedy_value,
             "decode_ms_per_llma_step": step_ms, "tokens_per_llma_step": n_new * args.steps / max(steps_taken, 1),
             "llma_steps_per_decode": steps_taken / args.steps, "trigger_steps_per_decode": trig / args.steps,
-            "accepted_per_decode": acc / args.steps, "step_latency_vs_k": lat,
+            "accepted_per_decode": acc / args.steps, "step_latency_vs_k": lat, "adaptive_k": adaptive,
             "prefill_s": t_pre, "weight_gen_s": t_gen,
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(ref.nbytes + offs.nbytes),

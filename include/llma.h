@@ -167,6 +167,19 @@ int llma_generate(llma_engine *e, int32_t max_new, int32_t n, int32_t k, int32_t
  */
 int llma_rewind(llma_engine *e, int32_t seq);
 
+/*
+ * Copy length chosen per step from how the last copy fared (a variant: the paper fixes n and k for a
+ * whole run and sweeps them, Section 3.5; nothing in it adapts k).  While it is on for a sequence, a
+ * step asks for min(k_cur, k) copied tokens instead of k, with k the argument of llma_step /
+ * llma_generate; k_cur starts at k_start and, after every step that copied something, becomes
+ * min(2 k_cur, max_k) if the model agreed with every copied token and max(k_min, ceil(k_cur / 2))
+ * otherwise.  The output stays the greedy output: only the number of rows per step changes.
+ * Call after llma_prefill; llma_rewind keeps the setting and puts k_cur back to k_start,
+ * llma_prefill and llma_reset clear it.  k_min = k_start = 0 switches it off.
+ * Errors: NULL, CAPACITY (seq), ARG (not 1 <= k_min <= k_start <= max_k), CUDA.
+ */
+int llma_set_adaptive_k(llma_engine *e, int32_t seq, int32_t k_min, int32_t k_start);
+
 /* Forget a sequence entirely (slot becomes idle; its reference is cleared). */
 int llma_reset(llma_engine *e, int32_t seq);
 

@@ -21,6 +21,12 @@ Readings of the paper taken here (each is a choice where the text is silent):
     least one token after it.  The copy length actually used is
     k_eff = min(k, tokens left in the document, N - len(y) - 1), so y never
     overshoots N; k_eff = 0 is an ordinary one-token step.
+
+One variant beyond the paper (which fixes n and k for a run and sweeps them, Section 3.5):
+``adaptive=(k_min, k_start, k_cap)`` lets the copy length follow the last copy's fate, see
+``next_copy_request``.  A fall-back from n to a shorter trigger needs no code of its own: with the
+longest-agreement rule above, trying n, n-1, ..., n_lo in turn finds exactly what a trigger of
+length n_lo finds, since the candidate that agrees for longest is the same for both.
 """
 from __future__ import annotations
 
@@ -65,6 +71,17 @@ def copy_length(pos: int, ref_len: int, doc_offsets: Optional[Sequence[int]], k:
         if s <= pos < e:
             return max(0, min(k, e - pos, remaining - 1))
     return 0
+
+
+def next_copy_request(k_cur: int, k_eff: int, accepted: int, k_min: int, k_cap: int) -> int:
+    """Adaptive copy length (variant): the number of tokens to ask for next.  Unchanged by a step
+    that copied nothing; doubled (up to k_cap) after a copy accepted in full; halved, rounding up
+    (down to k_min), after a copy the model cut short."""
+    if k_eff <= 0:
+        return k_cur
+    if accepted == k_eff:
+        return min(2 * k_cur, k_cap)
+    return max(k_min, (k_cur + 1) // 2)
 
 
 @dataclass
@@ -121,16 +138,21 @@ def greedy_decode(model, prompt: Sequence[int], n_new: int, keep_logits: bool = 
 
 
 def llma_decode(model, prompt: Sequence[int], ref: Sequence[int], doc_offsets: Optional[Sequence[int]],
-                n: int, k: int, n_new: int, keep_logits: bool = False) -> DecodeResult:
+                n: int, k: int, n_new: int, keep_logits: bool = False,
+                adaptive: Optional[Tuple[int, int, int]] = None) -> DecodeResult:
     """Algorithm 1.  The k+1 outputs of a copy step (Eq. 3) are computed one position
-    at a time, in order, on the inputs [pending, d_pos, ..., d_pos+k_eff-1]."""
+    at a time, in order, on the inputs [pending, d_pos, ..., d_pos+k_eff-1].
+    ``adaptive=(k_min, k_start, k_cap)``: the variant of ``next_copy_request``; a step then asks
+    for min(k_cur, k) tokens."""
     L, pending = prefill(model, prompt)
     y: List[int] = []
     res = DecodeResult(tokens=y)
     ref = [int(t) for t in ref]
+    k_cur = adaptive[1] if adaptive else 0
     while len(y) < n_new:
         matched, pos, _ = match_ngrams(y, ref, doc_offsets, n)
-        k_eff = copy_length(pos, len(ref), doc_offsets, k, n_new - len(y)) if matched else 0
+        k_ask = min(k_cur, k) if adaptive else k
+        k_eff = copy_length(pos, len(ref), doc_offsets, k_ask, n_new - len(y)) if matched else 0
         inputs = [pending] + ref[pos:pos + k_eff] if k_eff > 0 else [pending]
         outs, rows = [], []
         for j, tok in enumerate(inputs):
@@ -145,6 +167,8 @@ def llma_decode(model, prompt: Sequence[int], ref: Sequence[int], doc_offsets: O
         if keep_logits:
             res.logits.extend(rows[:a + 1])
         res.trace.append(StepRecord(k_eff > 0, pos if k_eff > 0 else -1, k_eff, a, a + 1))
+        if adaptive:
+            k_cur = next_copy_request(k_cur, k_eff, a, adaptive[0], adaptive[2])
         L += a + 1          # rows past L are stale and get overwritten by later steps
         pending = outs[a]
     return res

@@ -55,7 +55,7 @@ class LlmaError(RuntimeError):
 _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
-           "llma_rewind", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
+           "llma_rewind", "llma_set_adaptive_k", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
            "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16",
            "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity", "llma_debug_timeline",
            "llma_last_cuda_error", "llma_strerror")
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
         L.llma_step.argtypes = [vp, i32, i32, pi32, pi32]
         L.llma_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(LlmaStats)]
         L.llma_rewind.argtypes = [vp, i32]
+        L.llma_set_adaptive_k.argtypes = [vp, i32, i32, i32]
         L.llma_reset.argtypes = [vp, i32]
         L.llma_last_step_info.argtypes = [vp, C.POINTER(LlmaStepInfo)]
         L.llma_debug_logits.argtypes = [vp, C.POINTER(C.c_float)]
@@ -226,6 +227,9 @@ class Engine:
 
     def llma_rewind(self, seq: int) -> None:
         self._check(lib().llma_rewind(self._h, seq), "llma_rewind")
+
+    def llma_set_adaptive_k(self, seq: int, k_min: int, k_start: int) -> None:
+        self._check(lib().llma_set_adaptive_k(self._h, seq, k_min, k_start), "llma_set_adaptive_k")
 
     def llma_reset(self, seq: int) -> None:
         self._check(lib().llma_reset(self._h, seq), "llma_reset")

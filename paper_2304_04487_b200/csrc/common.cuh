@@ -23,6 +23,7 @@ struct SeqState {
     int32_t pos, k_eff, nrows;  // plan of the step in flight
     int32_t forced_rows, forced_emit;  // replay of a given step shape (0 = decide as Algorithm 1 does)
     int32_t trace_step;                // replay: index of the next step in the trace
+    int32_t k_min, k_start, k_cur;     // adaptive copy length: k_cur tokens are asked for next (0 = the step's k as given)
     int32_t last_pos, last_k_eff, last_accepted, last_emitted;
     int32_t steps, trigger_steps, copied_accepted;
 };

@@ -29,10 +29,24 @@ extern "C" int llma_rewind(llma_engine* e, int32_t seq) {
     if (!S.active) return LLMA_ERR_STATE;
     const int32_t ref_len = S.ref_len, plen = S.prompt_len;
     const int32_t last_tok = e->prompt_last[seq];  // kept on the host by llma_prefill
+    const int32_t k_min = S.k_min, k_start = S.k_start;
     std::memset(&S, 0, sizeof(S));
+    S.k_min = k_min; S.k_start = k_start; S.k_cur = k_start;
     S.active = 1; S.kv_len = plen - 1; S.pending = last_tok; S.ref_len = ref_len; S.prompt_len = plen;
     S.pos = -1; S.last_pos = -1; S.done = 1;
     e->last_step_valid = false;
+    return store_state(e, seq);
+}
+
+extern "C" int llma_set_adaptive_k(llma_engine* e, int32_t seq, int32_t k_min, int32_t k_start) {
+    if (!e) return LLMA_ERR_NULL;
+    if (seq < 0 || seq >= e->dims.max_batch) return LLMA_ERR_CAPACITY;
+    const bool off = k_min == 0 && k_start == 0;
+    if (!off && (k_min < 1 || k_start < k_min || k_start > e->dims.kp1 - 1)) return LLMA_ERR_ARG;
+    int rc = fetch_state(e);
+    if (rc) return rc;
+    SeqState& S = e->h_state[seq];
+    S.k_min = k_min; S.k_start = k_start; S.k_cur = k_start;
     return store_state(e, seq);
 }
 

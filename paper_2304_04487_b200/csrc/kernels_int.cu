@@ -115,6 +115,10 @@ __global__ void __launch_bounds__(kTailThreads) step_tail_kernel(const TailArgs 
                 }
                 for (int j = lane; j < m; j += 32) ys[ylen + j] = o[j];
                 pending = o[m - 1];
+                // adaptive copy length: twice as many tokens after a copy the model agreed with in full, half as
+                // many (rounded up) after one it cut short; within [k_min, the engine's largest k]
+                if (lane == 0 && S.k_cur > 0 && k_eff > 0)
+                    S.k_cur = acc == k_eff ? min(2 * S.k_cur, dims.kp1 - 1) : max(S.k_min, (S.k_cur + 1) >> 1);
             }
             __syncwarp();
             if (lane == 0) {
@@ -202,7 +206,8 @@ __global__ void __launch_bounds__(kTailThreads) step_tail_kernel(const TailArgs 
                     const int room_doc = __ldg(&de[pos - 1]) - pos;
                     const int room_out = S.target_len - ylen - 1;
                     const int room_kv = dims.max_seq - S.kv_len - 1;
-                    k_eff = min(min(a.k, room_doc), min(room_out, room_kv));
+                    const int k_want = S.k_cur > 0 ? min(S.k_cur, a.k) : a.k;
+                    k_eff = min(min(k_want, room_doc), min(room_out, room_kv));
                     if (k_eff <= 0) { k_eff = 0; pos = -1; }
                 }
                 nrows = k_eff + 1;

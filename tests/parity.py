@@ -55,16 +55,16 @@ def gpu_kv_rows(eng, seq: int, pos: int):
 
 def step_parity(eng, oracle_model, prompt: Sequence[int], ref: Sequence[int], offs: Optional[Sequence[int]],
                 n: int, k: int, n_new: int, mode: str, seq: int = 0, tie_margin: float = 1e-3,
-                prescribe_kv: bool = False, check_logits: bool = True) -> ParityReport:
+                prescribe_kv: bool = False, check_logits: bool = True, adaptive=None) -> ParityReport:
     """Drive ``eng.llma_step`` and the oracle side by side for ``n_new`` tokens of one sequence."""
     assert seq == 0
     return step_parity_batch(eng, [oracle_model], [prompt], [ref], [offs], n, k, n_new, mode, tie_margin,
-                             prescribe_kv, check_logits)[0]
+                             prescribe_kv, check_logits, adaptive)[0]
 
 
 def step_parity_batch(eng, oracle_models, prompts, refs, offs_list, n: int, k: int, n_new: int, mode: str,
-                      tie_margin: float = 1e-3, prescribe_kv: bool = False, check_logits: bool = True
-                      ) -> List[ParityReport]:
+                      tie_margin: float = 1e-3, prescribe_kv: bool = False, check_logits: bool = True,
+                      adaptive=None) -> List[ParityReport]:
     """Several sequences decoded together by ``eng.llma_step`` (one forward pass per step for all of
     them), each compared with its own oracle run: integer results per step, every logits row, tokens.
     Runs until every sequence has at least ``n_new`` tokens.
@@ -74,7 +74,10 @@ def step_parity_batch(eng, oracle_models, prompts, refs, offs_list, n: int, k: i
     tolerance (1e-4 of the row scale) of the oracle's unrounded value gives that code (counted in ``code_flips``;
     anything else is counted in ``code_violations`` and must not happen).  Both sides then take that decision
     alike and the logits compare the arithmetic instead of the butterfly effect of single rounding flips.
-    Prompt rows are prescribed too."""
+    Prompt rows are prescribed too.
+
+    ``adaptive = (k_min, k_start)``: the adaptive copy length is switched on for every sequence and the plan the
+    engine must follow comes from ``oracle.decoding.next_copy_request``."""
     B = len(prompts)
     reps = [ParityReport() for _ in range(B)]
     refs = [[int(t) for t in r] for r in refs]
@@ -90,12 +93,16 @@ def step_parity_batch(eng, oracle_models, prompts, refs, offs_list, n: int, k: i
         else:
             L[s], pending[s] = D.prefill(oracle_models[s], prompts[s])
         assert eng.llma_kv_len(s) == L[s]
+        if adaptive:
+            eng.llma_set_adaptive_k(s, adaptive[0], adaptive[1])
+    k_cur = [adaptive[1] if adaptive else 0] * B
     while min(len(y) for y in ys) < n_new:
         want = []
         for s in range(B):
             ref, offs, y = refs[s], offs_list[s], ys[s]
             matched, pos, _ = D.match_ngrams(y, ref, offs, n)
-            k_eff = D.copy_length(pos, len(ref), offs, k, eng.max_seq - L[s]) if matched else 0
+            k_ask = min(k_cur[s], k) if adaptive else k
+            k_eff = D.copy_length(pos, len(ref), offs, k_ask, eng.max_seq - L[s]) if matched else 0
             want.append((pos, k_eff, [pending[s]] + (ref[pos:pos + k_eff] if k_eff > 0 else [])))
         # the integer plan above needs no model, so the engine can go first and its cache rows (also those of
         # copied tokens that will be rejected: they stay in the cache until overwritten) can be prescribed
@@ -131,6 +138,8 @@ def step_parity_batch(eng, oracle_models, prompts, refs, offs_list, n: int, k: i
                 ga += 1
             assert got_tokens == gouts[:ga + 1], (s, rep.steps, got_tokens, gouts, ga)
             assert info.accepted == ga and info.emitted == ga + 1
+            if adaptive:
+                k_cur[s] = D.next_copy_request(k_cur[s], k_eff, ga, adaptive[0], eng.max_k)
             if got_tokens != want_tokens:
                 common = min(len(got_tokens), len(want_tokens))
                 diff = [i for i in range(common) if got_tokens[i] != want_tokens[i]]

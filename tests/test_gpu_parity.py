@@ -242,6 +242,52 @@ def test_batched_ragged_stepwise_parity(name, B, k):
     eng.llma_destroy()
 
 
+@pytest.mark.parametrize("name,B,k_max,adaptive", [("tiny-bf16", 6, 16, (1, 2)), ("tiny-fp32", 3, 8, (2, 4))])
+def test_adaptive_copy_length_stepwise_parity(name, B, k_max, adaptive):
+    """The adaptive copy length (a variant beyond the paper): every step's plan must be the one the oracle's
+    rule gives, per sequence, and llma_generate over the whole loop must follow the oracle's trace too."""
+    from paper_2304_04487_b200 import LlmaError
+    shape = SHAPES[name]
+    w = _weights(shape)
+    N = 40
+    prompts = [make_prompt(15 + 6 * s, shape.vocab, seed=60 + s) for s in range(B)]
+    max_seq = max(len(p) for p in prompts) + N + 2 * k_max + 8
+    refs, offs_list, models = [], [], []
+    for s in range(B):
+        y_star = D.greedy_decode(OM.OracleModel(shape, w, max_seq=max_seq), prompts[s], N).tokens
+        ref, offs, _ = build_reference(y_star, [40, 40], 0.6 + 0.08 * s, shape.vocab, seed=70 + s)
+        refs.append(ref); offs_list.append(offs)
+        models.append(OM.OracleModel(shape, w, max_seq=max_seq))
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=80, max_k=k_max, max_batch=B, keep_logits=True)
+    mode = "fp32" if shape.dtype == "fp32" else "bf16"
+    reps = step_parity_batch(eng, models, prompts, refs, offs_list, 1, k_max, N, mode, adaptive=adaptive)
+    assert sum(r.trigger_steps for r in reps) > B and sum(r.copied_accepted for r in reps) > 2 * B
+    for r in reps:
+        assert r.max_logit_err <= (2e-2 if mode == "bf16" else 1e-4 * max(1.0, r.max_logit_scale))
+    # the whole loop on the device: sequence 0 alone after a rewind, against the oracle's adaptive decode
+    for s in range(1, B):
+        eng.llma_reset(s)
+    eng.llma_rewind(0)                                            # keeps the setting, k_cur back to k_start
+    outs, st = eng.llma_generate(N, 1, k_max)
+    got = outs[0]
+    want = D.llma_decode(OM.OracleModel(shape, w, max_seq=max_seq), prompts[0], refs[0], offs_list[0], 1, k_max, N,
+                         adaptive=(adaptive[0], adaptive[1], k_max))
+    fixed = D.llma_decode(OM.OracleModel(shape, w, max_seq=max_seq), prompts[0], refs[0], offs_list[0], 1, k_max, N)
+    assert list(got) == want.tokens == fixed.tokens
+    assert (st.steps, st.trigger_steps, st.copied_accepted) == (want.steps, want.trigger_steps, want.copied_accepted)
+    assert want.steps != fixed.steps or [r.k_eff for r in want.trace] != [r.k_eff for r in fixed.trace]
+    # switched off again: the fixed-k trace
+    eng.llma_set_adaptive_k(0, 0, 0)
+    eng.llma_rewind(0)
+    outs, st = eng.llma_generate(N, 1, k_max)
+    got = outs[0]
+    assert list(got) == fixed.tokens and st.steps == fixed.steps
+    for bad in ((0, 3), (3, 2), (1, k_max + 1), (-1, 2)):
+        with pytest.raises(LlmaError):
+            eng.llma_set_adaptive_k(0, *bad)
+    eng.llma_destroy()
+
+
 def test_batched_generate_equals_single_sequence_runs():
     """llma_generate over 16 sequences: each output equals what the same sequence gives alone (greedy on a
     one-sequence engine), and the whole-loop statistics add up."""

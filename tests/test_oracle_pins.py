@@ -216,6 +216,81 @@ def test_loop_invariants_scripted(seed):
         assert pos_calls[0] == 2
 
 
+# --------------------------------------------------------------------------------------
+# the adaptive copy length (a variant beyond the paper) and the trigger fall-back identity
+# --------------------------------------------------------------------------------------
+def test_next_copy_request_by_hand():
+    f = D.next_copy_request
+    assert f(4, 0, 0, 1, 16) == 4        # nothing copied: unchanged
+    assert f(4, 4, 4, 1, 16) == 8        # accepted in full: doubled
+    assert f(4, 2, 2, 1, 16) == 8        # ... also when the document end had cut the copy short
+    assert f(12, 12, 12, 1, 16) == 16    # capped
+    assert f(5, 5, 1, 1, 16) == 3        # cut short: halved, rounding up
+    assert f(3, 3, 0, 2, 16) == 2
+    assert f(2, 2, 1, 2, 16) == 2        # never below k_min
+    assert f(1, 1, 0, 1, 16) == 1
+
+
+def test_adaptive_copy_length_trace_by_hand():
+    # the reference repeats the target except for one token (index 6: 40 instead of 16)
+    target = list(range(10, 26))
+    ref = target[:6] + [40] + target[7:]
+    prompt = [7, 8, 9]
+    m = ScriptedModel(target, len(prompt) - 1, prompt[-1], 50)
+    res = D.llma_decode(m, prompt, ref, None, 1, 8, len(target), adaptive=(1, 2, 8))
+    assert res.tokens == target
+    # step by step: nothing generated yet; 2 asked, both accepted (-> 4); 4 asked, the third is the changed
+    # token (-> 2); "16" is nowhere in the reference; 2 asked, both accepted (-> 4); 4 asked and accepted
+    assert [(r.pos, r.k_eff, r.accepted) for r in res.trace] == [
+        (-1, 0, 0), (1, 2, 2), (4, 4, 2), (-1, 0, 0), (8, 2, 2), (11, 4, 4)]
+    # the same run at the fixed k = 8 needs fewer steps but feeds more rows
+    fixed, _ = scripted_run(target, ref, None, 1, 8, vocab=50)
+    assert [(r.k_eff, r.accepted) for r in fixed.trace] == [(0, 0), (8, 5), (0, 0), (7, 7)]
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_adaptive_copy_length_invariants(seed):
+    rng = np.random.default_rng(100 + seed)
+    N = 70
+    target = rng.integers(1, 6, N).tolist()
+    ref = []
+    for _ in range(6):
+        a = int(rng.integers(0, N - 10)); ref += target[a:a + int(rng.integers(3, 14))]
+        ref += rng.integers(1, 6, int(rng.integers(0, 3))).tolist()
+    offs = [0, len(ref) // 2, len(ref)]
+    prompt = [7, 8, 9]
+    for n, (k_min, k_start, k_cap) in itertools.product((1, 2), ((1, 1, 8), (2, 4, 8), (1, 8, 8), (3, 3, 12))):
+        m = ScriptedModel(target, len(prompt) - 1, prompt[-1], 8)
+        res = D.llma_decode(m, prompt, ref, offs, n, k_cap, N, adaptive=(k_min, k_start, k_cap))
+        assert res.tokens == target                                   # still the greedy output
+        k_cur = k_start
+        for r in res.trace:
+            assert r.k_eff <= k_cur and k_min <= k_cur <= k_cap      # never more than was asked for
+            k_cur = D.next_copy_request(k_cur, r.k_eff, r.accepted, k_min, k_cap)
+    # pinned at one value the variant is the fixed-k algorithm
+    for k in (1, 5):
+        m = ScriptedModel(target, len(prompt) - 1, prompt[-1], 8)
+        res = D.llma_decode(m, prompt, ref, offs, 1, k, N, adaptive=(k, k, k))
+        fixed, _ = scripted_run(target, ref, offs, 1, k, vocab=8)
+        assert res.trace == fixed.trace
+
+
+def test_trigger_fallback_is_the_shorter_trigger():
+    """Trying triggers of length n, n-1, ..., n_lo in turn finds what a trigger of length n_lo finds."""
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        ref = rng.integers(1, 4, int(rng.integers(4, 30))).tolist()
+        y = rng.integers(1, 4, int(rng.integers(0, 12))).tolist()
+        offs = [0, int(rng.integers(1, len(ref))), len(ref)]
+        for n, n_lo in ((3, 1), (3, 2), (2, 1)):
+            chain = (False, -1, 0)
+            for nn in range(n, n_lo - 1, -1):
+                chain = D.match_ngrams(y, ref, offs, nn)
+                if chain[0]:
+                    break
+            assert chain == D.match_ngrams(y, ref, offs, n_lo)
+
+
 def test_nontrigger_steps_match_bruteforce_count():
     rng = np.random.default_rng(11)
     N = 80
