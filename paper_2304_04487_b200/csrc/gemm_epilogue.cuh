@@ -128,6 +128,55 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, int tile, int ro
     epi_sync();
 }
 
+// The same for the wide kernel (blocks of up to 32 rows, rotary factors read from the tables in global
+// memory): a tile of many rows is not latency-critical code, so eight rows are in flight at a time --
+// their positions, rotary factors and staged values are all requested before any is used.
+__device__ __forceinline__ void epilogue_qkv_wide(const GemmArgs& g, int tile, int row, int jb, int nj,
+                                                  float (*stage)[33], const int* row_pos, const int* row_seq) {
+    const ModelDims& d = g.dims;
+    const int mat = tile / g.tiles_per_map;
+    const int col = (tile % g.tiles_per_map) * 128 + row;
+    const int hd = d.head_dim, half = hd >> 1;
+    const int head = col / hd, idx = col % hd;
+    const bool lower = idx < half;
+    const int prow = lower ? row + half : row - half;
+    const int fi = idx % half;
+    if (col < g.n_out) {
+        const int64_t thread_off = (((int64_t)g.layer * d.max_batch * d.n_heads + head) * d.max_seq) * hd + idx;
+        const int64_t seq_stride = (int64_t)d.n_heads * d.max_seq * hd;
+        constexpr int kU = 8;
+#pragma unroll 1
+        for (int j0 = 0; j0 < nj; j0 += kU) {
+            int pos[kU];
+            float2 cs[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                pos[u] = j0 + u < nj ? row_pos[jb + j0 + u] : -1;
+                cs[u] = make_float2(1.f, 0.f);
+                if (mat < 2 && pos[u] >= 0)
+                    cs[u] = make_float2(__ldg(&g.rope_cos[(int64_t)pos[u] * half + fi]), __ldg(&g.rope_sin[(int64_t)pos[u] * half + fi]));
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                if (pos[u] < 0) continue;
+                const int j = j0 + u;
+                float v = stage[row][j];
+                if (mat < 2) {
+                    const float other = stage[prow][j];
+                    v = lower ? (v * cs[u].x - other * cs[u].y) : (other * cs[u].y + v * cs[u].x);
+                }
+                if (mat == 0) {
+                    g.out_f32[(int64_t)(jb + j) * g.ld + col] = v;
+                } else {
+                    __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
+                    cache[thread_off + row_seq[jb + j] * seq_stride + (int64_t)pos[u] * hd] = __float2bfloat16_rn(v);
+                }
+            }
+        }
+    }
+    epi_sync();
+}
+
 // SwiGLU: tile rows 0..63 are gate features, 64..127 the matching up features.
 __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33]) {

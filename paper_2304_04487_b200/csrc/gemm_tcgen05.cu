@@ -495,6 +495,18 @@ int make_tensor_map_bf16_pair(CUtensorMap* out, const void* base0, const void* b
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+int make_tensor_map_bf16_terms(CUtensorMap* out, const void* base, uint64_t rc, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || box_rows > 256) return -1;
+    const cuuint64_t dims[3] = {cols, rc, 2};
+    const cuuint64_t strides[2] = {cols * 2, rc * cols * 2};
+    const cuuint32_t box[3] = {64, box_rows, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return (int)fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return -1;

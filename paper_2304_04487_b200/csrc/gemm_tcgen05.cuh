@@ -103,9 +103,9 @@ template <int NR> struct GemmCfg {
 // Shared-memory plan of gemm_wide_kernel for nr rows: a ring of weight tiles (16 KB each) and a ring of
 // activation tiles (nr rows of 128 bytes each: one term of one 64-wide k-chunk), as many as fit.
 struct GemmWideCfg {
-    uint32_t b_slot;    // bytes of one activation tile
+    uint32_t b_slot;    // bytes of one activation tile: nr rows of 128 bytes for each of the two terms
     int sa, sb;         // ring depths (each at most 8)
-    uint32_t tmem_cols; // power of two >= 2 nr (two accumulators)
+    uint32_t tmem_cols; // power of two >= the accumulators' columns (2 nr each; two of them up to 128 rows, else one)
     size_t smem_bytes;
 };
 GemmWideCfg gemm_wide_cfg(int nr);
@@ -116,6 +116,9 @@ int gemm_grid_for(int64_t work, int num_sms);
 // Encode a 2-D bf16 row-major [rows, cols] tensor for TMA with a {64, box_rows} box and
 // 128-byte swizzle.  Returns a CUresult (0 = success).
 int make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// A split activation buffer [2 rc, cols] (hi rows, then lo rows) seen as (cols, rc rows, 2 terms) with a
+// {64, box_rows, 2} box: one copy lands the hi rows of a 64-wide k-chunk followed by its lo rows.
+int make_tensor_map_bf16_terms(CUtensorMap* out, const void* base, uint64_t rc, uint64_t cols, uint32_t box_rows);
 // The same tensor seen as (64 columns, rows, cols / 64 chunks) with a {64, box_rows, 2} box: two
 // consecutive k-chunks of box_rows rows per copy, landing as two tiles of the 2-D layout one after the other.
 int make_tensor_map_bf16_chunks(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);

@@ -1,9 +1,11 @@
 // Weight-streaming GEMM for up to 256 activation rows (batched decoding steps, prompt passes).
 // Same contract, work split and fused epilogues as gemm_ws_kernel (see gemm_tcgen05.cuh); what differs:
-//   * the activation tiles are large enough for TMA to pay: a second producer thread streams them
-//     through a ring of their own (one slot = nr rows x 64 columns of ONE bf16 term, hi or lo); both terms
-//     are accumulated into the same TMEM columns, so 256 rows fit two accumulators;
-//   * MMA N = the rows in use rounded up to 16 (a run-time field of the instruction descriptor);
+//   * the activation tiles are large enough for TMA to pay: a second producer warp streams them
+//     through a ring of their own (one slot = the nr hi rows, then the nr lo rows, of one 64-wide k-chunk,
+//     fetched by one copy through a 3-D view of the split buffer);
+//   * an accumulator has 2 nr columns [hi | lo], summed by the epilogue: up to 128 rows one MMA of N = 2 nr per
+//     k-slice and two accumulators in turn; beyond, two MMAs per k-slice (N = the rows in use rounded up to 16,
+//     a run-time field of the instruction descriptor) and a single accumulator;
 //   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
 //
 // Roles inside one CTA of 224 threads:
@@ -36,8 +38,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const int nr = g.nr;
-    constexpr int NT = 2;  // bf16 terms of the activation operand: hi, lo
-    const uint32_t b_slot = (uint32_t)nr * 128u;
+    // accumulators of 2 nr columns (hi | lo): two of them while they fit the 512 TMEM columns, else one
+    const int n_acc = 4 * nr <= 512 ? 2 : 1;
+    const uint32_t b_slot = (uint32_t)nr * 256u;  // nr hi rows, then nr lo rows, of one 64-wide k-chunk
     const uint32_t sA = base, sB = base + (uint32_t)SA * kGemmABytes;
     uint8_t* after = gen_base + (size_t)SA * kGemmABytes + (size_t)SB * b_slot;
     float (*stage)[33] = reinterpret_cast<float (*)[33]>(after);
@@ -93,7 +96,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     // One thread gets a TMA copy under way about every 0.5 us, whatever the copy's size (measured: 16 KB boxes from one
     // thread stream 31 GB/s per CTA, from two threads 59, from four 95, L2-resident).  A work item needs three copies
     // (a weight tile and the two terms of the activation tile), so the copies are dealt over several issuing threads.
-    constexpr int kPA = 2, kPB = 4;  // issuing lanes of the weight producer warp / of the activation producer warp
+    // (the ring depths are multiples of the lane counts: see gemm_wide_cfg)
+    constexpr int kPA = 2;              // issuing lanes of the weight producer warp
+    const int kPB = SB < 4 ? SB : 4;    // issuing lanes of the activation producer warp
     if (warp == 4) {
         // ------------------------------- weight producers (lane p takes items p, p + kPA, ...) -----------------
         if (lane < kPA) {
@@ -121,20 +126,18 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             }
         }
     } else if (warp == 6) {
-        // ------------------------------- activation producers (lane p takes (item, term) pairs p, p + kPB, ...) --
+        // ------------------------------- activation producers (lane p takes items p, p + kPB, ...) -------------
         if (lane < kPB) {
             grid_dependency_wait();  // activations are written by the kernel before this one
-            const int64_t n_pairs = n_items * NT;
             int64_t q = lane;
-            for (; q < n_pairs && !sh[1]; q += kPB) {
-                const int64_t w = w_beg + q / NT;
-                const int t = (int)(q % NT);
+            for (; q < n_items && !sh[1]; q += kPB) {
+                const int64_t w = w_beg + q;
                 const int c = (int)(w % C);
                 const int s = (int)(q % SB);
                 const uint32_t ph = (uint32_t)((q / SB) & 1);
                 if (q >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_b(s), b_slot);
-                tma_load_2d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, t * g.rc);
+                tma_load_3d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, 0, 0);
             }
             if (sh[1]) {
                 for (int64_t j = q - kPB; j >= 0 && j > q - kPB * (SB + 1); j -= kPB)
@@ -147,33 +150,57 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             grid_dependency_wait();  // the count of rows in use comes from the planning kernel
             int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : nr;
             rows_used = max(1, min(rows_used, nr));
-            const uint32_t idesc = idesc_bf16_m128((uint32_t)((rows_used + 15) & ~15));
+            // Up to 128 rows: ONE MMA per k-slice over the hi and the lo rows together (N = 2 nr, columns [hi | lo]).
+            // Consecutive MMAs into one accumulator run one after the other, each for about 0.1 us however narrow
+            // it is, so what counts is their number.  Beyond 128 rows N = 2 nr would pass the instruction's 256:
+            // two MMAs per k-slice, hi rows into the first nr columns and lo rows into the next nr (two
+            // independent accumulation chains), N = the rows in use rounded up to 16.
+            const bool one_mma = 2 * nr <= 256;
+            const uint32_t idesc = idesc_bf16_m128(one_mma ? (uint32_t)(2 * nr) : (uint32_t)((rows_used + 15) & ~15));
             int64_t ia = 0, ib = 0;
             int seg = 0;
+#ifdef LLMA_STAMPS
+            // measurement build: time this thread spends waiting for weight stages (word 6) and for activation
+            // slots (word 7), in ns
+            unsigned long long wait_a = 0, wait_b = 0, tw;
+#define LLMA_WAIT_BEGIN() (tw = globaltimer_ns())
+#define LLMA_WAIT_END(acc) (acc += globaltimer_ns() - tw)
+#else
+#define LLMA_WAIT_BEGIN() ((void)0)
+#define LLMA_WAIT_END(acc) ((void)0)
+#endif
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
                 const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
                 const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
-                const int buf = seg & 1;
-                const uint32_t use = (uint32_t)(seg >> 1);
+                const int buf = seg % n_acc;
+                const uint32_t use = (uint32_t)(seg / n_acc);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)nr;
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)(2 * nr);
                 for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
                     const int s = (int)(ia % SA);
+                    LLMA_WAIT_BEGIN();
                     if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    LLMA_WAIT_END(wait_a);
                     if (ia == 0) LLMA_STAMP(stp, 2);
                     const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
-                    for (int t = 0; t < NT; ++t, ++ib) {
+                    {
                         const int sb = (int)(ib % SB);
+                        LLMA_WAIT_BEGIN();
                         if (!mbar_wait(full_b(sb), (uint32_t)((ib / SB) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                        LLMA_WAIT_END(wait_b);
                         tc_fence_after();
                         const uint64_t db = smem_desc_sw128(sB + (uint32_t)sb * b_slot);
+                        const uint64_t db_lo = smem_desc_sw128(sB + (uint32_t)sb * b_slot + (uint32_t)nr * 128u);
+                        const uint32_t acc_on = c > c0 ? 1u : 0u;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (c > c0 || kk > 0 || t > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk) {  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
+                            if (!one_mma) umma_bf16(d_tmem + (uint32_t)nr, da + 2 * kk, db_lo + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
+                        }
                         umma_commit(empty_b(sb));  // slot is free once these MMAs have read it
+                        ++ib;
                     }
-                    if (sh[1]) break;
                     umma_commit(empty_a(s));
                 }
                 if (sh[1]) break;
@@ -181,6 +208,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 LLMA_STAMP(stp, 3);
                 w += c1 - c0;
             }
+#ifdef LLMA_STAMPS
+            if (stp) { stp[6] = wait_a; stp[7] = wait_b; }
+#endif
         }
     } else {
         // ------------------------------- epilogue warps ------------------------------------------
@@ -223,29 +253,32 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
             }
             epi_sync();
-            if constexpr (MODE == kGemmQKV) epilogue_qkv(g, tile, row, jb, nj, stage, s_pos, s_seq, nullptr);
+            if constexpr (MODE == kGemmQKV) epilogue_qkv_wide(g, tile, row, jb, nj, stage, s_pos, s_seq);
             else if constexpr (MODE == kGemmResid) epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
             else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, jb, nj, stage);
             else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, jb, nj, stage);
             else epilogue_lmhead(g, tile, row, jb, nj, stage, red_f, red_i);
             epi_sync();  // the staging area is rewritten by the next block
         };
-        // Tiles cut by a range boundary.  The CTA whose range holds the tile's LAST chunks owns it: it parks its own
-        // partial in slot 0 of its workspace and completes the tile after its last segment; every other CTA of the tile
-        // hands its partial over through slot 1 (all-ones words while empty, see gemm_ws_kernel).
+        // Tiles cut by a range boundary are summed block by block: every CTA of such a tile writes its whole partial
+        // (all-ones words while empty, see gemm_ws_kernel) into its own workspace slot -- slot 0 for the tile its
+        // range begins in, slot 1 for any other -- and the tile's 32-row blocks are dealt over its CTAs: after its
+        // last segment a CTA collects, for each block dealt to it, the partials of all the tile's CTAs in ascending
+        // k order (its own among them), puts all-ones back and runs the block's epilogue.  A tile cut into five
+        // thus ends with five CTAs each finishing a fifth of it, instead of one CTA finishing all of it.
         constexpr uint32_t kEmpty = 0xFFFFFFFFu;
         // slots are laid out for the engine's row capacity whatever nr is: a prompt pass and a decoding step (different nr)
-        // then agree on where every CTA's slots are, and the never-emptied slot 0 of one cannot sit in a slot 1 of the other
+        // then agree on where every CTA's slots are
         const int qn = g.rc >> 2;
-        int own_tile = -1, own_first = 0;
+        const int tile_first = (int)(w_beg / C);
         bool aborted = false;
         int seg = 0;
         for (int64_t w = w_beg; w < w_end; ++seg) {
             const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
             const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
             w += c1 - c0;
-            const int buf = seg & 1;
-            const uint32_t use = (uint32_t)(seg >> 1);
+            const int buf = seg % n_acc;
+            const uint32_t use = (uint32_t)(seg / n_acc);
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
                 if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
@@ -259,13 +292,18 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             tc_fence_after();
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
             const bool shared_tile = w_beg > t_lo || w_end < t_hi;
-            const bool owner = w_end >= t_hi;
-            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)nr;
+            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)(2 * nr);
             for (int rb = 0; rb < nblk; ++rb) {
                 float acc[32];
                 tmem_ld_32cols(t0 + (uint32_t)rb * 32u, acc);
+                {
+                    float lo[32];
+                    tmem_ld_32cols(t0 + (uint32_t)nr + (uint32_t)rb * 32u, lo);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j] += lo[j];  // W * hi + W * lo
+                }
                 if (shared_tile) {
-                    float4* dst = ws_slot(g.ws, qn, b, owner ? 0 : 1, row) + (int64_t)rb * 8 * 128;
+                    float4* dst = ws_slot(g.ws, qn, b, tile == tile_first ? 0 : 1, row) + (int64_t)rb * 8 * 128;
 #pragma unroll
                     for (int q = 0; q < 8; ++q)  // only the columns of rows in use travel
                         if (rb * 32 + 4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
@@ -276,63 +314,64 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acce_bar(buf));  // MMA may overwrite this accumulator
-            if (shared_tile && owner) {
+        }
+        if (!aborted && w_end > w_beg) {
+            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
+            bool timed_out = false;
+            const int tile_last = (int)((w_end - 1) / C);
+            for (int which = 0; which < 2; ++which) {
+                const int tile = which == 0 ? tile_first : tile_last;
+                if (which == 1 && tile_last == tile_first) break;
+                const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
+                if (!(w_beg > t_lo || w_end < t_hi)) continue;  // the whole tile was this CTA's: finished above
+                // the tile's CTAs: those whose ranges hold its first and its last chunk, and everyone between
                 int b_first = (int)(t_lo * G / work);
                 while (cta_begin(work, b_first + 1, G) <= t_lo) ++b_first;
                 while (cta_begin(work, b_first, G) > t_lo) --b_first;
-                own_tile = tile; own_first = b_first;
-            }
-        }
-        if (own_tile >= 0 && !aborted) {
-            const unsigned long long give_up = globaltimer_ns() + 2000000000ull;
-            bool timed_out = false;
-            for (int rb = 0; rb < nblk; ++rb) {
-                const int jb = rb * 32;
-                float acc[32];
+                int b_last = (int)((t_hi - 1) * G / work);
+                while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
+                while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
+                const int P = b_last - b_first + 1, me = b - b_first;
+                for (int rb = 0; rb < nblk; ++rb) {
+                    if (rb * P / nblk != me) continue;  // dealt to another CTA of the tile
+                    const int jb = rb * 32;
+                    float acc[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-                for (int bb = own_first; bb < b; ++bb) {  // ascending k: a fixed summation order
-                    const float4* src = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
-                    float4 p[8];
-                    bool valid;
-                    do {
-                        valid = true;
+                    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+                    for (int bb = b_first; bb <= b_last; ++bb) {  // ascending k: a fixed summation order
+                        const int slot = (int)(cta_begin(work, bb, G) / C) == tile ? 0 : 1;
+                        float4* src = ws_slot(g.ws, qn, bb, slot, row) + (int64_t)rb * 8 * 128;
+                        float4 p[8];
+                        bool valid;
+                        do {
+                            valid = true;
 #pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
+                            for (int q = 0; q < 8; ++q)
+                                if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                if (jb + 4 * q < rows_used) {
+                                    valid = valid && __float_as_uint(p[q].x) != kEmpty;
+                                    if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
+                                    if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
+                                    if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
+                                }
+                            }
+                            if (!valid && (timed_out || globaltimer_ns() > give_up)) {
+                                atomicExch(g.dev_err, kDevErrTimeout); timed_out = true; break;
+                            }
+                        } while (!valid);
+                        const float e = __uint_as_float(kEmpty);
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
                             if (jb + 4 * q < rows_used) {
-                                valid = valid && __float_as_uint(p[q].x) != kEmpty;
-                                if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
-                                if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
-                                if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
+                                src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
+                                acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
                             }
                         }
-                        if (!valid && (timed_out || globaltimer_ns() > give_up)) {
-                            atomicExch(g.dev_err, kDevErrTimeout); timed_out = true; break;
-                        }
-                    } while (!valid);
-                    const float e = __uint_as_float(kEmpty);
-                    float4* wr = ws_slot(g.ws, qn, bb, 1, row) + (int64_t)rb * 8 * 128;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (jb + 4 * q < rows_used) {
-                            wr[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
-                            acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
-                        }
                     }
+                    finish_block(tile, rb, acc);
                 }
-                // this CTA's own partial comes last (it holds the highest k)
-                const float4* mine = ws_slot(g.ws, qn, b, 0, row) + (int64_t)rb * 8 * 128;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    if (jb + 4 * q < rows_used) {
-                        const float4 o = mine[q * 128];
-                        acc[4 * q] += o.x; acc[4 * q + 1] += o.y; acc[4 * q + 2] += o.z; acc[4 * q + 3] += o.w;
-                    }
-                }
-                finish_block(own_tile, rb, acc);
             }
         }
     }
@@ -348,15 +387,18 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
 // ---- host side ------------------------------------------------------------------------------------
 GemmWideCfg gemm_wide_cfg(int nr) {
     GemmWideCfg c;
-    c.b_slot = (uint32_t)nr * 128u;
+    c.b_slot = (uint32_t)nr * 256u;
     const size_t budget = (size_t)227 * 1024 - 1024 - kWideStageBytes - kWideTailBytes;
     // four weight tiles in flight first, then as many activation tiles as fit, then more weight tiles
+    // Ring depths are multiples of the number of issuing lanes (a power of two), so that a slot is always refilled
+    // by the same lane: a lane that waited for "released for the second time" on a slot whose first release it never
+    // waited for could be let through by the parity of a barrier that has not completed any phase yet.
     c.sb = (int)((budget - 4 * kGemmABytes) / c.b_slot);
-    if (c.sb > 8) c.sb = 8;
+    c.sb = c.sb >= 8 ? 8 : (c.sb >= 4 ? 4 : 2);
     c.sa = (int)((budget - (size_t)c.sb * c.b_slot) / kGemmABytes);
-    if (c.sa > 8) c.sa = 8;
+    c.sa = c.sa >= 8 ? 8 : (c.sa >= 6 ? 6 : 4);
     uint32_t cols = 32;
-    while (cols < 2u * (uint32_t)nr) cols <<= 1;
+    while (cols < (4u * (uint32_t)nr <= 512u ? 4u : 2u) * (uint32_t)nr) cols <<= 1;
     c.tmem_cols = cols;
     c.smem_bytes = 1024 + (size_t)c.sa * kGemmABytes + (size_t)c.sb * c.b_slot + kWideStageBytes + kWideTailBytes;
     if (c.smem_bytes < 120 * 1024) c.smem_bytes = 120 * 1024;  // one CTA per SM, as for the narrow kernel
