@@ -1,11 +1,16 @@
 // Weight-streaming GEMM for up to 256 activation rows (batched decoding steps, prompt passes).
 // Same contract, work split and fused epilogues as gemm_ws_kernel (see gemm_tcgen05.cuh); what differs:
-//   * the activation tiles are large enough for TMA to pay: a second producer warp streams them
-//     through a ring of their own (one slot = the nr hi rows, then the nr lo rows, of one 64-wide k-chunk,
-//     fetched by one copy through a 3-D view of the split buffer);
+//   * the activation tiles are large enough for TMA to pay: a ring stage holds the weight tile of one 64-wide
+//     k-chunk and, behind it, the chunk's activation tile (the nr hi rows, then the nr lo rows, fetched by one
+//     copy through a 3-D view of the split buffer); two producer warps fill the two halves of a stage, because
+//     only the activations have to wait for the kernel before;
 //   * an accumulator has 2 nr columns [hi | lo], summed by the epilogue: up to 128 rows one MMA of N = 2 nr per
 //     k-slice and two accumulators in turn; beyond, two MMAs per k-slice (N = the rows in use rounded up to 16,
-//     a run-time field of the instruction descriptor) and a single accumulator;
+//     a run-time field of the instruction descriptor) and a single accumulator.  An MMA of this shape (M 128,
+//     K 16) occupies the tensor core for about 81 ns whatever its N (measured for N = 16 .. 256, alone and dealt
+//     over several accumulators) and a commit costs the issuing thread another 45 ns, so the number of MMAs and
+//     commits per weight tile is what bounds the kernel: 4 + 1 up to 128 rows (0.37 us per 16 KB, the HBM rate),
+//     8 + 1 beyond;
 //   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
 //
 // Roles inside one CTA of 224 threads:
@@ -33,19 +38,24 @@ template <int MODE>
 __global__ void __launch_bounds__(kGemmWideThreads, 1)
 gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                  const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
-                 const int SA, const int SB, const uint32_t tmem_cols) {
+                 const int SA, const uint32_t tmem_cols) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
     const int nr = g.nr;
-    // accumulators of 2 nr columns (hi | lo): two of them while they fit the 512 TMEM columns, else one
-    const int n_acc = 4 * nr <= 512 ? 2 : 1;
+    // An accumulator has 2 nr columns [hi | lo] (see the MMA warp); two accumulators take turns while they fit the
+    // 512 TMEM columns, else there is one.
+    const bool one_mma = 2 * nr <= 256;
+    const int acc_cols = 2 * nr;
+    const int n_acc = 2 * acc_cols <= 512 ? 2 : 1;
     const uint32_t b_slot = (uint32_t)nr * 256u;  // nr hi rows, then nr lo rows, of one 64-wide k-chunk
-    const uint32_t sA = base, sB = base + (uint32_t)SA * kGemmABytes;
-    uint8_t* after = gen_base + (size_t)SA * kGemmABytes + (size_t)SB * b_slot;
+    const uint32_t stage_bytes = kGemmABytes + b_slot;  // weight tile, then activation tile
+    const int SB = SA;                                   // one ring: S stages
+    const uint32_t sA = base, sB = base + kGemmABytes;   // stage s: sA + s * stage_bytes, sB + s * stage_bytes
+    uint8_t* after = gen_base + (size_t)SA * stage_bytes;
     float (*stage)[33] = reinterpret_cast<float (*)[33]>(after);
     uint8_t* tail = after + kWideStageBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full_a[8], empty_a[8], full_b[8], empty_b[8], acc_full[2], acc_empty[2]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);  // full[8], empty[8], (16 unused), acc_full[2], acc_empty[2]
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(tail + 36 * 8);  // [0] TMEM base, [1] abort, [2] broadcast
     float* rscale = reinterpret_cast<float*>(tail + 36 * 8 + 16);                 // [256] per-row norm scales
     float* red_f = rscale + kRowCap;                                              // [4][32]
@@ -55,8 +65,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const uint32_t bar0 = smem_u32(bars);
     auto full_a = [&](int s) { return bar0 + 8u * s; };
     auto empty_a = [&](int s) { return bar0 + 8u * (8 + s); };
-    auto full_b = [&](int s) { return bar0 + 8u * (16 + s); };
-    auto empty_b = [&](int s) { return bar0 + 8u * (24 + s); };
+    auto full_b = full_a;    // both halves of a stage land on one barrier (two arrivals with their byte counts)
+    auto empty_b = empty_a;  // and are released together
     auto accf_bar = [&](int i) { return bar0 + 8u * (32 + i); };
     auto acce_bar = [&](int i) { return bar0 + 8u * (34 + i); };
 
@@ -72,7 +82,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     if (threadIdx.x == 0) LLMA_STAMP(stp, 0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < 8; ++s) {
-            mbar_init(full_a(s), 1); mbar_init(empty_a(s), 1); mbar_init(full_b(s), 1); mbar_init(empty_b(s), 1);
+            mbar_init(full_a(s), 2); mbar_init(empty_a(s), 1);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(accf_bar(i), 1); mbar_init(acce_bar(i), 4); }
         sh[1] = 0; sh[2] = 0;
@@ -97,8 +107,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     // thread stream 31 GB/s per CTA, from two threads 59, from four 95, L2-resident).  A work item needs three copies
     // (a weight tile and the two terms of the activation tile), so the copies are dealt over several issuing threads.
     // (the ring depths are multiples of the lane counts: see gemm_wide_cfg)
-    constexpr int kPA = 2;              // issuing lanes of the weight producer warp
-    const int kPB = SB < 4 ? SB : 4;    // issuing lanes of the activation producer warp
+    const int kPA = SA >= 4 ? 2 : 1;    // issuing lanes of the weight producer warp (SA is even from four stages on)
+    const int kPB = kPA;                // issuing lanes of the activation producer warp
     if (warp == 4) {
         // ------------------------------- weight producers (lane p takes items p, p + kPA, ...) -----------------
         if (lane < kPA) {
@@ -110,7 +120,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 if (it >= SA && !mbar_wait(empty_a(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_a(s), kGemmABytes);
                 const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
-                const uint32_t dstA = sA + s * kGemmABytes;
+                const uint32_t dstA = sA + (uint32_t)s * stage_bytes;
                 if (MODE == kGemmSwiGLU) {
                     tma_load_2d(dstA, &map_a0, full_a(s), c * 64, tile * 64);
                     tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_a(s), c * 64, tile * 64);
@@ -137,7 +147,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 const uint32_t ph = (uint32_t)((q / SB) & 1);
                 if (q >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_b(s), b_slot);
-                tma_load_3d(sB + (uint32_t)s * b_slot, &map_b, full_b(s), c * 64, 0, 0);
+                tma_load_3d(sB + (uint32_t)s * stage_bytes, &map_b, full_b(s), c * 64, 0, 0);
             }
             if (sh[1]) {
                 for (int64_t j = q - kPB; j >= 0 && j > q - kPB * (SB + 1); j -= kPB)
@@ -150,14 +160,12 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             grid_dependency_wait();  // the count of rows in use comes from the planning kernel
             int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : nr;
             rows_used = max(1, min(rows_used, nr));
-            // Up to 128 rows: ONE MMA per k-slice over the hi and the lo rows together (N = 2 nr, columns [hi | lo]).
-            // Consecutive MMAs into one accumulator run one after the other, each for about 0.1 us however narrow
-            // it is, so what counts is their number.  Beyond 128 rows N = 2 nr would pass the instruction's 256:
-            // two MMAs per k-slice, hi rows into the first nr columns and lo rows into the next nr (two
-            // independent accumulation chains), N = the rows in use rounded up to 16.
-            const bool one_mma = 2 * nr <= 256;
+            // Up to 128 rows: one MMA per k-slice over the hi and the lo rows together (N = 2 nr, columns [hi | lo]).
+            // Beyond (N = 2 nr would pass the instruction's 256): two MMAs per k-slice, the hi rows into the first
+            // nr columns and the lo rows into the next nr, N = the rows in use rounded up to 16.  Either way a
+            // column is summed over k in the same order, so a row's result does not depend on which applies.
             const uint32_t idesc = idesc_bf16_m128(one_mma ? (uint32_t)(2 * nr) : (uint32_t)((rows_used + 15) & ~15));
-            int64_t ia = 0, ib = 0;
+            int64_t ia = 0;
             int seg = 0;
 #ifdef LLMA_STAMPS
             // measurement build: time this thread spends waiting for weight stages (word 6) and for activation
@@ -176,32 +184,24 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 const uint32_t use = (uint32_t)(seg / n_acc);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)(2 * nr);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)acc_cols;
                 for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
                     const int s = (int)(ia % SA);
                     LLMA_WAIT_BEGIN();
                     if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                     LLMA_WAIT_END(wait_a);
                     if (ia == 0) LLMA_STAMP(stp, 2);
-                    const uint64_t da = smem_desc_sw128(sA + s * kGemmABytes);
-                    {
-                        const int sb = (int)(ib % SB);
-                        LLMA_WAIT_BEGIN();
-                        if (!mbar_wait(full_b(sb), (uint32_t)((ib / SB) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
-                        LLMA_WAIT_END(wait_b);
-                        tc_fence_after();
-                        const uint64_t db = smem_desc_sw128(sB + (uint32_t)sb * b_slot);
-                        const uint64_t db_lo = smem_desc_sw128(sB + (uint32_t)sb * b_slot + (uint32_t)nr * 128u);
-                        const uint32_t acc_on = c > c0 ? 1u : 0u;
+                    tc_fence_after();
+                    const uint64_t da = smem_desc_sw128(sA + (uint32_t)s * stage_bytes);
+                    const uint64_t db = smem_desc_sw128(sB + (uint32_t)s * stage_bytes);
+                    const uint64_t db_lo = smem_desc_sw128(sB + (uint32_t)s * stage_bytes + (uint32_t)nr * 128u);
+                    const uint32_t acc_on = c > c0 ? 1u : 0u;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
-                            umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
-                            if (!one_mma) umma_bf16(d_tmem + (uint32_t)nr, da + 2 * kk, db_lo + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
-                        }
-                        umma_commit(empty_b(sb));  // slot is free once these MMAs have read it
-                        ++ib;
+                    for (int kk = 0; kk < 4; ++kk) {  // 4 x K=16 slices of the 64-wide chunk: +32 bytes each
+                        umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
+                        if (!one_mma) umma_bf16(d_tmem + (uint32_t)nr, da + 2 * kk, db_lo + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty_a(s));
+                    umma_commit(empty_a(s));  // the stage is free once these MMAs have read it
                 }
                 if (sh[1]) break;
                 umma_commit(accf_bar(buf));  // accumulator complete
@@ -292,7 +292,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             tc_fence_after();
             const int64_t t_lo = (int64_t)tile * C, t_hi = t_lo + C;
             const bool shared_tile = w_beg > t_lo || w_end < t_hi;
-            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)(2 * nr);
+            const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)buf * (uint32_t)acc_cols;
             for (int rb = 0; rb < nblk; ++rb) {
                 float acc[32];
                 tmem_ld_32cols(t0 + (uint32_t)rb * 32u, acc);
@@ -389,18 +389,20 @@ GemmWideCfg gemm_wide_cfg(int nr) {
     GemmWideCfg c;
     c.b_slot = (uint32_t)nr * 256u;
     const size_t budget = (size_t)227 * 1024 - 1024 - kWideStageBytes - kWideTailBytes;
-    // four weight tiles in flight first, then as many activation tiles as fit, then more weight tiles
-    // Ring depths are multiples of the number of issuing lanes (a power of two), so that a slot is always refilled
-    // by the same lane: a lane that waited for "released for the second time" on a slot whose first release it never
-    // waited for could be let through by the parity of a barrier that has not completed any phase yet.
-    c.sb = (int)((budget - 4 * kGemmABytes) / c.b_slot);
-    c.sb = c.sb >= 8 ? 8 : (c.sb >= 4 ? 4 : 2);
-    c.sa = (int)((budget - (size_t)c.sb * c.b_slot) / kGemmABytes);
-    c.sa = c.sa >= 8 ? 8 : (c.sa >= 6 ? 6 : 4);
+    const size_t stage_bytes = kGemmABytes + c.b_slot;
+    // As many stages as fit, at most 8; an even number where there are four or more, because two lanes of each
+    // producer warp take turns (a stage must always be refilled by the same lane: a lane that waited for "released
+    // for the second time" on a stage whose first release it never waited for could be let through by the parity
+    // of a barrier that has not completed any phase yet).  With two or three stages one lane issues.
+    int S = (int)(budget / stage_bytes);
+    if (S > 8) S = 8;
+    if (S >= 4) S &= ~1;
+    c.sa = c.sb = S;
     uint32_t cols = 32;
-    while (cols < (4u * (uint32_t)nr <= 512u ? 4u : 2u) * (uint32_t)nr) cols <<= 1;
+    const uint32_t acc_cols = 2u * (uint32_t)nr;  // as in the kernel
+    while (cols < (2u * acc_cols <= 512u ? 2u : 1u) * acc_cols) cols <<= 1;
     c.tmem_cols = cols;
-    c.smem_bytes = 1024 + (size_t)c.sa * kGemmABytes + (size_t)c.sb * c.b_slot + kWideStageBytes + kWideTailBytes;
+    c.smem_bytes = 1024 + (size_t)S * stage_bytes + kWideStageBytes + kWideTailBytes;
     if (c.smem_bytes < 120 * 1024) c.smem_bytes = 120 * 1024;  // one CTA per SM, as for the narrow kernel
     return c;
 }
@@ -432,14 +434,14 @@ void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    const int sa = c.sa, sb = c.sb;
+    const int sa = c.sa;
     const uint32_t cols = c.tmem_cols;
     switch (args.mode) {
-        case kGemmQKV: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmQKV>, args, a0, a1, a2, map_b, sa, sb, cols); break;
-        case kGemmResid: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmResid>, args, a0, a1, a2, map_b, sa, sb, cols); break;
-        case kGemmSwiGLU: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmSwiGLU>, args, a0, a1, a2, map_b, sa, sb, cols); break;
-        case kGemmLmHead: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmLmHead>, args, a0, a1, a2, map_b, sa, sb, cols); break;
-        default: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmStore>, args, a0, a1, a2, map_b, sa, sb, cols); break;
+        case kGemmQKV: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmQKV>, args, a0, a1, a2, map_b, sa, cols); break;
+        case kGemmResid: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmResid>, args, a0, a1, a2, map_b, sa, cols); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmSwiGLU>, args, a0, a1, a2, map_b, sa, cols); break;
+        case kGemmLmHead: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmLmHead>, args, a0, a1, a2, map_b, sa, cols); break;
+        default: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmStore>, args, a0, a1, a2, map_b, sa, cols); break;
     }
 }
 
