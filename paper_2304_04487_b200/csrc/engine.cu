@@ -220,9 +220,12 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         // activation operands of the wide kernel: one box of nr rows per (buffer, use)
         auto act_maps = [&](llma_engine::ActMaps& m, int nr) {
             int bad2 = 0;
-            bad2 |= make_tensor_map_bf16_terms(&m.x_hat, e->x_hat, RC, d.d_model, nr);
-            bad2 |= make_tensor_map_bf16_terms(&m.attn, e->attn, RC, HD, nr);
-            bad2 |= make_tensor_map_bf16_terms(&m.h, e->h, RC, d.d_ffn, nr);
+            for (int i = 0; i < 4; ++i) {
+                const int box = wide_box_rows(nr, i);
+                bad2 |= make_tensor_map_bf16_terms(&m.x_hat[i], e->x_hat, RC, d.d_model, box);
+                bad2 |= make_tensor_map_bf16_terms(&m.attn[i], e->attn, RC, HD, box);
+                bad2 |= make_tensor_map_bf16_terms(&m.h[i], e->h, RC, d.d_ffn, box);
+            }
             return bad2;
         };
         bad |= act_maps(e->act_prefill, e->prefill_rows);

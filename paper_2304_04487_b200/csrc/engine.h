@@ -45,7 +45,9 @@ struct llma_engine {
     CUtensorMap map_lm_head, map_lm_head2;
     struct PairMap { CUtensorMap map; int gate_second; };   // gate and up matrices of a layer in one view (gemm_ws_kernel)
     std::vector<PairMap> gate_up_map;
-    struct ActMaps { CUtensorMap x_hat, attn, h; };  // activation operands of gemm_wide_kernel, box of nr rows
+    // activation operands of gemm_wide_kernel: boxes of min(32, nr), min(64, nr), min(128, nr) and nr rows (the kernel
+    // takes the smallest that holds the step's rows)
+    struct ActMaps { CUtensorMap x_hat[4], attn[4], h[4]; };
     ActMaps act_decode, act_prefill;
     bool decode_wide = false;       // decoding steps of more than 32 rows use gemm_wide_kernel
     int decode_nr = 32;             // rows the decoding GEMMs are shaped for (16 / 32 narrow, decode_rows wide)

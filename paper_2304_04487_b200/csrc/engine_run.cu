@@ -41,7 +41,7 @@ static void run_gemm(llma_engine* e, GemmArgs& a, const CUtensorMap& a0, const C
                      const void* act, const CUtensorMap* act_map) {
     a.act = act;
     const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
-    if (e->cur_wide) launch_gemm_wide(e->stream, grid, true, a, a0, a1, a2, *act_map);
+    if (e->cur_wide) launch_gemm_wide(e->stream, grid, true, a, a0, a1, a2, act_map);
     else launch_gemm_tcgen05(e->stream, grid, true, a, a0, a1, a2);
 }
 
@@ -65,7 +65,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         with_norm(e, q);
         q.out_f32 = e->qkv; q.ld = 3 * HD; q.layer = l; q.rope_cos = e->rope_cos; q.rope_sin = e->rope_sin;
         q.kcache = (__nv_bfloat16*)e->kcache; q.vcache = (__nv_bfloat16*)e->vcache;
-        run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat, am ? &am->x_hat : nullptr);
+        run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat, am ? am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_QKV);
         AttnArgs at;
         at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
@@ -78,13 +78,13 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
         o.out_f32 = e->x; o.ld = D; o.gain_next = e->ffn_norm[l]; o.xs_out = e->x_hat; o.ss_out = e->norm_ss;
-        run_gemm(e, o, m.wo, m.wo, m.wo, e->attn, am ? &am->attn : nullptr);
+        run_gemm(e, o, m.wo, m.wo, m.wo, e->attn, am ? am->attn : nullptr);
         mark(e, LLMA_K_GEMM_O);
         GemmArgs gu = gemm_args(e, kGemmSwiGLU, F, (F + 63) / 64, D, (F + 63) / 64);
         with_norm(e, gu);
         gu.out_act = e->h;
         if (e->cur_wide) {
-            run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat, &am->x_hat);
+            run_gemm(e, gu, m.w_gate, m.w_up, m.w_up, e->x_hat, am->x_hat);
         } else {  // one view over both matrices; whichever lies lower in memory fills the tile's first 64 rows
             gu.gate_second = e->gate_up_map[l].gate_second;
             run_gemm(e, gu, e->gate_up_map[l].map, e->gate_up_map[l].map, e->gate_up_map[l].map, e->x_hat, nullptr);
@@ -93,7 +93,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         GemmArgs dn = gemm_args(e, kGemmResid, D, (D + 127) / 128, F, (D + 127) / 128);
         dn.out_f32 = e->x; dn.ld = D; dn.xs_out = e->x_hat; dn.ss_out = e->norm_ss;
         dn.gain_next = l + 1 < d.n_layers ? e->attn_norm[l + 1] : e->final_norm;
-        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h, am ? &am->h : nullptr);
+        run_gemm(e, dn, m.w_down, m.w_down, m.w_down, e->h, am ? am->h : nullptr);
         mark(e, LLMA_K_GEMM_DOWN);
         e->launch_counter += 6;
     }
@@ -104,7 +104,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         lm.out_f32 = e->cfg.keep_logits ? e->logits : nullptr; lm.ld = d.vocab;
         lm.part_max = e->part_max; lm.part_idx = e->part_idx;
         const CUtensorMap& lmm = e->cur_wide ? e->map_lm_head : e->map_lm_head2;
-        run_gemm(e, lm, lmm, lmm, lmm, e->x_hat, am ? &am->x_hat : nullptr);
+        run_gemm(e, lm, lmm, lmm, lmm, e->x_hat, am ? am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_LMHEAD);
         e->launch_counter += 1;
     }
@@ -248,7 +248,8 @@ extern "C" int llma_prefill(llma_engine* e, int32_t seq, const int32_t* prompt, 
     if (rc) return rc;
     // push prompt[0 .. P-2] through the decoder, prefill_rows consecutive positions per pass
     const int n_cache = n_prompt - 1;
-    const int PR = e->prefill_rows;
+    // positions per prompt pass: at most 128 on the tensor-core path, so that the wide GEMM needs one MMA per k-slice
+    const int PR = e->gemm_impl == LLMA_GEMM_TCGEN05 ? std::min(e->prefill_rows, 128) : e->prefill_rows;
     shape_for_prefill(e);
     for (int p0 = 0; p0 < n_cache; p0 += PR) {
         const int cnt = std::min(PR, n_cache - p0);

@@ -137,10 +137,17 @@ cudaError_t init_gemm_tcgen05();
 void launch_gemm_tcgen05(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
                          const CUtensorMap& a1, const CUtensorMap& a2);
 
-// args.nr = 32 .. 256 (multiple of 16); map_b covers the activation buffer [2 rc][k_in] with a
-// {64, nr} box
+// args.nr = 32 .. 256 (multiple of 16); map_b[i] (make_tensor_map_bf16_terms) covers the split activation buffer
+// with a box of wide_box_rows(nr, i) rows, i = 0 .. 3
 cudaError_t init_gemm_wide();
 void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
-                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& map_b);
+                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap* map_b);
+// Activation rows per copy of gemm_wide_kernel, candidate i of four: 32, 64, 128 (none above nr), then nr itself.
+// A step takes the first candidate that holds its rows, so the activation traffic follows the rows in use, and
+// up to 128 rows the hi and lo rows sit close enough for one MMA over both.
+__host__ __device__ inline int wide_box_rows(int nr, int i) {
+    const int c = i == 0 ? 32 : (i == 1 ? 64 : (i == 2 ? 128 : nr));
+    return c < nr ? c : nr;
+}
 
 }  // namespace llma

@@ -37,19 +37,20 @@ constexpr size_t kWideTailBytes = 5120;  // barriers, flags, per-row scales, red
 template <int MODE>
 __global__ void __launch_bounds__(kGemmWideThreads, 1)
 gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
-                 const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
-                 const int SA, const uint32_t tmem_cols) {
+                 const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b0,
+                 const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_b2,
+                 const __grid_constant__ CUtensorMap map_b3, const int SA, const uint32_t tmem_cols) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const int nr = g.nr;
-    // An accumulator has 2 nr columns [hi | lo] (see the MMA warp); two accumulators take turns while they fit the
-    // 512 TMEM columns, else there is one.
-    const bool one_mma = 2 * nr <= 256;
-    const int acc_cols = 2 * nr;
-    const int n_acc = 2 * acc_cols <= 512 ? 2 : 1;
-    const uint32_t b_slot = (uint32_t)nr * 256u;  // nr hi rows, then nr lo rows, of one 64-wide k-chunk
-    const uint32_t stage_bytes = kGemmABytes + b_slot;  // weight tile, then activation tile
+    // g.nr is the row capacity the launch was shaped for; the rows a copy brings (nr below) are chosen per step from
+    // the rows in use, by every role that needs them, once the planning kernel's count may be read
+    const uint32_t stage_bytes = kGemmABytes + (uint32_t)g.nr * 256u;  // weight tile, then the largest activation tile
+    auto box_index = [&](int rows_used) {
+        int i = 0;
+        while (i < 3 && wide_box_rows(g.nr, i) < rows_used) ++i;
+        return i;
+    };
     const int SB = SA;                                   // one ring: S stages
     const uint32_t sA = base, sB = base + kGemmABytes;   // stage s: sA + s * stage_bytes, sB + s * stage_bytes
     uint8_t* after = gen_base + (size_t)SA * stage_bytes;
@@ -97,7 +98,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         if (MODE == kGemmQKV) { tma_prefetch_desc(&map_a1); tma_prefetch_desc(&map_a2); }
         if (MODE == kGemmSwiGLU) tma_prefetch_desc(&map_a1);
     }
-    if (warp == 6 && lane == 0) tma_prefetch_desc(&map_b);
+    if (warp == 6 && lane == 0) { tma_prefetch_desc(&map_b0); tma_prefetch_desc(&map_b1); tma_prefetch_desc(&map_b2); tma_prefetch_desc(&map_b3); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -139,6 +140,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         // ------------------------------- activation producers (lane p takes items p, p + kPB, ...) -------------
         if (lane < kPB) {
             grid_dependency_wait();  // activations are written by the kernel before this one
+            const int bi = box_index(g.rows ? min(__ldcg(&g.rows->rows_used), g.nr) : g.nr);
+            const CUtensorMap* map_b = bi == 0 ? &map_b0 : (bi == 1 ? &map_b1 : (bi == 2 ? &map_b2 : &map_b3));
+            const uint32_t b_slot = (uint32_t)wide_box_rows(g.nr, bi) * 256u;  // hi rows, then lo rows, of one k-chunk
             int64_t q = lane;
             for (; q < n_items && !sh[1]; q += kPB) {
                 const int64_t w = w_beg + q;
@@ -147,7 +151,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 const uint32_t ph = (uint32_t)((q / SB) & 1);
                 if (q >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_b(s), b_slot);
-                tma_load_3d(sB + (uint32_t)s * stage_bytes, &map_b, full_b(s), c * 64, 0, 0);
+                tma_load_3d(sB + (uint32_t)s * stage_bytes, map_b, full_b(s), c * 64, 0, 0);
             }
             if (sh[1]) {
                 for (int64_t j = q - kPB; j >= 0 && j > q - kPB * (SB + 1); j -= kPB)
@@ -158,12 +162,18 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         // ------------------------------- MMA issuer ---------------------------------------------
         if (lane == 0) {
             grid_dependency_wait();  // the count of rows in use comes from the planning kernel
-            int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : nr;
-            rows_used = max(1, min(rows_used, nr));
+            int rows_used = g.rows ? __ldcg(&g.rows->rows_used) : g.nr;
+            rows_used = max(1, min(rows_used, g.nr));
+            const int nr = wide_box_rows(g.nr, box_index(rows_used));  // hi rows at 0, lo rows nr further on
+            // An accumulator has 2 nr columns [hi | lo]; two accumulators take turns while they fit the 512 TMEM
+            // columns, else there is one.
+            const int acc_cols = 2 * nr;
+            const int n_acc = 2 * acc_cols <= 512 ? 2 : 1;
             // Up to 128 rows: one MMA per k-slice over the hi and the lo rows together (N = 2 nr, columns [hi | lo]).
             // Beyond (N = 2 nr would pass the instruction's 256): two MMAs per k-slice, the hi rows into the first
             // nr columns and the lo rows into the next nr, N = the rows in use rounded up to 16.  Either way a
             // column is summed over k in the same order, so a row's result does not depend on which applies.
+            const bool one_mma = 2 * nr <= 256;
             const uint32_t idesc = idesc_bf16_m128(one_mma ? (uint32_t)(2 * nr) : (uint32_t)((rows_used + 15) & ~15));
             int64_t ia = 0;
             int seg = 0;
@@ -216,7 +226,10 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         // ------------------------------- epilogue warps ------------------------------------------
         grid_dependency_wait();  // everything below reads or writes what earlier kernels produced
         if (threadIdx.x == 0) LLMA_STAMP(stp, 1);
-        const int rows_used = g.rows ? min(g.rows->rows_used, nr) : nr;
+        const int rows_used = g.rows ? min(g.rows->rows_used, g.nr) : g.nr;
+        const int nr = wide_box_rows(g.nr, box_index(max(rows_used, 1)));  // as the MMA warp sees it
+        const int acc_cols = 2 * nr;
+        const int n_acc = 2 * acc_cols <= 512 ? 2 : 1;
         const int nblk = (rows_used + 31) >> 5;
         const int row = threadIdx.x;  // 0..127 = TMEM lane = output feature inside the tile
         if (g.ss_in) {  // folded RMSNorm: one scale per activation row, tiles summed in ascending order
@@ -399,8 +412,10 @@ GemmWideCfg gemm_wide_cfg(int nr) {
     if (S >= 4) S &= ~1;
     c.sa = c.sb = S;
     uint32_t cols = 32;
-    const uint32_t acc_cols = 2u * (uint32_t)nr;  // as in the kernel
-    while (cols < (2u * acc_cols <= 512u ? 2u : 1u) * acc_cols) cols <<= 1;
+    for (int i = 0; i < 4; ++i) {  // the largest need over the row counts a step may choose (as in the kernel)
+        const uint32_t acc_cols = 2u * (uint32_t)wide_box_rows(nr, i);
+        while (cols < (2u * acc_cols <= 512u ? 2u : 1u) * acc_cols) cols <<= 1;
+    }
     c.tmem_cols = cols;
     c.smem_bytes = 1024 + (size_t)S * stage_bytes + kWideStageBytes + kWideTailBytes;
     if (c.smem_bytes < 120 * 1024) c.smem_bytes = 120 * 1024;  // one CTA per SM, as for the narrow kernel
@@ -422,7 +437,7 @@ cudaError_t init_gemm_wide() {
 }
 
 void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args, const CUtensorMap& a0,
-                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& map_b) {
+                      const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap* map_b) {
     const GemmWideCfg c = gemm_wide_cfg(args.nr);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -437,11 +452,11 @@ void launch_gemm_wide(cudaStream_t st, int grid, bool pdl, const GemmArgs& args,
     const int sa = c.sa;
     const uint32_t cols = c.tmem_cols;
     switch (args.mode) {
-        case kGemmQKV: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmQKV>, args, a0, a1, a2, map_b, sa, cols); break;
-        case kGemmResid: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmResid>, args, a0, a1, a2, map_b, sa, cols); break;
-        case kGemmSwiGLU: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmSwiGLU>, args, a0, a1, a2, map_b, sa, cols); break;
-        case kGemmLmHead: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmLmHead>, args, a0, a1, a2, map_b, sa, cols); break;
-        default: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmStore>, args, a0, a1, a2, map_b, sa, cols); break;
+        case kGemmQKV: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmQKV>, args, a0, a1, a2, map_b[0], map_b[1], map_b[2], map_b[3], sa, cols); break;
+        case kGemmResid: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmResid>, args, a0, a1, a2, map_b[0], map_b[1], map_b[2], map_b[3], sa, cols); break;
+        case kGemmSwiGLU: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmSwiGLU>, args, a0, a1, a2, map_b[0], map_b[1], map_b[2], map_b[3], sa, cols); break;
+        case kGemmLmHead: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmLmHead>, args, a0, a1, a2, map_b[0], map_b[1], map_b[2], map_b[3], sa, cols); break;
+        default: cudaLaunchKernelEx(&cfg, gemm_wide_kernel<kGemmStore>, args, a0, a1, a2, map_b[0], map_b[1], map_b[2], map_b[3], sa, cols); break;
     }
 }
 
