@@ -51,7 +51,6 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         while (i < 3 && wide_box_rows(g.nr, i) < rows_used) ++i;
         return i;
     };
-    const int SB = SA;                                   // one ring: S stages
     const uint32_t sA = base, sB = base + kGemmABytes;   // stage s: sA + s * stage_bytes, sB + s * stage_bytes
     uint8_t* after = gen_base + (size_t)SA * stage_bytes;
     float (*stage)[33] = reinterpret_cast<float (*)[33]>(after);
@@ -105,57 +104,63 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
     const uint32_t tmem_base = sh[0];
 
     // One thread gets a TMA copy under way about every 0.5 us, whatever the copy's size (measured: 16 KB boxes from one
-    // thread stream 31 GB/s per CTA, from two threads 59, from four 95, L2-resident).  A work item needs three copies
-    // (a weight tile and the two terms of the activation tile), so the copies are dealt over several issuing threads.
-    // (the ring depths are multiples of the lane counts: see gemm_wide_cfg)
-    const int kPA = SA >= 4 ? 2 : 1;    // issuing lanes of the weight producer warp (SA is even from four stages on)
-    const int kPB = kPA;                // issuing lanes of the activation producer warp
+    // thread stream 31 GB/s per CTA, from two threads 59, from four 95, L2-resident), so each half of a stage is
+    // filled by two lanes in turn where the ring has four stages or more (its depth is then even: see gemm_wide_cfg).
+    // Stage, parity, tile and chunk of a lane's next item are kept as running counters: divisions by run-time
+    // values would cost these threads as much as the copies.
+    const int kP = SA >= 4 ? 2 : 1;
     if (warp == 4) {
-        // ------------------------------- weight producers (lane p takes items p, p + kPA, ...) -----------------
-        if (lane < kPA) {
+        // ------------------------------- weight producers (lane p takes items p, p + kP, ...) ------------------
+        if (lane < kP) {
             int64_t it = lane;
-            for (; it < n_items && !sh[1]; it += kPA) {
-                const int64_t w = w_beg + it;
-                const int s = (int)(it % SA);
-                const uint32_t ph = (uint32_t)((it / SA) & 1);
+            int tile = (int)((w_beg + lane) / C), c = (int)((w_beg + lane) - (int64_t)tile * C);
+            int m = tile / g.tiles_per_map, rt = tile - m * g.tiles_per_map;  // matrix and tile inside it
+            int s = lane;       // lane < kP <= SA
+            uint32_t ph = 0;
+            for (; it < n_items && !sh[1]; it += kP) {
                 if (it >= SA && !mbar_wait(empty_a(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_a(s), kGemmABytes);
-                const int tile = (int)(w / C), c = (int)(w - (int64_t)tile * C);
                 const uint32_t dstA = sA + (uint32_t)s * stage_bytes;
                 if (MODE == kGemmSwiGLU) {
                     tma_load_2d(dstA, &map_a0, full_a(s), c * 64, tile * 64);
                     tma_load_2d(dstA + kGemmABytes / 2, &map_a1, full_a(s), c * 64, tile * 64);
                 } else {
-                    const int m = tile / g.tiles_per_map, r0 = (tile % g.tiles_per_map) * 128;
                     const CUtensorMap* mp = m == 0 ? &map_a0 : (m == 1 ? &map_a1 : &map_a2);
-                    tma_load_2d(dstA, mp, full_a(s), c * 64, r0);
+                    tma_load_2d(dstA, mp, full_a(s), c * 64, rt * 128);
                 }
+                c += kP;
+                while (c >= C) { c -= C; ++tile; if (++rt == g.tiles_per_map) { rt = 0; ++m; } }
+                s += kP;
+                if (s >= SA) { s -= SA; ph ^= 1u; }
             }
             if (sh[1]) {  // give up: let this lane's copies already issued land before the CTA's memory goes away
-                for (int64_t j = it - kPA; j >= 0 && j > it - kPA * (SA + 1); j -= kPA)
+                for (int64_t j = it - kP; j >= 0 && j > it - kP * (SA + 1); j -= kP)
                     (void)mbar_wait(full_a((int)(j % SA)), (uint32_t)((j / SA) & 1), 100000000ull);
             }
         }
     } else if (warp == 6) {
-        // ------------------------------- activation producers (lane p takes items p, p + kPB, ...) -------------
-        if (lane < kPB) {
+        // ------------------------------- activation producers (lane p takes items p, p + kP, ...) --------------
+        if (lane < kP) {
             grid_dependency_wait();  // activations are written by the kernel before this one
             const int bi = box_index(g.rows ? min(__ldcg(&g.rows->rows_used), g.nr) : g.nr);
             const CUtensorMap* map_b = bi == 0 ? &map_b0 : (bi == 1 ? &map_b1 : (bi == 2 ? &map_b2 : &map_b3));
             const uint32_t b_slot = (uint32_t)wide_box_rows(g.nr, bi) * 256u;  // hi rows, then lo rows, of one k-chunk
             int64_t q = lane;
-            for (; q < n_items && !sh[1]; q += kPB) {
-                const int64_t w = w_beg + q;
-                const int c = (int)(w % C);
-                const int s = (int)(q % SB);
-                const uint32_t ph = (uint32_t)((q / SB) & 1);
-                if (q >= SB && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+            int c = (int)((w_beg + lane) % C);
+            int s = lane;
+            uint32_t ph = 0;
+            for (; q < n_items && !sh[1]; q += kP) {
+                if (q >= SA && !mbar_wait(empty_b(s), ph ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 mbar_arrive_expect_tx(full_b(s), b_slot);
                 tma_load_3d(sB + (uint32_t)s * stage_bytes, map_b, full_b(s), c * 64, 0, 0);
+                c += kP;
+                while (c >= C) c -= C;
+                s += kP;
+                if (s >= SA) { s -= SA; ph ^= 1u; }
             }
             if (sh[1]) {
-                for (int64_t j = q - kPB; j >= 0 && j > q - kPB * (SB + 1); j -= kPB)
-                    (void)mbar_wait(full_b((int)(j % SB)), (uint32_t)((j / SB) & 1), 100000000ull);
+                for (int64_t j = q - kP; j >= 0 && j > q - kP * (SA + 1); j -= kP)
+                    (void)mbar_wait(full_b((int)(j % SA)), (uint32_t)((j / SA) & 1), 100000000ull);
             }
         }
     } else if (warp == 5) {
@@ -176,6 +181,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             const bool one_mma = 2 * nr <= 256;
             const uint32_t idesc = idesc_bf16_m128(one_mma ? (uint32_t)(2 * nr) : (uint32_t)((rows_used + 15) & ~15));
             int64_t ia = 0;
+            int s = 0;            // ring stage of item ia and the parity of its use: kept by hand, a division by the
+            uint32_t s_ph = 0;    // run-time ring depth would cost this thread more than a commit
             int seg = 0;
 #ifdef LLMA_STAMPS
             // measurement build: time this thread spends waiting for weight stages (word 6) and for activation
@@ -190,15 +197,14 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             for (int64_t w = w_beg; w < w_end && !sh[1]; ++seg) {
                 const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
                 const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
-                const int buf = seg % n_acc;
-                const uint32_t use = (uint32_t)(seg / n_acc);
+                const int buf = n_acc == 2 ? (seg & 1) : 0;
+                const uint32_t use = (uint32_t)(n_acc == 2 ? seg >> 1 : seg);
                 if (!mbar_wait(acce_bar(buf), (use & 1u) ^ 1u)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * (uint32_t)acc_cols;
                 for (int c = c0; c < c1 && !sh[1]; ++c, ++ia) {
-                    const int s = (int)(ia % SA);
                     LLMA_WAIT_BEGIN();
-                    if (!mbar_wait(full_a(s), (uint32_t)((ia / SA) & 1))) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
+                    if (!mbar_wait(full_a(s), s_ph)) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; break; }
                     LLMA_WAIT_END(wait_a);
                     if (ia == 0) LLMA_STAMP(stp, 2);
                     tc_fence_after();
@@ -212,6 +218,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                         if (!one_mma) umma_bf16(d_tmem + (uint32_t)nr, da + 2 * kk, db_lo + 2 * kk, idesc, (acc_on || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(empty_a(s));  // the stage is free once these MMAs have read it
+                    if (++s == SA) { s = 0; s_ph ^= 1u; }
                 }
                 if (sh[1]) break;
                 umma_commit(accf_bar(buf));  // accumulator complete
@@ -290,8 +297,8 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
             const int tile = (int)(w / C), c0 = (int)(w - (int64_t)tile * C);
             const int c1 = (int)min((int64_t)C, c0 + (w_end - w));
             w += c1 - c0;
-            const int buf = seg % n_acc;
-            const uint32_t use = (uint32_t)(seg / n_acc);
+            const int buf = n_acc == 2 ? (seg & 1) : 0;
+            const uint32_t use = (uint32_t)(n_acc == 2 ? seg >> 1 : seg);
             if (threadIdx.x == 0) {
                 bool ok = !sh[1] && mbar_wait(accf_bar(buf), use & 1u);
                 if (!ok) { atomicExch(g.dev_err, kDevErrTimeout); sh[1] = 1; }
