@@ -342,6 +342,9 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
     // Slots past the row's last chunk hold older (finite) values; they are read but never used.
     const int rows_used = __ldcg(&a.rows->rows_used);
     const int pos = __ldcg(&a.rows->pos[r]);
+    // a step shaped for many rows (batched decoding) usually uses a fraction of its row slots: there a warp first
+    // learns whether its slot is in use, at the price of one more round trip for those that are
+    if (a.n_rows > 32 && (r >= rows_used || pos < 0)) return;
     const float4* src = reinterpret_cast<const float4*>(a.ws_o + (head_base + r) * HD) + (lane < HD / 4 ? lane : 0);
     float2 ml[2];
 #pragma unroll

@@ -72,7 +72,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         at.n_rows = e->cur_rows;
         at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml;
         at.dev_err = e->dev_err;
-        at.stamps = e->cur_wide ? nullptr : e->stamps;
+        at.stamps = e->stamps;
         at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0;  // prompt passes: the device-side length is stale
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
