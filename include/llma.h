@@ -273,6 +273,18 @@ typedef struct {
 int llma_profile_steps(llma_engine *e, int32_t n, int32_t k, int32_t steps, llma_profile *out);
 
 /*
+ * Measurement aid (no counterpart in the paper): the time one tcgen05.mma of the projection kernels' shape
+ * (M 128, K 16, bf16 inputs, fp32 accumulator) occupies the tensor core, measured on the current device by one
+ * CTA that issues 4 * groups MMAs of width n on operands resident in shared memory, dealt over `regions`
+ * accumulator regions of n TMEM columns each, with commits_per_group tcgen05.commit between groups of four.
+ * ns_per_mma (host pointer) receives the wall time from the first issue to the completion of the last MMA,
+ * divided by the number of MMAs.  Allocates and frees two words of device memory; synchronises the device.
+ * Errors: NULL; ARG (n not a multiple of 16 in [16, 256], regions * n > 512, groups outside [1, 65536],
+ * commits_per_group outside [0, 4]); CONFIG (not an sm_100 device); CUDA; DEVICE_TIMEOUT.
+ */
+int llma_microbench_mma(int32_t n, int32_t regions, int32_t groups, int32_t commits_per_group, double *ns_per_mma);
+
+/*
  * The engine's projection kernel on its own: out[r, n] = sum_k W[n, k] * a[r, k] for the 32
  * activation rows a step can hold (Eq. 3 evaluates k+1 <= 32 positions against every weight
  * matrix in one pass).  W: device, bf16, row-major [n_out, k_in]; a: device, bf16, row-major

@@ -13,5 +13,6 @@ from .binding import (  # noqa: F401
     lib,
     llma_gemm_rows32_bf16,
     llma_gemm_rows32_bf16_noalloc,
+    llma_microbench_mma,
     LIB_PATH,
 )

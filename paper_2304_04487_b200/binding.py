@@ -56,7 +56,7 @@ _lib = None
 
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_set_adaptive_k", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
-           "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16",
+           "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_microbench_mma",
            "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity", "llma_debug_timeline",
            "llma_last_cuda_error", "llma_strerror")
 
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
         L.llma_step.argtypes = [vp, i32, i32, pi32, pi32]
         L.llma_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(LlmaStats)]
         L.llma_rewind.argtypes = [vp, i32]
+        L.llma_microbench_mma.argtypes = [i32, i32, i32, i32, C.POINTER(C.c_double)]
         L.llma_set_adaptive_k.argtypes = [vp, i32, i32, i32]
         L.llma_reset.argtypes = [vp, i32]
         L.llma_last_step_info.argtypes = [vp, C.POINTER(LlmaStepInfo)]
@@ -136,6 +137,15 @@ def llma_gemm_rows32_bf16_noalloc(W, a, out, stream=None) -> None:
     rc = lib().llma_gemm_rows32_bf16_noalloc(W.data_ptr(), a.data_ptr(), out.data_ptr(), n_out, k_in, st.cuda_stream)
     if rc != 0:
         raise LlmaError(rc, "llma_gemm_rows32_bf16_noalloc")
+
+
+def llma_microbench_mma(n: int, regions: int = 1, groups: int = 512, commits_per_group: int = 0) -> float:
+    """Nanoseconds one M128 x n x K16 bf16 tcgen05.mma occupies the tensor core (see include/llma.h)."""
+    ns = C.c_double(0.0)
+    rc = lib().llma_microbench_mma(n, regions, groups, commits_per_group, C.byref(ns))
+    if rc != 0:
+        raise LlmaError(rc, "llma_microbench_mma")
+    return float(ns.value)
 
 
 class Engine:

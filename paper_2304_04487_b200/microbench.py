@@ -1,6 +1,7 @@
 """Micro-benchmark of the projection GEMM on its own (weight streaming at 32 activation rows).
 
     python -m paper_2304_04487_b200.microbench --n-out 22016 --k-in 4096 --iters 40
+    python -m paper_2304_04487_b200.microbench --mma      # tensor-core time per MMA against N, regions, commits
 
 Cycles through several weight buffers so that every launch streams its matrix from HBM
 (one matrix may fit in the 126 MB L2), times the launches with CUDA events on the launching
@@ -20,7 +21,21 @@ def main():
     ap.add_argument("--k-in", type=int, default=4096)
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--buffers", type=int, default=4)
+    ap.add_argument("--mma", action="store_true")
     a = ap.parse_args()
+    if a.mma:
+        from . import llma_microbench_mma
+        rows = []
+        for n in (16, 32, 64, 96, 128, 144, 192, 256):
+            for regions in (1, 2):
+                if regions * n <= 512:
+                    rows.append({"n": n, "regions": regions, "commits_per_group": 0,
+                                 "ns_per_mma": round(llma_microbench_mma(n, regions, 512, 0), 1)})
+        for commits in (1, 2):
+            rows.append({"n": 32, "regions": 1, "commits_per_group": commits,
+                         "ns_per_mma": round(llma_microbench_mma(32, 1, 512, commits), 1)})
+        print(json.dumps({"mma_m128_k16_bf16": rows}))
+        return
     torch.manual_seed(0)
     Ws = [(torch.randn(a.n_out, a.k_in, device="cuda") * 0.02).to(torch.bfloat16) for _ in range(a.buffers)]
     act = torch.randn(32, a.k_in, device="cuda").to(torch.bfloat16)

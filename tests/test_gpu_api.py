@@ -102,3 +102,14 @@ def test_edge_cases(setup):
     e2.llma_set_reference(0, g[:20])
     (t,), st = e2.llma_generate(20, 1, 8)
     assert t == g[:first + 1]
+
+
+def test_microbench_mma_runs_and_rejects_bad_arguments():
+    """The tensor-core timing probe: a plausible figure for a legal shape, LLMA_ERR_ARG for the rest."""
+    from paper_2304_04487_b200 import LlmaError, llma_microbench_mma
+    t32 = llma_microbench_mma(32, 1, 256, 0)
+    t256 = llma_microbench_mma(256, 2, 256, 1)
+    assert 10.0 < t32 < 1000.0 and 10.0 < t256 < 1000.0, (t32, t256)
+    for bad in ((24, 1, 256, 0), (272, 1, 256, 0), (256, 3, 256, 0), (32, 1, 0, 0), (32, 1, 256, 5), (0, 1, 1, 0)):
+        with pytest.raises(LlmaError):
+            llma_microbench_mma(*bad)
