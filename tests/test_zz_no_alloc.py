@@ -47,6 +47,25 @@ def test_noalloc_matches_allocating_entry_point_twice():
     assert free_after == free_before
 
 
+def test_noalloc_matches_oracle_directly():
+    """The same entry point against the CPU oracle's matrix-vector product, with no other entry point in between."""
+    import torch
+    from oracle import model as OM
+    from workloads import bf16_bits_from_f32, f32_from_bf16_bits
+    from paper_2304_04487_b200 import llma_gemm_rows32_bf16_noalloc
+    rng = np.random.default_rng(7)
+    for n_out, k_in in ((200, 256), (512, 2816)):
+        W = bf16_bits_from_f32((rng.standard_normal((n_out, k_in)) * 0.05).astype(np.float32))
+        a = bf16_bits_from_f32(rng.standard_normal((32, k_in)).astype(np.float32))
+        dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+        out = torch.full((32, n_out), float("nan"), device="cuda")
+        llma_gemm_rows32_bf16_noalloc(dev(W), dev(a), out)
+        got, af = out.cpu().numpy(), f32_from_bf16_bits(a)
+        for r in (0, 5, 31):
+            want = OM.matvec(W, af[r])
+            assert np.abs(got[r] - want).max() <= 1e-4 * max(1.0, np.abs(want).max()), (n_out, k_in, r)
+
+
 def test_noalloc_rejects_sizes_beyond_its_scratch():
     import torch
     from paper_2304_04487_b200 import lib
