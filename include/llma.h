@@ -312,12 +312,11 @@ int llma_gemm_rows32_bf16(const void *W, const void *a, float *out, int32_t n_ou
  * n_out <= 262144 and k_in <= 16384; larger sizes return LLMA_ERR_CAPACITY and do nothing.
  *
  * The first call on a device resolves the array's device address (with the caller's current
- * device) and opts the kernel into its shared-memory size; make that first call before any
- * stream capture is begun.  All calls on a device share the array and it keeps the previous
- * call's contents: the call itself puts the hand-over slots into their empty state and clears the
- * error word, but two calls that
- * overlap on the GPU (different streams, or different threads) race on it and give wrong
- * results -- serialise them.  Synchronous.
+ * device) and opts the kernel into its shared-memory size.  All calls on a device share the array
+ * and it keeps the previous call's contents: the call itself puts the hand-over slots into their
+ * empty state and clears the error word, but two calls that overlap on the GPU (different streams,
+ * or different threads) race on it and give wrong results -- serialise them.  The call is
+ * synchronous: it waits for the kernel and reads its error word back before it returns.
  * Errors: NULL, ARG, CAPACITY, CONFIG (not an sm_100 device), CUDA, DEVICE_TIMEOUT.
  */
 int llma_gemm_rows32_bf16_noalloc(const void *W, const void *a, float *out, int32_t n_out, int32_t k_in,
