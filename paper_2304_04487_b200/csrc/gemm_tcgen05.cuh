@@ -94,7 +94,7 @@ template <int NR> struct GemmCfg {
     static constexpr uint32_t kABytes = kGemmKC * kGemmABytes;
     static constexpr uint32_t kBTile = 2 * NR * 64 * 2;   // activation rows (hi, lo) of one k-chunk
     static constexpr uint32_t kBBytes = kGemmKC * kBTile;
-    static constexpr int kStages = NR == 16 ? 4 : 3;
+    static constexpr int kStages = 4;  // at 32 rows this fills the 227 KB of shared memory to the byte
     static constexpr size_t kRopeBytes = 32 * 64 * 8;  // (cos, sin) of every row's position, 64 rotary pairs
     static constexpr size_t kUsedBytes = 1024 + (size_t)kStages * (kABytes + kBBytes) + 128 * 33 * 4 + 1536 + kRopeBytes;
     static constexpr size_t kSmemBytes = kUsedBytes > 120 * 1024 ? kUsedBytes : 120 * 1024;
