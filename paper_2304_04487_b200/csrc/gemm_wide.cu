@@ -11,13 +11,16 @@
 //     over several accumulators) and a commit costs the issuing thread another 45 ns, so the number of MMAs and
 //     commits per weight tile is what bounds the kernel: 4 + 1 up to 128 rows (0.37 us per 16 KB, the HBM rate),
 //     8 + 1 beyond;
-//   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows.
+//   * the rows a copy brings (nr: 32, 64, 128 or the launch's capacity) are chosen per step from the rows in use;
+//   * the epilogue walks a finished 128 x nr accumulator in blocks of 32 rows; tiles cut by a range boundary
+//     are summed and finished block by block by all the CTAs that share them.
 //
 // Roles inside one CTA of 224 threads:
-//   warps 0-3  epilogue: TMEM -> registers -> (cross-CTA fix-up) -> fused epilogue, block by block
-//   warp  4    one thread issues the TMA loads of the weight tiles (they depend on no earlier kernel)
+//   warps 0-3  epilogue: TMEM -> registers -> workspace (cut tiles) or fused epilogue, block by block; then the
+//              blocks of cut tiles dealt to this CTA
+//   warp  4    one or two lanes issue the TMA loads of the weight tiles (they depend on no earlier kernel)
 //   warp  5    MMA: allocates TMEM; one thread issues tcgen05.mma and the commits
-//   warp  6    one thread issues the TMA loads of the activation tiles (after the dependency wait)
+//   warp  6    one or two lanes issue the TMA loads of the activation tiles (after the dependency wait)
 //
 // Every wait is bounded: when one runs out the kernel raises the device error word, stops
 // issuing work, lets its outstanding copies land, frees TMEM and returns.
