@@ -365,11 +365,12 @@ def run_sweep13b(args, rank, local_rank, world, small=False):
     from paper_2304_04487_b200 import Engine
     shape = SHAPES["mid-bf16" if small else "llama13b-shape"]
     P, R, N = (200, 128, 64) if small else (2048, 1024, 256)
-    overlaps, ks = (0.2, 0.5, 0.8, 0.95), (4, 8, 16)
+    # k = 15 is the largest copy the 16-row kernel verifies (16 rows); k = 16 needs the 32-row engine
+    overlaps, ks = (0.2, 0.5, 0.8, 0.95), (4, 8, 15, 16)
     w = make_weights(shape, seed=0)
     prompt = make_prompt(P, shape.vocab, seed=1)
     max_seq = P + N + 32
-    eng8 = Engine(shape, w, max_seq=max_seq, max_ref=R, max_k=8, device=f"cuda:{local_rank}")
+    eng8 = Engine(shape, w, max_seq=max_seq, max_ref=R, max_k=15, device=f"cuda:{local_rank}")   # 16 rows
     eng16 = Engine(shape, None, max_seq=max_seq, max_ref=R, max_k=16, device=f"cuda:{local_rank}", share_weights_with=eng8)
     t0 = time.perf_counter()
     eng8.llma_prefill(0, prompt)
@@ -392,7 +393,7 @@ def run_sweep13b(args, rank, local_rank, world, small=False):
     for f in overlaps:
         ref, offs, info = build_reference(y_star, [R], f, shape.vocab, seed=0)
         for k in ks:
-            eng, gname = (eng8, "16rows") if k <= 8 else (eng16, "32rows")
+            eng, gname = (eng8, "16rows") if k <= 15 else (eng16, "32rows")
             eng.llma_set_reference(0, ref, offs)
             ms, st = [], None
             for it in range(args.warmup + args.steps):
@@ -670,6 +671,15 @@ def main():
         eng.llma_rewind(0)
         _, st = eng.llma_generate(n_new, 1, kk)
         lat[str(kk)] = {"ms_per_step": st.device_ms / st.steps, "tokens_per_step": st.tokens / st.steps}
+    if k < 15:  # the largest copy the 16-row kernel verifies: an engine of its own (same kernels, 16 rows)
+        eng15 = Engine(shape, None, max_seq=max_seq, max_ref=sum(docs), max_k=15, device=f"cuda:{local_rank}",
+                       share_weights_with=eng)
+        eng15.llma_prefill(0, prompt)
+        eng15.llma_set_reference(0, y_star, None)
+        eng15.llma_rewind(0)
+        _, st = eng15.llma_generate(n_new, 1, 15)
+        lat["15"] = {"ms_per_step": st.device_ms / st.steps, "tokens_per_step": st.tokens / st.steps}
+        eng15.llma_destroy()
     eng16 = Engine(shape, None, max_seq=max_seq, max_ref=sum(docs), max_k=16, device=f"cuda:{local_rank}",
                    share_weights_with=eng)
     eng16.llma_prefill(0, prompt)
