@@ -177,6 +177,67 @@ __device__ __forceinline__ void epilogue_qkv_wide(const GemmArgs& g, int tile, i
     epi_sync();
 }
 
+// Row-major variant for the wide kernel: thread t takes activation row j = t & 31 of the block and the 16 rotary
+// pairs 16 (t >> 5) .. + 15 of the tile, i.e. two runs of 16 consecutive features.  The rotary factors of a row are
+// then 64 contiguous bytes per table and the results leave as 16-byte stores; nothing in a thread's work depends
+// on another load, so the whole block is one round trip instead of one per row.  Same arithmetic per element as
+// epilogue_qkv.  Requires head_dim = 64 or 128 (a tile of 128 features holds whole heads).
+__device__ __forceinline__ void epilogue_qkv_rows(const GemmArgs& g, int tile, int t, int jb, int nj,
+                                                  float (*stage)[33], const int* row_pos, const int* row_seq) {
+    const ModelDims& d = g.dims;
+    const int mat = tile / g.tiles_per_map;
+    const int col0 = (tile % g.tiles_per_map) * 128;
+    const int hd = d.head_dim, half = hd >> 1;
+    const int j = t & 31, p0 = (t >> 5) * 16;            // row of the block, first rotary pair
+    const int f_lo = (p0 / half) * hd + (p0 % half);     // feature of the pair's lower element inside the tile
+    const int f_hi = f_lo + half;
+    const int fi0 = p0 % half;
+    const int pos = j < nj ? row_pos[jb + j] : -1;
+    if (pos >= 0) {
+        float lo[16], hi[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { lo[i] = stage[f_lo + i][j]; hi[i] = stage[f_hi + i][j]; }
+        if (mat < 2) {
+            float4 c4[4], s4[4];
+            const float4* cp = reinterpret_cast<const float4*>(g.rope_cos + (int64_t)pos * half + fi0);
+            const float4* sp = reinterpret_cast<const float4*>(g.rope_sin + (int64_t)pos * half + fi0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { c4[u] = __ldg(cp + u); s4[u] = __ldg(sp + u); }
+            const float* c = reinterpret_cast<const float*>(c4);
+            const float* sn = reinterpret_cast<const float*>(s4);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float a = lo[i], b = hi[i];
+                lo[i] = a * c[i] - b * sn[i];
+                hi[i] = a * sn[i] + b * c[i];
+            }
+        }
+        if (mat == 0) {
+            float* o = g.out_f32 + (int64_t)(jb + j) * g.ld + col0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                *reinterpret_cast<float4*>(o + f_lo + 4 * u) = make_float4(lo[4 * u], lo[4 * u + 1], lo[4 * u + 2], lo[4 * u + 3]);
+                *reinterpret_cast<float4*>(o + f_hi + 4 * u) = make_float4(hi[4 * u], hi[4 * u + 1], hi[4 * u + 2], hi[4 * u + 3]);
+            }
+        } else {
+            __nv_bfloat16* cache = mat == 1 ? g.kcache : g.vcache;
+            const int head = (col0 + f_lo) / hd, idx = (col0 + f_lo) % hd;
+            __nv_bfloat16* dst = cache + (kv_row_index(d, g.layer, row_seq[jb + j], head, pos) * hd + idx);
+            auto pack = [](float x, float y) {
+                return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(y)) << 16);
+            };
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                *reinterpret_cast<uint4*>(dst + 8 * u) = make_uint4(pack(lo[8 * u], lo[8 * u + 1]), pack(lo[8 * u + 2], lo[8 * u + 3]),
+                                                                     pack(lo[8 * u + 4], lo[8 * u + 5]), pack(lo[8 * u + 6], lo[8 * u + 7]));
+                *reinterpret_cast<uint4*>(dst + half + 8 * u) = make_uint4(pack(hi[8 * u], hi[8 * u + 1]), pack(hi[8 * u + 2], hi[8 * u + 3]),
+                                                                            pack(hi[8 * u + 4], hi[8 * u + 5]), pack(hi[8 * u + 6], hi[8 * u + 7]));
+            }
+        }
+    }
+    epi_sync();
+}
+
 // SwiGLU: tile rows 0..63 are gate features, 64..127 the matching up features.
 __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33]) {

@@ -276,7 +276,10 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 for (int j = 0; j < 32; ++j) stage[row][j] = acc[j];
             }
             epi_sync();
-            if constexpr (MODE == kGemmQKV) epilogue_qkv_wide(g, tile, row, jb, nj, stage, s_pos, s_seq);
+            if constexpr (MODE == kGemmQKV) {
+                if (g.dims.head_dim == 128 || g.dims.head_dim == 64) epilogue_qkv_rows(g, tile, row, jb, nj, stage, s_pos, s_seq);
+                else epilogue_qkv_wide(g, tile, row, jb, nj, stage, s_pos, s_seq);
+            }
             else if constexpr (MODE == kGemmResid) epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
             else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, jb, nj, stage);
             else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, jb, nj, stage);
