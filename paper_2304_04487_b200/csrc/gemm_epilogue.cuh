@@ -252,6 +252,99 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, int tile, int
     epi_sync();
 }
 
+// Row-major variants for the wide kernel (see epilogue_qkv_rows): thread t takes activation row j = t & 31 of
+// the block and a run of consecutive features chosen by t >> 5, so that the residual stream, the split operand and
+// the gains move as 16-byte accesses and nothing waits for an earlier load of the same thread.
+__device__ __forceinline__ uint32_t pack_bf16x2(float x, float y) {
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(y)) << 16);
+}
+// hi = bf16(v), lo = bf16(v - hi) of 8 values, as the two 16-byte words of the split layout
+__device__ __forceinline__ void split8(const float (&v)[8], uint4& hi, uint4& lo) {
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 a = __float2bfloat16_rn(v[2 * i]), b = __float2bfloat16_rn(v[2 * i + 1]);
+        h[i] = (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+        l[i] = pack_bf16x2(v[2 * i] - __bfloat162float(a), v[2 * i + 1] - __bfloat162float(b));
+    }
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+// x[r, n] += acc for 32 features per thread; requires n_out % 128 == 0.  The sum of squares of a row is taken
+// over ascending features: 32 per thread, then the four threads of the row in ascending order.
+__device__ __forceinline__ void epilogue_resid_rows(const GemmArgs& g, int tile, int t, int jb, int nj,
+                                                    float (*stage)[33], float* red_f) {
+    const int j = t & 31, w = t >> 5, f0 = 32 * w;
+    const int col0 = tile * 128 + f0;
+    const bool fold = g.xs_out != nullptr;
+    float sq = 0.f;
+    if (j < nj) {
+        float* xrow = g.out_f32 + (int64_t)(jb + j) * g.ld + col0;
+        float4 x4[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x4[u] = __ldcg(reinterpret_cast<const float4*>(xrow) + u);
+        float xn[32];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            xn[4 * u] = stage[f0 + 4 * u][j] + x4[u].x; xn[4 * u + 1] = stage[f0 + 4 * u + 1][j] + x4[u].y;
+            xn[4 * u + 2] = stage[f0 + 4 * u + 2][j] + x4[u].z; xn[4 * u + 3] = stage[f0 + 4 * u + 3][j] + x4[u].w;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            reinterpret_cast<float4*>(xrow)[u] = make_float4(xn[4 * u], xn[4 * u + 1], xn[4 * u + 2], xn[4 * u + 3]);
+        if (fold) {
+            __nv_bfloat16* hi_row = reinterpret_cast<__nv_bfloat16*>(g.xs_out) + (int64_t)(jb + j) * g.n_out + col0;
+            __nv_bfloat16* lo_row = hi_row + (int64_t)g.rc * g.n_out;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float4 ga = __ldg(reinterpret_cast<const float4*>(g.gain_next + col0) + 2 * u);
+                const float4 gb = __ldg(reinterpret_cast<const float4*>(g.gain_next + col0) + 2 * u + 1);
+                const float v[8] = {xn[8 * u] * ga.x, xn[8 * u + 1] * ga.y, xn[8 * u + 2] * ga.z, xn[8 * u + 3] * ga.w,
+                                    xn[8 * u + 4] * gb.x, xn[8 * u + 5] * gb.y, xn[8 * u + 6] * gb.z, xn[8 * u + 7] * gb.w};
+                uint4 hi, lo;
+                split8(v, hi, lo);
+                reinterpret_cast<uint4*>(hi_row)[u] = hi;
+                reinterpret_cast<uint4*>(lo_row)[u] = lo;
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sq = __fmaf_rn(xn[i], xn[i], sq);
+        }
+    }
+    if (!fold) { epi_sync(); return; }
+    red_f[w * 32 + j] = sq;
+    epi_sync();
+    if (w == 0 && j < nj)
+        g.ss_out[(int64_t)tile * g.rc + jb + j] = ((red_f[j] + red_f[32 + j]) + red_f[64 + j]) + red_f[96 + j];
+    epi_sync();
+}
+
+// h = silu(gate) * up for 16 features per thread; requires n_out % 16 == 0
+__device__ __forceinline__ void epilogue_swiglu_rows(const GemmArgs& g, int tile, int t, int jb, int nj,
+                                                     float (*stage)[33]) {
+    const int j = t & 31, f0 = 16 * (t >> 5);
+    const int f = tile * 64 + f0;
+    if (j < nj && f < g.n_out) {
+        const int gb = g.gate_second ? 64 : 0, ub = g.gate_second ? 0 : 64;
+        __nv_bfloat16* hi_row = reinterpret_cast<__nv_bfloat16*>(g.out_act) + (int64_t)(jb + j) * g.n_out + f;
+        __nv_bfloat16* lo_row = hi_row + (int64_t)g.rc * g.n_out;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float gate = stage[gb + f0 + 8 * u + i][j], up = stage[ub + f0 + 8 * u + i][j];
+                v[i] = gate / (1.f + expf(-gate)) * up;
+            }
+            uint4 hi, lo;
+            split8(v, hi, lo);
+            reinterpret_cast<uint4*>(hi_row)[u] = hi;
+            reinterpret_cast<uint4*>(lo_row)[u] = lo;
+        }
+    }
+    epi_sync();
+}
+
 // LM head: optional logits store, then the tile's (max, lowest argmax) for every used row.
 __device__ __forceinline__ void epilogue_lmhead(const GemmArgs& g, int tile, int row, int jb, int nj,
                                                 float (*stage)[33], float* red_f, int* red_i) {

@@ -280,8 +280,13 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 if (g.dims.head_dim == 128 || g.dims.head_dim == 64) epilogue_qkv_rows(g, tile, row, jb, nj, stage, s_pos, s_seq);
                 else epilogue_qkv_wide(g, tile, row, jb, nj, stage, s_pos, s_seq);
             }
-            else if constexpr (MODE == kGemmResid) epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
-            else if constexpr (MODE == kGemmSwiGLU) epilogue_swiglu(g, tile, row, jb, nj, stage);
+            else if constexpr (MODE == kGemmResid) {
+                if ((g.n_out & 127) == 0) epilogue_resid_rows(g, tile, row, jb, nj, stage, red_f);
+                else epilogue_resid<false>(g, tile, row, jb, nj, stage, red_f, xnone);
+            } else if constexpr (MODE == kGemmSwiGLU) {
+                if ((g.n_out & 15) == 0) epilogue_swiglu_rows(g, tile, row, jb, nj, stage);
+                else epilogue_swiglu(g, tile, row, jb, nj, stage);
+            }
             else if constexpr (MODE == kGemmStore) epilogue_store(g, tile, row, jb, nj, stage);
             else epilogue_lmhead(g, tile, row, jb, nj, stage, red_f, red_i);
             epi_sync();  // the staging area is rewritten by the next block
