@@ -51,7 +51,7 @@ struct AttnSmem {
     static constexpr uint32_t kBytes = offStat + 2 * 4 * 16 * 4 + 64 + kRowCap * 4 + 16;  // + row positions, barriers
 };
 
-template <int HD>
+template <int HD, bool kPrompt>
 __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v) {
     using L = AttnSmem<HD>;
@@ -144,6 +144,127 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     // chunk partials are indexed by the row's slot in the step: [head][chunk][row][HD]
     const int64_t part_base = ((int64_t)head * a.n_chunks + chunk) * d.row_cap + first;
 
+    if (kPrompt && n_mt >= 4) {
+        // Many rows of one sequence (prompt passes; an instance of its own, so that the decoding steps' instance keeps its registers): every warp takes whole 16-row query tiles (tile w, w + 4, ...) against
+        // all 128 positions of the chunk, 32 positions at a time with a running maximum and sum, so that nothing is
+        // combined across warps and no barrier separates the tiles.  A row's partial still depends on its position and
+        // on the chunk only.
+        const int mi = lane >> 3, t8 = lane & 7;
+        bool v_ready = false;
+        for (int mt = warp; mt < n_mt; mt += 4) {
+            load_q(mt);
+            const int r_lo = mt * 16 + g8, r_hi = r_lo + 8;
+            const int lim_lo = r_lo < cnt ? s_pos[r_lo] : -1;
+            const int lim_hi = r_hi < cnt ? s_pos[r_hi] : -1;
+            const int lim_tile = s_pos[min(cnt - 1, mt * 16 + 15)];  // highest position of the tile (positions ascend with the row)
+            float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+            float o[HD / 8][4];
+#pragma unroll
+            for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+#pragma unroll 1
+            for (int sb = 0; sb < 4; ++sb) {
+                const int wp0 = sb * 32;
+                if (c0 + wp0 > lim_tile) break;  // warp-uniform: the rest of the chunk lies beyond every row of the tile
+                float sc[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks) {
+                    const uint32_t (&ah)[4] = qh[ks];
+                    const uint32_t (&al)[4] = ql[ks];
+#pragma unroll
+                    for (int np = 0; np < 2; ++np) {
+                        const int row = wp0 + np * 16 + (mi >> 1) * 8 + t8;
+                        const int col = ks * 16 + (mi & 1) * 8;
+                        const uint32_t kaddr = base + L::offK + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                               ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                        uint32_t b[4];
+                        ldsm_x4(kaddr, b);
+                        mma_bf16(sc[2 * np], ah, b[0], b[1]);
+                        mma_bf16(sc[2 * np], al, b[0], b[1]);
+                        mma_bf16(sc[2 * np + 1], ah, b[2], b[3]);
+                        mma_bf16(sc[2 * np + 1], al, b[2], b[3]);
+                    }
+                }
+                float bm_lo = -INFINITY, bm_hi = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int p = c0 + wp0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                        const int lim = e < 2 ? lim_lo : lim_hi;
+                        const float v = p <= lim ? sc[nt][e] * scale : -INFINITY;
+                        sc[nt][e] = v;
+                        if (e < 2) bm_lo = fmaxf(bm_lo, v); else bm_hi = fmaxf(bm_hi, v);
+                    }
+                }
+                bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 1)); bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 2));
+                bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 1)); bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 2));
+                const float n_lo = fmaxf(m_lo, bm_lo), n_hi = fmaxf(m_hi, bm_hi);
+                const float ref_lo = n_lo == -INFINITY ? 0.f : n_lo, ref_hi = n_hi == -INFINITY ? 0.f : n_hi;
+                const float f_lo = m_lo == -INFINITY ? 0.f : expf(m_lo - ref_lo);  // what was gathered so far, on the new scale
+                const float f_hi = m_hi == -INFINITY ? 0.f : expf(m_hi - ref_hi);
+                float bl_lo = 0.f, bl_hi = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float pe = expf(sc[nt][e] - (e < 2 ? ref_lo : ref_hi));  // exp(-inf) = 0 for masked positions
+                        sc[nt][e] = pe;
+                        if (e < 2) bl_lo += pe; else bl_hi += pe;
+                    }
+                }
+                bl_lo += __shfl_xor_sync(0xffffffffu, bl_lo, 1); bl_lo += __shfl_xor_sync(0xffffffffu, bl_lo, 2);
+                bl_hi += __shfl_xor_sync(0xffffffffu, bl_hi, 1); bl_hi += __shfl_xor_sync(0xffffffffu, bl_hi, 2);
+                l_lo = __fmaf_rn(l_lo, f_lo, bl_lo); l_hi = __fmaf_rn(l_hi, f_hi, bl_hi);
+                m_lo = n_lo; m_hi = n_hi;
+#pragma unroll
+                for (int i = 0; i < HD / 8; ++i) { o[i][0] *= f_lo; o[i][1] *= f_lo; o[i][2] *= f_hi; o[i][3] *= f_hi; }
+                if (!v_ready) {  // the V tile, once per warp
+                    bool ok = true;
+                    if (lane == 0) ok = mbar_wait(bar_v, 0);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) { if (lane == 0) atomicExch(a.dev_err, kDevErrTimeout); return; }
+                    v_ready = true;
+                }
+#pragma unroll
+                for (int kp = 0; kp < 2; ++kp) {
+                    uint32_t ph[4], pl[4];
+                    split_pack(sc[2 * kp][0], sc[2 * kp][1], ph[0], pl[0]);
+                    split_pack(sc[2 * kp][2], sc[2 * kp][3], ph[1], pl[1]);
+                    split_pack(sc[2 * kp + 1][0], sc[2 * kp + 1][1], ph[2], pl[2]);
+                    split_pack(sc[2 * kp + 1][2], sc[2 * kp + 1][3], ph[3], pl[3]);
+#pragma unroll
+                    for (int nn = 0; nn < HD / 16; ++nn) {
+                        const int row = wp0 + kp * 16 + (mi & 1) * 8 + t8;
+                        const int col = nn * 16 + (mi >> 1) * 8;
+                        const uint32_t vaddr = base + L::offV + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                               ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                        uint32_t b[4];
+                        ldsm_x4_trans(vaddr, b);
+                        mma_bf16(o[2 * nn], ph, b[0], b[1]);
+                        mma_bf16(o[2 * nn], pl, b[0], b[1]);
+                        mma_bf16(o[2 * nn + 1], ph, b[2], b[3]);
+                        mma_bf16(o[2 * nn + 1], pl, b[2], b[3]);
+                    }
+                }
+            }
+            // the tile's partial of this chunk, straight from the fragments (rows past cnt are not written)
+#pragma unroll
+            for (int nt = 0; nt < HD / 8; ++nt) {
+                const int col = nt * 8 + 2 * t4;
+                if (r_lo < cnt) *reinterpret_cast<float2*>(a.ws_o + (part_base + r_lo) * HD + col) = make_float2(o[nt][0], o[nt][1]);
+                if (r_hi < cnt) *reinterpret_cast<float2*>(a.ws_o + (part_base + r_hi) * HD + col) = make_float2(o[nt][2], o[nt][3]);
+            }
+            if (t4 == 0) {
+                if (r_lo < cnt) { a.ws_ml[(part_base + r_lo) * 2] = m_lo; a.ws_ml[(part_base + r_lo) * 2 + 1] = l_lo; }
+                if (r_hi < cnt) { a.ws_ml[(part_base + r_hi) * 2] = m_hi; a.ws_ml[(part_base + r_hi) * 2 + 1] = l_hi; }
+            }
+        }
+        if (!v_ready && lane == 0) (void)mbar_wait(bar_v, 0);  // a copy in flight must land before the CTA's memory goes away
+        if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 6);
+        return;
+    }
     for (int mt = 0; mt < n_mt; ++mt) {
         if (mt > 0) load_q(mt);
         // ---------------- S = Q K^T over this warp's 32 positions ----------------------------
@@ -414,10 +535,16 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
 constexpr size_t kAttnPad = 0;  // extra shared memory per CTA (a knob for the number of CTAs per SM)
 
 cudaError_t init_attention_mma() {
-    cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(AttnSmem<128>::kBytes + 1024 + kAttnPad));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attention_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<128>::kBytes + 1024 + kAttnPad));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attention_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<64>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attention_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)(AttnSmem<64>::kBytes + 1024));
 }
 
@@ -426,10 +553,12 @@ void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap&
     dim3 mgrid(a.dims.n_heads, (a.n_rows + 3) / 4);
     const size_t msmem = (size_t)8 * a.n_chunks * sizeof(float);
     if (a.dims.head_dim == 128) {
-        launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128>, a, map_k, map_v);
+        if (a.prompt) launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128, true>, a, map_k, map_v);
+        else launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128, false>, a, map_k, map_v);
         launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<128>, a);
     } else {
-        launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64>, a, map_k, map_v);
+        if (a.prompt) launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64, true>, a, map_k, map_v);
+        else launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_mma_kernel<64, false>, a, map_k, map_v);
         launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<64>, a);
     }
 }

@@ -14,6 +14,7 @@ struct AttnArgs {
     int32_t n_chunks;        // grid.x = ceil(max_seq / 128); CTAs past a sequence's last position exit
     const RowDesc* rows;
     const SeqState* seq_state;  // decode steps: kv_len here is the length committed before this step
+    int32_t prompt;          // 1: a prompt pass (many rows of one sequence): the kernel instance with the per-warp query tiles
     int32_t early_kv;        // 1: chunks wholly below that length may be fetched before the predecessor has finished
     int32_t n_rows;          // row slots of this pass (grid of the merge kernel)
     const float* qkv;        // [rows][3*H*hd] fp32, q already rotated

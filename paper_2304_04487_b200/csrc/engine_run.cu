@@ -73,7 +73,7 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml;
         at.dev_err = e->dev_err;
         at.stamps = e->stamps;
-        at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0;  // prompt passes: the device-side length is stale
+        at.seq_state = e->seq_state; at.early_kv = lm_head ? 1 : 0; at.prompt = lm_head ? 0 : 1;  // prompt passes: the device-side length is stale
         launch_attention_mma(st, at, e->map_kcache, e->map_vcache);
         mark(e, LLMA_K_ATTN);
         GemmArgs o = gemm_args(e, kGemmResid, D, (D + 127) / 128, HD, (D + 127) / 128);
