@@ -129,7 +129,34 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
             for (int i = 0; i < 4; ++i) split_pack(x[ks][i].x, x[ks][i].y, qh[ks][i], ql[ks][i]);
         }
     };
-    load_q(0);
+    // The first tile's rows go through shared memory: the CTA fetches them as whole 16-byte accesses (a few per thread
+    // instead of 32 eight-byte loads per lane, which filled the load/store queues once a sequence had more than a
+    // row or two) into the buffer that later holds the merged tile, columns XOR-ed by (row & 3) * 8 so that the fragment
+    // reads of a half-warp (four rows) fall into different banks.  With one or two rows the direct loads are few and
+    // spare the barrier.
+    if (cnt <= 2) {
+        load_q(0);
+    } else {
+        float* sQ = sO;
+        const int64_t ldq = 3 * (int64_t)d.hd_total;
+        for (int idx = threadIdx.x; idx < 16 * (HD / 4); idx += blockDim.x) {
+            const int r = idx / (HD / 4), c4 = idx - r * (HD / 4);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r < cnt) v = __ldcg(reinterpret_cast<const float4*>(a.qkv + (first + r) * ldq + head * HD) + c4);
+            *reinterpret_cast<float4*>(sQ + r * HD + ((c4 * 4) ^ ((r & 3) << 3))) = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = (i & 1) ? g8 + 8 : g8;
+                const int col = ks * 16 + 2 * t4 + ((i >> 1) ? 8 : 0);
+                const float2 x = *reinterpret_cast<const float2*>(sQ + row * HD + (col ^ ((row & 3) << 3)));
+                split_pack(x.x, x.y, qh[ks][i], ql[ks][i]);
+            }
+        }
+    }
     if (threadIdx.x == 0) {
         const bool ok = mbar_wait(bar_u, 0);
         if (!ok) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
