@@ -232,6 +232,10 @@ int llma_debug_set_device_error(llma_engine *e, int32_t code);
  * Only a library built with -DLLMA_STAMPS records anything; otherwise LLMA_ERR_STATE.  Errors: NULL, STATE, CUDA. */
 int llma_debug_timeline(llma_engine *e, int32_t clear, unsigned long long *out);
 
+/* Inspection: how many 128-position tiles of the K/V cache one attention CTA takes in a decoding step of this engine
+ * (1, 2 or 4; chosen at llma_create from max_batch, max_seq and the head count alone).  Errors: NULL. */
+int llma_debug_attention_tiles(llma_engine *e);
+
 /* Rows the engine's activation buffers hold (the leading dimension of llma_debug_buffer), or a negative
  * status. */
 int llma_row_capacity(llma_engine *e);

@@ -57,7 +57,7 @@ _lib = None
 EXPORTS = ("llma_create", "llma_destroy", "llma_prefill", "llma_set_reference", "llma_step", "llma_generate",
            "llma_rewind", "llma_set_adaptive_k", "llma_reset", "llma_last_step_info", "llma_debug_logits", "llma_debug_kv_row",
            "llma_kv_len", "llma_debug_buffer", "llma_gemm_impl", "llma_profile_steps", "llma_gemm_rows32_bf16", "llma_microbench_mma",
-           "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity", "llma_debug_timeline",
+           "llma_gemm_rows32_bf16_noalloc", "llma_generate_forced", "llma_debug_set_device_error", "llma_row_capacity", "llma_debug_attention_tiles", "llma_debug_timeline",
            "llma_last_cuda_error", "llma_strerror")
 
 
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
         L.llma_kv_len.argtypes = [vp, i32]
         L.llma_gemm_impl.argtypes = [vp]
         L.llma_row_capacity.argtypes = [vp]
+        L.llma_debug_attention_tiles.argtypes = [vp]
         L.llma_debug_timeline.argtypes = [vp, i32, vp]
         L.llma_debug_set_device_error.argtypes = [vp, i32]
         L.llma_generate_forced.argtypes = [vp, i32, pi32, i32, pi32, i32, C.POINTER(LlmaStats)]
@@ -234,6 +235,9 @@ class Engine:
         st = LlmaStats()
         self._check(lib().llma_generate(self._h, max_new, n, k, _pi32(out), _pi32(cnt), C.byref(st)), "llma_generate")
         return [out[s, :cnt[s]].tolist() for s in range(self.max_batch)], st
+
+    def llma_debug_attention_tiles(self) -> int:
+        return int(lib().llma_debug_attention_tiles(self._h))
 
     def llma_rewind(self, seq: int) -> None:
         self._check(lib().llma_rewind(self._h, seq), "llma_rewind")

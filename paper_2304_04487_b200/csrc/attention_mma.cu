@@ -467,6 +467,257 @@ __global__ void __launch_bounds__(128, 3) attention_mma_kernel(const AttnArgs a,
     if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 6);
 }
 
+// Long contexts, many sequences: a CTA takes kT consecutive 128-position tiles of one (sequence, head) instead of one,
+// so that the chunk partials (and the merge pass over them) shrink by kT and the next tile's K and V are already on
+// their way while the current one is being multiplied.  Each warp keeps its 32-position slice's running maximum, sum
+// and output across the tiles; the four warps are combined once, at the end, exactly as in attention_mma_kernel.
+// For steps of at most 16 rows per sequence; which kT an engine uses depends on its capacity only (never on the step).
+template <int HD, int kT>
+__global__ void __launch_bounds__(128, 3) attention_long_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+                                                             const __grid_constant__ CUtensorMap map_v) {
+    using L = AttnSmem<HD>;
+    pdl_trigger();
+    const int chunk = blockIdx.x, head = blockIdx.y, seq = blockIdx.z;
+    [[maybe_unused]] unsigned long long* stp = LLMA_STAMP_PTR(a.stamps, 300 + a.layer, 0);
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const ModelDims& d = a.dims;
+    const int c0 = chunk * kAttnChunk * kT;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+    float* sO = reinterpret_cast<float*>(gbase + L::offO);
+    float* s_m = reinterpret_cast<float*>(gbase + L::offStat);   // [4][16]
+    float* s_l = s_m + 64;                                        // [4][16]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(s_l + 64);
+    volatile uint32_t* flag = reinterpret_cast<volatile uint32_t*>(bar + 2);
+    const uint32_t bar_u = smem_u32(bar), bar_v = bar_u + 8;  // K tile, V tile
+    int* s_pos = reinterpret_cast<int*>(const_cast<uint32_t*>(flag) + 2);
+
+    auto fetch_k = [&](int t) {  // one thread
+        const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0 + t * kAttnChunk);
+        mbar_arrive_expect_tx(bar_u, L::kTileBytes);
+        for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offK + b * L::kBoxBytes, &map_k, bar_u, b * 64, row0);
+    };
+    auto fetch_v = [&](int t) {
+        const int32_t row0 = (int32_t)kv_row_index(d, a.layer, seq, head, c0 + t * kAttnChunk);
+        mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+        for (int b = 0; b < L::kBoxes; ++b) tma_load_2d(base + L::offV + b * L::kBoxBytes, &map_v, bar_v, b * 64, row0);
+    };
+    // the first tile may be requested before the QKV projection has finished if it lies wholly below the committed length
+    const bool early = a.early_kv && c0 + kAttnChunk <= __ldcg(&a.seq_state[seq].kv_len);
+    if (threadIdx.x == 0) {
+        mbar_init(bar_u, 1); mbar_init(bar_v, 1); fence_mbar_init(); flag[0] = 0; flag[1] = 0;
+        if (early) { fetch_k(0); fetch_v(0); }
+    }
+    pdl_wait();
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 2);
+
+    const int first = __ldcg(&a.rows->seq_first[seq]), cnt = __ldcg(&a.rows->seq_cnt[seq]);
+    const int maxpos = __ldcg(&a.rows->seq_maxpos[seq]);
+    if (cnt == 0 || c0 > maxpos) {
+        if (early && threadIdx.x == 0) { (void)mbar_wait(bar_u, 0); (void)mbar_wait(bar_v, 0); }
+        return;
+    }
+    if (cnt > 16) {  // not this kernel's case: the host never launches it for such steps
+        if (threadIdx.x == 0) {
+            atomicExch(a.dev_err, kDevErrCapacity);
+            if (early) { (void)mbar_wait(bar_u, 0); (void)mbar_wait(bar_v, 0); }
+        }
+        return;
+    }
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) s_pos[i] = __ldcg(&a.rows->pos[first + i]);
+    __syncthreads();
+    if (!early && threadIdx.x == 0) { fetch_k(0); fetch_v(0); }
+    const int n_tiles = min(kT, (maxpos - c0) / kAttnChunk + 1);  // tiles that hold a position some row attends to
+
+    const int g8 = lane >> 2, t4 = lane & 3;
+    uint32_t qh[HD / 16][4], ql[HD / 16][4];
+    {   // the step's rows of q for this head through shared memory (see attention_mma_kernel)
+        float* sQ = sO;
+        const int64_t ldq = 3 * (int64_t)d.hd_total;
+        for (int idx = threadIdx.x; idx < 16 * (HD / 4); idx += blockDim.x) {
+            const int r = idx / (HD / 4), c4 = idx - r * (HD / 4);
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r < cnt) v = __ldcg(reinterpret_cast<const float4*>(a.qkv + (first + r) * ldq + head * HD) + c4);
+            *reinterpret_cast<float4*>(sQ + r * HD + ((c4 * 4) ^ ((r & 3) << 3))) = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = (i & 1) ? g8 + 8 : g8;
+                const int col = ks * 16 + 2 * t4 + ((i >> 1) ? 8 : 0);
+                const float2 x = *reinterpret_cast<const float2*>(sQ + row * HD + (col ^ ((row & 3) << 3)));
+                split_pack(x.x, x.y, qh[ks][i], ql[ks][i]);
+            }
+        }
+    }
+    const float scale = rsqrtf((float)HD);
+    const int wpos0 = warp * 32;
+    const int mi = lane >> 3, t8 = lane & 7;
+    const int r_lo = g8, r_hi = g8 + 8;
+    const int lim_lo = r_lo < cnt ? s_pos[r_lo] : -1;
+    const int lim_hi = r_hi < cnt ? s_pos[r_hi] : -1;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    float o[HD / 8][4];
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+
+#pragma unroll 1
+    for (int t = 0; t < n_tiles; ++t) {
+        const uint32_t par = (uint32_t)(t & 1);
+        if (threadIdx.x == 0 && !mbar_wait(bar_u, par)) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
+        __syncthreads();
+        if (flag[0]) break;  // uniform; what is still in flight is awaited below
+        if (t == 0 && threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 4);
+        float sc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+            const uint32_t (&ah)[4] = qh[ks];
+            const uint32_t (&al)[4] = ql[ks];
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+                const int row = wpos0 + np * 16 + (mi >> 1) * 8 + t8;
+                const int col = ks * 16 + (mi & 1) * 8;
+                const uint32_t kaddr = base + L::offK + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                       ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                uint32_t b[4];
+                ldsm_x4(kaddr, b);
+                mma_bf16(sc[2 * np], ah, b[0], b[1]);
+                mma_bf16(sc[2 * np], al, b[0], b[1]);
+                mma_bf16(sc[2 * np + 1], ah, b[2], b[3]);
+                mma_bf16(sc[2 * np + 1], al, b[2], b[3]);
+            }
+        }
+        __syncthreads();  // every warp has read the K tile: the next one may land in it
+        if (threadIdx.x == 0 && t + 1 < n_tiles) fetch_k(t + 1);
+        const int p0 = c0 + t * kAttnChunk + wpos0;
+        float bm_lo = -INFINITY, bm_hi = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int p = p0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                const int lim = e < 2 ? lim_lo : lim_hi;
+                const float v = p <= lim ? sc[nt][e] * scale : -INFINITY;
+                sc[nt][e] = v;
+                if (e < 2) bm_lo = fmaxf(bm_lo, v); else bm_hi = fmaxf(bm_hi, v);
+            }
+        }
+        bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 1)); bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 2));
+        bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 1)); bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 2));
+        const float n_lo = fmaxf(m_lo, bm_lo), n_hi = fmaxf(m_hi, bm_hi);
+        const float ref_lo = n_lo == -INFINITY ? 0.f : n_lo, ref_hi = n_hi == -INFINITY ? 0.f : n_hi;
+        const float f_lo = m_lo == -INFINITY ? 0.f : expf(m_lo - ref_lo);
+        const float f_hi = m_hi == -INFINITY ? 0.f : expf(m_hi - ref_hi);
+        float bl_lo = 0.f, bl_hi = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float pe = expf(sc[nt][e] - (e < 2 ? ref_lo : ref_hi));
+                sc[nt][e] = pe;
+                if (e < 2) bl_lo += pe; else bl_hi += pe;
+            }
+        }
+        bl_lo += __shfl_xor_sync(0xffffffffu, bl_lo, 1); bl_lo += __shfl_xor_sync(0xffffffffu, bl_lo, 2);
+        bl_hi += __shfl_xor_sync(0xffffffffu, bl_hi, 1); bl_hi += __shfl_xor_sync(0xffffffffu, bl_hi, 2);
+        l_lo = __fmaf_rn(l_lo, f_lo, bl_lo); l_hi = __fmaf_rn(l_hi, f_hi, bl_hi);
+        m_lo = n_lo; m_hi = n_hi;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) { o[i][0] *= f_lo; o[i][1] *= f_lo; o[i][2] *= f_hi; o[i][3] *= f_hi; }
+        if (threadIdx.x == 0 && !mbar_wait(bar_v, par)) { atomicExch(a.dev_err, kDevErrTimeout); flag[0] = 1; }
+        __syncthreads();
+        if (flag[0]) break;
+#pragma unroll
+        for (int kp = 0; kp < 2; ++kp) {
+            uint32_t ph[4], pl[4];
+            split_pack(sc[2 * kp][0], sc[2 * kp][1], ph[0], pl[0]);
+            split_pack(sc[2 * kp][2], sc[2 * kp][3], ph[1], pl[1]);
+            split_pack(sc[2 * kp + 1][0], sc[2 * kp + 1][1], ph[2], pl[2]);
+            split_pack(sc[2 * kp + 1][2], sc[2 * kp + 1][3], ph[3], pl[3]);
+#pragma unroll
+            for (int nn = 0; nn < HD / 16; ++nn) {
+                const int row = wpos0 + kp * 16 + (mi & 1) * 8 + t8;
+                const int col = nn * 16 + (mi >> 1) * 8;
+                const uint32_t vaddr = base + L::offV + (uint32_t)(col >> 6) * L::kBoxBytes + (uint32_t)row * 128 +
+                                       ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)row & 7u)) << 4);
+                uint32_t b[4];
+                ldsm_x4_trans(vaddr, b);
+                mma_bf16(o[2 * nn], ph, b[0], b[1]);
+                mma_bf16(o[2 * nn], pl, b[0], b[1]);
+                mma_bf16(o[2 * nn + 1], ph, b[2], b[3]);
+                mma_bf16(o[2 * nn + 1], pl, b[2], b[3]);
+            }
+        }
+        __syncthreads();  // every warp has read the V tile
+        if (threadIdx.x == 0 && t + 1 < n_tiles) fetch_v(t + 1);
+    }
+    if (flag[0]) {
+        // a copy never landed (error word is set): the K copy of the next tile may still be in flight
+        if (threadIdx.x == 0) {
+            (void)mbar_wait(bar_u, 0, 100000000ull); (void)mbar_wait(bar_u, 1, 100000000ull);
+            (void)mbar_wait(bar_v, 0, 100000000ull); (void)mbar_wait(bar_v, 1, 100000000ull);
+        }
+        return;
+    }
+    // ---------------- the four warps' (max, sum, output) combined in warp order -> the chunk's partial ----------------
+    const int64_t part_base = ((int64_t)head * a.n_chunks + chunk) * d.row_cap + first;
+    if ((lane & 3) == 0) {
+        s_m[warp * 16 + g8] = m_lo; s_m[warp * 16 + g8 + 8] = m_hi;
+        s_l[warp * 16 + g8] = l_lo; s_l[warp * 16 + g8 + 8] = l_hi;
+    }
+    {
+        float* buf = reinterpret_cast<float*>(gbase + L::offK) + warp * 16 * HD;  // the K tile is dead
+#pragma unroll
+        for (int nt = 0; nt < HD / 8; ++nt) {
+            const int col = nt * 8 + 2 * t4;
+            *reinterpret_cast<float2*>(buf + g8 * HD + (col ^ ((g8 & 3) << 3))) = make_float2(o[nt][0], o[nt][1]);
+            *reinterpret_cast<float2*>(buf + (g8 + 8) * HD + (col ^ ((g8 & 3) << 3))) = make_float2(o[nt][2], o[nt][3]);
+        }
+        __syncthreads();
+        const float* all = reinterpret_cast<const float*>(gbase + L::offK);
+        for (int e = threadIdx.x; e < cnt * (HD / 4); e += blockDim.x) {
+            const int r = e / (HD / 4), c4 = e - r * (HD / 4);
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) M = fmaxf(M, s_m[w * 16 + r]);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const float mw = s_m[w * 16 + r];
+                const float f = mw == -INFINITY ? 0.f : expf(mw - M);
+                const float4 v = *reinterpret_cast<const float4*>(all + (w * 16 + r) * HD + ((c4 * 4) ^ ((r & 3) << 3)));
+                if (w == 0) {
+                    acc = make_float4(__fmul_rn(f, v.x), __fmul_rn(f, v.y), __fmul_rn(f, v.z), __fmul_rn(f, v.w));
+                } else {
+                    acc.x = __fmaf_rn(f, v.x, acc.x); acc.y = __fmaf_rn(f, v.y, acc.y);
+                    acc.z = __fmaf_rn(f, v.z, acc.z); acc.w = __fmaf_rn(f, v.w, acc.w);
+                }
+            }
+            *reinterpret_cast<float4*>(a.ws_o + (part_base + r) * HD + c4 * 4) = acc;
+        }
+    }
+    if (threadIdx.x < cnt) {
+        const int r = threadIdx.x;
+        float M = -INFINITY;
+        for (int w = 0; w < 4; ++w) M = fmaxf(M, s_m[w * 16 + r]);
+        float lsum = 0.f;
+        for (int w = 0; w < 4; ++w) {
+            const float mw = s_m[w * 16 + r];
+            lsum += mw == -INFINITY ? 0.f : expf(mw - M) * s_l[w * 16 + r];
+        }
+        a.ws_ml[(part_base + r) * 2] = M;
+        a.ws_ml[(part_base + r) * 2 + 1] = lsum;
+    }
+    if (threadIdx.x == 0) LLMA_STAMP_MINMAX(stp, 6);
+}
+
 // Second pass: one warp per (head, row) combines the row's chunk partials in ascending chunk
 // order.  A kernel of its own, so that every head is merged at once instead of by whichever CTA of the
 // head happened to finish last; a row's result still depends on its own position only.
@@ -506,7 +757,7 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs a) 
     for (int u = 0; u < 16; ++u)
         p0[u] = u < a.n_chunks ? __ldcg(src + (int64_t)u * d.row_cap * (HD / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
     if (r >= rows_used || pos < 0) return;
-    const int nc = pos / kAttnChunk + 1;
+    const int nc = pos / a.chunk_pos + 1;
     float M = -INFINITY;
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
@@ -571,7 +822,19 @@ cudaError_t init_attention_mma() {
     e = cudaFuncSetAttribute(attention_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(AttnSmem<64>::kBytes + 1024));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attention_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attention_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<64>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attention_long_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<128>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attention_long_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<128>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attention_long_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(AttnSmem<64>::kBytes + 1024));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attention_long_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)(AttnSmem<64>::kBytes + 1024));
 }
 
@@ -579,6 +842,18 @@ void launch_attention_mma(cudaStream_t st, const AttnArgs& a, const CUtensorMap&
     dim3 grid(a.n_chunks, a.dims.n_heads, a.dims.max_batch);
     dim3 mgrid(a.dims.n_heads, (a.n_rows + 3) / 4);
     const size_t msmem = (size_t)8 * a.n_chunks * sizeof(float);
+    if (!a.prompt && a.tiles > 1) {  // long contexts, many sequences: several tiles per CTA
+        if (a.dims.head_dim == 128) {
+            if (a.tiles == 4) launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024, attention_long_kernel<128, 4>, a, map_k, map_v);
+            else launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024, attention_long_kernel<128, 2>, a, map_k, map_v);
+            launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<128>, a);
+        } else {
+            if (a.tiles == 4) launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_long_kernel<64, 4>, a, map_k, map_v);
+            else launch_pdl(st, true, grid, dim3(128), AttnSmem<64>::kBytes + 1024, attention_long_kernel<64, 2>, a, map_k, map_v);
+            launch_pdl(st, true, mgrid, dim3(128), msmem, attention_merge_kernel<64>, a);
+        }
+        return;
+    }
     if (a.dims.head_dim == 128) {
         if (a.prompt) launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128, true>, a, map_k, map_v);
         else launch_pdl(st, true, grid, dim3(128), AttnSmem<128>::kBytes + 1024 + kAttnPad, attention_mma_kernel<128, false>, a, map_k, map_v);

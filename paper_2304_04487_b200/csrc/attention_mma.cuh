@@ -11,7 +11,9 @@ constexpr int kAttnChunk = 128;  // cache positions per CTA; chunk c covers [128
 struct AttnArgs {
     ModelDims dims;
     int32_t layer;
-    int32_t n_chunks;        // grid.x = ceil(max_seq / 128); CTAs past a sequence's last position exit
+    int32_t n_chunks;        // grid.x = ceil(max_seq / chunk_pos); CTAs past a sequence's last position exit
+    int32_t tiles;           // 128-position tiles per CTA: 1, or 2 / 4 (attention_long_kernel; steps of at most 16 rows per sequence)
+    int32_t chunk_pos;       // cache positions per CTA = 128 * tiles
     const RowDesc* rows;
     const SeqState* seq_state;  // decode steps: kv_len here is the length committed before this step
     int32_t prompt;          // 1: a prompt pass (many rows of one sequence): the kernel instance with the per-warp query tiles

@@ -234,6 +234,13 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         CREATE_TRY(init_gemm_tcgen05());
         CREATE_TRY(init_gemm_wide());
         e->attn_chunks = (d.max_seq + kAttnChunk - 1) / kAttnChunk;
+        // With far more (sequence, head, 128-position tile) triples than CTAs fit on the GPU, a CTA takes several tiles in
+        // a row: fewer chunk partials, and the next tile's copies overlap the arithmetic.  A function of the engine's
+        // capacity only, so a row's result does not depend on the step.
+        {
+            const long long triples = (long long)d.max_batch * d.n_heads * e->attn_chunks, slots = 3LL * e->num_sms;
+            e->attn_tiles = (d.kp1 <= 16 && triples >= 16 * slots) ? 4 : ((d.kp1 <= 16 && triples >= 8 * slots) ? 2 : 1);
+        }
         const size_t parts = (size_t)d.n_heads * e->attn_chunks * RC;
         CREATE_TRY(dalloc(&e->attn_ws_o, parts * d.head_dim));
         CREATE_TRY(dalloc(&e->attn_ws_ml, parts * 2));

@@ -68,6 +68,7 @@ struct llma_engine {
     // tensor-core attention: TMA descriptors of the K/V cache, chunk partials
     CUtensorMap map_kcache, map_vcache;
     int attn_chunks = 0;
+    int attn_tiles = 1;             // 128-position tiles per attention CTA in decoding steps (a function of the capacity only)
     float *attn_ws_o = nullptr, *attn_ws_ml = nullptr;
 
     // replay of a given step sequence (llma_generate_forced)

@@ -141,6 +141,11 @@ extern "C" int llma_debug_timeline(llma_engine* e, int32_t clear, unsigned long 
     return LLMA_OK;
 }
 
+extern "C" int llma_debug_attention_tiles(llma_engine* e) {
+    if (!e) return LLMA_ERR_NULL;
+    return e->attn_tiles;
+}
+
 extern "C" int llma_row_capacity(llma_engine* e) {
     if (!e) return LLMA_ERR_NULL;
     return e->row_cap;

@@ -68,7 +68,10 @@ static void enqueue_forward_tc(llma_engine* e, bool lm_head) {
         run_gemm(e, q, m.wq, m.wk, m.wv, e->x_hat, am ? am->x_hat : nullptr);
         mark(e, LLMA_K_GEMM_QKV);
         AttnArgs at;
-        at.dims = d; at.layer = l; at.n_chunks = e->attn_chunks; at.rows = e->rows; at.qkv = e->qkv;
+        at.dims = d; at.layer = l; at.rows = e->rows; at.qkv = e->qkv;
+        at.tiles = lm_head ? e->attn_tiles : 1;  // prompt passes keep one tile per CTA
+        at.chunk_pos = kAttnChunk * at.tiles;
+        at.n_chunks = (d.max_seq + at.chunk_pos - 1) / at.chunk_pos;
         at.n_rows = e->cur_rows;
         at.attn_out = e->attn; at.ws_o = e->attn_ws_o; at.ws_ml = e->attn_ws_ml;
         at.dev_err = e->dev_err;

@@ -288,6 +288,31 @@ def test_adaptive_copy_length_stepwise_parity(name, B, k_max, adaptive):
     eng.llma_destroy()
 
 
+@pytest.mark.parametrize("max_seq,tiles", [(7300, 2), (14400, 4)])
+def test_long_context_batch_attention_tiles(max_seq, tiles):
+    """Engines whose capacity makes an attention CTA take several K/V tiles in a row (many sequences, long max_seq):
+    stepwise parity of 16 sequences whose contexts span one to several such chunks, ragged tails included."""
+    shape = SHAPES["tiny-bf16"]
+    w = _weights(shape)
+    B, k, N = 16, 4, 10
+    prompts = [make_prompt(90 + 61 * s, shape.vocab, seed=80 + s) for s in range(B)]     # 90 .. 1005 cached positions
+    refs, offs_list, models = [], [], []
+    o_seq = max(len(p) for p in prompts) + N + 2 * k + 8
+    for s in range(B):
+        y_star = D.greedy_decode(OM.OracleModel(shape, w, max_seq=o_seq), prompts[s], N).tokens
+        ref, offs, _ = build_reference(y_star, [24], 0.7, shape.vocab, seed=90 + s)
+        refs.append(ref); offs_list.append(offs)
+        models.append(OM.OracleModel(shape, w, max_seq=o_seq))
+    eng = _engine(shape, w, max_seq=max_seq, max_ref=32, max_k=k, max_batch=B, keep_logits=True)
+    assert eng.llma_debug_attention_tiles() == tiles
+    reps = step_parity_batch(eng, models, prompts, refs, offs_list, 1, k, N, "bf16")
+    assert sum(r.trigger_steps for r in reps) > 4
+    assert sum(r.near_ties for r in reps) <= 3
+    for r in reps:
+        assert r.max_logit_err <= 2e-2
+    eng.llma_destroy()
+
+
 def test_batched_generate_equals_single_sequence_runs():
     """llma_generate over 16 sequences: each output equals what the same sequence gives alone (greedy on a
     one-sequence engine), and the whole-loop statistics add up."""
