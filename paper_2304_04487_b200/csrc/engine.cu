@@ -236,10 +236,12 @@ extern "C" int llma_create(const llma_config* cfg, const llma_weights* w, void* 
         e->attn_chunks = (d.max_seq + kAttnChunk - 1) / kAttnChunk;
         // With far more (sequence, head, 128-position tile) triples than CTAs fit on the GPU, a CTA takes several tiles in
         // a row: fewer chunk partials, and the next tile's copies overlap the arithmetic.  A function of the engine's
-        // capacity only, so a row's result does not depend on the step.
+        // capacity only, so a row's result does not depend on the step.  Thresholds from the one-layer grid (batch x
+        // cached length): from four CTAs per resident slot on two tiles pay, from eight on four; at about one CTA per
+        // slot (one sequence, 2 k positions) two tiles cost 5 % of the step.
         {
             const long long triples = (long long)d.max_batch * d.n_heads * e->attn_chunks, slots = 3LL * e->num_sms;
-            e->attn_tiles = (d.kp1 <= 16 && triples >= 16 * slots) ? 4 : ((d.kp1 <= 16 && triples >= 8 * slots) ? 2 : 1);
+            e->attn_tiles = (d.kp1 <= 16 && triples >= 8 * slots) ? 4 : ((d.kp1 <= 16 && triples >= 4 * slots) ? 2 : 1);
         }
         const size_t parts = (size_t)d.n_heads * e->attn_chunks * RC;
         CREATE_TRY(dalloc(&e->attn_ws_o, parts * d.head_dim));

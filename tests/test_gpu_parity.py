@@ -288,7 +288,7 @@ def test_adaptive_copy_length_stepwise_parity(name, B, k_max, adaptive):
     eng.llma_destroy()
 
 
-@pytest.mark.parametrize("max_seq,tiles", [(7300, 2), (14400, 4)])
+@pytest.mark.parametrize("max_seq,tiles", [(5000, 2), (7300, 4)])
 def test_long_context_batch_attention_tiles(max_seq, tiles):
     """Engines whose capacity makes an attention CTA take several K/V tiles in a row (many sequences, long max_seq):
     stepwise parity of 16 sequences whose contexts span one to several such chunks, ragged tails included."""
