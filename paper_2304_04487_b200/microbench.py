@@ -2,6 +2,10 @@
 
     python -m paper_2304_04487_b200.microbench --n-out 22016 --k-in 4096 --iters 40
     python -m paper_2304_04487_b200.microbench --mma      # tensor-core time per MMA against N, regions, commits
+    python -m paper_2304_04487_b200.microbench --attention --batch 16 --history 4096 --k 8
+                                                          # one 7B-shaped layer, B sequences: per-kernel-class times of
+                                                          # a one-row and a (k+1)-row step; prints how many attention
+                                                          # launches precede them (for a profiler's launch-skip)
 
 Cycles through several weight buffers so that every launch streams its matrix from HBM
 (one matrix may fit in the 126 MB L2), times the launches with CUDA events on the launching
@@ -22,7 +26,30 @@ def main():
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--buffers", type=int, default=4)
     ap.add_argument("--mma", action="store_true")
+    ap.add_argument("--attention", action="store_true")
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--history", type=int, default=4096)
+    ap.add_argument("--k", type=int, default=8)
     a = ap.parse_args()
+    if a.attention:
+        from workloads import SHAPES, make_prompt, make_weights
+        from . import Engine
+        shape = SHAPES["llama7b-1layer"]
+        eng = Engine(shape, make_weights(shape, seed=0), max_seq=a.history + 100, max_ref=64, max_k=a.k, max_batch=a.batch)
+        for s_ in range(a.batch):
+            eng.llma_prefill(s_, make_prompt(a.history, shape.vocab, seed=100 + s_))
+        ys, _ = eng.llma_generate(24, 1, 0)
+        for s_ in range(a.batch):
+            eng.llma_set_reference(s_, ys[s_], None)     # every sequence then copies k tokens per step
+            eng.llma_rewind(s_)
+        before = a.batch * ((a.history - 1 + 127) // 128) + 24     # prompt passes + the greedy steps above (one layer)
+        out = {"attention_tiles_per_cta": eng.llma_debug_attention_tiles(), "attention_launches_before": before}
+        for kk in (0, a.k):
+            eng.llma_step(1, kk); eng.llma_step(1, kk)
+            pr = eng.llma_profile_steps(1, kk, 3)
+            out[f"k={kk}"] = {n: round(1e3 * v["ms_per_step"], 1) for n, v in pr.items()}
+        print(json.dumps(out))
+        return
     if a.mma:
         from . import llma_microbench_mma
         rows = []
