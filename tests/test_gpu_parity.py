@@ -288,11 +288,12 @@ def test_adaptive_copy_length_stepwise_parity(name, B, k_max, adaptive):
     eng.llma_destroy()
 
 
-@pytest.mark.parametrize("max_seq,tiles", [(5000, 2), (7300, 4)])
-def test_long_context_batch_attention_tiles(max_seq, tiles):
+@pytest.mark.parametrize("name,max_seq,tiles", [("tiny-bf16", 5000, 2), ("tiny-bf16", 7300, 4), ("small-bf16", 7300, 4)])
+def test_long_context_batch_attention_tiles(name, max_seq, tiles):
     """Engines whose capacity makes an attention CTA take several K/V tiles in a row (many sequences, long max_seq):
-    stepwise parity of 16 sequences whose contexts span one to several such chunks, ragged tails included."""
-    shape = SHAPES["tiny-bf16"]
+    stepwise parity of 16 sequences whose contexts span one to several such chunks, ragged tails included
+    (head_dim 64 and 128)."""
+    shape = SHAPES[name]
     w = _weights(shape)
     B, k, N = 16, 4, 10
     prompts = [make_prompt(90 + 61 * s, shape.vocab, seed=80 + s) for s in range(B)]     # 90 .. 1005 cached positions
