@@ -26,6 +26,8 @@
 // issuing work, lets its outstanding copies land, frees TMEM and returns.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "gemm_epilogue.cuh"
 #include "gemm_tcgen05.cuh"
 #include "ptx_sm100.cuh"
@@ -265,9 +267,9 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         }
         epi_sync();
         const float xnone[kXPre] = {};
-        // stage a 32-row block in shared memory (scaled by the folded RMSNorm), then the fused epilogue
-        auto finish_block = [&](int tile, int rb, float (&acc)[32]) {
-            const int jb = rb * 32, nj = min(32, rows_used - jb);
+        // stage up to 32 rows (jb .. jb + nj - 1, held in acc[0 .. nj - 1]) in shared memory, scaled by the folded
+        // RMSNorm, then the fused epilogue
+        auto finish_block = [&](int tile, int jb, int nj, float (&acc)[32]) {
             if (g.ss_in) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) stage[row][j] = acc[j] * rscale[min(jb + j, kRowCap - 1)];
@@ -293,9 +295,10 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
         };
         // Tiles cut by a range boundary are summed block by block: every CTA of such a tile writes its whole partial
         // (all-ones words while empty, see gemm_ws_kernel) into its own workspace slot -- slot 0 for the tile its
-        // range begins in, slot 1 for any other -- and the tile's 32-row blocks are dealt over its CTAs: after its
-        // last segment a CTA collects, for each block dealt to it, the partials of all the tile's CTAs in ascending
-        // k order (its own among them), puts all-ones back and runs the block's epilogue.  A tile cut into five
+        // range begins in, slot 1 for any other -- and the tile's rows are dealt over its CTAs in blocks of 32 (of 16
+        // where the tile has at least as many CTAs as 16-row blocks): after its last segment a CTA collects, for each
+        // block dealt to it, the partials of all the tile's CTAs in ascending k order (its own among them), puts
+        // all-ones back and runs the block's epilogue.  A tile cut into five
         // thus ends with five CTAs each finishing a fifth of it, instead of one CTA finishing all of it.
         constexpr uint32_t kEmpty = 0xFFFFFFFFu;
         // slots are laid out for the engine's row capacity whatever nr is: a prompt pass and a decoding step (different nr)
@@ -339,7 +342,7 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                     for (int q = 0; q < 8; ++q)  // only the columns of rows in use travel
                         if (rb * 32 + 4 * q < rows_used) dst[q * 128] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
                 } else {
-                    finish_block(tile, rb, acc);
+                    finish_block(tile, rb * 32, min(32, rows_used - rb * 32), acc);
                 }
             }
             tc_fence_before();
@@ -363,29 +366,31 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                 while (cta_begin(work, b_last + 1, G) <= t_hi - 1) ++b_last;
                 while (cta_begin(work, b_last, G) > t_hi - 1) --b_last;
                 const int P = b_last - b_first + 1, me = b - b_first;
-                for (int rb = 0; rb < nblk; ++rb) {
-                    if (rb * P / nblk != me) continue;  // dealt to another CTA of the tile
-                    const int jb = rb * 32;
+                // collect rows r_lo .. r_hi - 1 (NQ groups of four, starting at group q0 of 32-row block rb) from every
+                // CTA of the tile in ascending k order, then run their epilogue; NQ is a compile-time 8 or 4 so that
+                // the 32-row case carries no trace of the 16-row one
+                auto collect = [&](auto nq_tag, int r_lo, int r_hi, int rb, int q0) {
+                    constexpr int NQ = decltype(nq_tag)::value;
                     float acc[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) acc[j] = 0.f;
                     for (int bb = b_first; bb <= b_last; ++bb) {  // ascending k: a fixed summation order
                         const int slot = (int)(cta_begin(work, bb, G) / C) == tile ? 0 : 1;
-                        float4* src = ws_slot(g.ws, qn, bb, slot, row) + (int64_t)rb * 8 * 128;
-                        float4 p[8];
+                        float4* src = ws_slot(g.ws, qn, bb, slot, row) + ((int64_t)rb * 8 + q0) * 128;
+                        float4 p[NQ];
                         bool valid;
                         do {
                             valid = true;
 #pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                if (jb + 4 * q < rows_used) p[q] = ld_poll_f4(src + q * 128);
+                            for (int q = 0; q < NQ; ++q)
+                                if (r_lo + 4 * q < r_hi) p[q] = ld_poll_f4(src + q * 128);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                if (jb + 4 * q < rows_used) {
+                            for (int q = 0; q < NQ; ++q) {
+                                if (r_lo + 4 * q < r_hi) {
                                     valid = valid && __float_as_uint(p[q].x) != kEmpty;
-                                    if (jb + 4 * q + 1 < rows_used) valid = valid && __float_as_uint(p[q].y) != kEmpty;
-                                    if (jb + 4 * q + 2 < rows_used) valid = valid && __float_as_uint(p[q].z) != kEmpty;
-                                    if (jb + 4 * q + 3 < rows_used) valid = valid && __float_as_uint(p[q].w) != kEmpty;
+                                    if (r_lo + 4 * q + 1 < r_hi) valid = valid && __float_as_uint(p[q].y) != kEmpty;
+                                    if (r_lo + 4 * q + 2 < r_hi) valid = valid && __float_as_uint(p[q].z) != kEmpty;
+                                    if (r_lo + 4 * q + 3 < r_hi) valid = valid && __float_as_uint(p[q].w) != kEmpty;
                                 }
                             }
                             if (!valid && (timed_out || globaltimer_ns() > give_up)) {
@@ -394,14 +399,29 @@ gemm_wide_kernel(const GemmArgs g, const __grid_constant__ CUtensorMap map_a0, c
                         } while (!valid);
                         const float e = __uint_as_float(kEmpty);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            if (jb + 4 * q < rows_used) {
+                        for (int q = 0; q < NQ; ++q) {
+                            if (r_lo + 4 * q < r_hi) {
                                 src[q * 128] = make_float4(e, e, e, e);  // empty again for the next projection
                                 acc[4 * q] += p[q].x; acc[4 * q + 1] += p[q].y; acc[4 * q + 2] += p[q].z; acc[4 * q + 3] += p[q].w;
                             }
                         }
                     }
-                    finish_block(tile, rb, acc);
+                    finish_block(tile, r_lo, r_hi - r_lo, acc);
+                };
+                // units of 32 rows, or of 16 where that gives more of the tile's CTAs something to finish without
+                // giving any of them two units
+                if (nblk < P && ((rows_used + 15) >> 4) <= P) {
+                    const int n_units = (rows_used + 15) >> 4;
+                    for (int u = 0; u < n_units; ++u) {
+                        if (u * P / n_units != me) continue;  // dealt to another CTA of the tile
+                        const int r_lo = u * 16;
+                        collect(std::integral_constant<int, 4>{}, r_lo, min(rows_used, r_lo + 16), r_lo >> 5, (r_lo & 31) >> 2);
+                    }
+                } else {
+                    for (int rb = 0; rb < nblk; ++rb) {
+                        if (rb * P / nblk != me) continue;
+                        collect(std::integral_constant<int, 8>{}, rb * 32, min(rows_used, rb * 32 + 32), rb, 0);
+                    }
                 }
             }
         }
