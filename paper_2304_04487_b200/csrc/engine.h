@@ -52,7 +52,7 @@ struct llma_engine {
     bool decode_wide = false;       // decoding steps of more than 32 rows use gemm_wide_kernel
     int decode_nr = 32;             // rows the decoding GEMMs are shaped for (16 / 32 narrow, decode_rows wide)
     // what the launches being enqueued use (decoding step or prompt pass)
-    bool cur_wide = false;
+    bool cur_wide = false, cur_prompt = false;
     int cur_nr = 32, cur_rows = 32;
     const ActMaps* cur_maps = nullptr;
     int num_sms = 0;

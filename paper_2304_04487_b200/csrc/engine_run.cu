@@ -40,7 +40,10 @@ static GemmArgs gemm_args(llma_engine* e, int mode, int n_out, int n_tiles, int 
 static void run_gemm(llma_engine* e, GemmArgs& a, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
                      const void* act, const CUtensorMap* act_map) {
     a.act = act;
-    const int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
+    int grid = gemm_grid_for((int64_t)a.n_tiles * a.chunks, e->num_sms);
+    // Prompt passes (many rows: a tile's epilogue is long): where a projection has nearly as many tiles as there are
+    // SMs, one whole tile per CTA spares every tile the hand-over between the CTAs that would share it.
+    if (e->cur_wide && e->cur_prompt && a.n_tiles <= e->num_sms && 5 * a.n_tiles >= 3 * e->num_sms) grid = a.n_tiles;
     if (e->cur_wide) launch_gemm_wide(e->stream, grid, true, a, a0, a1, a2, act_map);
     else launch_gemm_tcgen05(e->stream, grid, true, a, a0, a1, a2);
 }
@@ -169,10 +172,12 @@ static void enqueue_embed(llma_engine* e) {
 
 // what the launches that follow are shaped for: a decoding step or a prompt pass
 static void shape_for_decode(llma_engine* e) {
+    e->cur_prompt = false;
     e->cur_wide = e->decode_wide; e->cur_nr = e->decode_nr; e->cur_rows = e->decode_rows;
     e->cur_maps = e->decode_wide ? &e->act_decode : nullptr;
 }
 static void shape_for_prefill(llma_engine* e) {
+    e->cur_prompt = true;
     e->cur_wide = e->gemm_impl == LLMA_GEMM_TCGEN05; e->cur_nr = e->prefill_rows; e->cur_rows = e->prefill_rows;
     e->cur_maps = e->cur_wide ? &e->act_prefill : nullptr;
 }
